@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the binarised-DNN forward pass on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config wsj]
+
+One step = one whole forward pass (every layer, through one bnn_forward call of the C ABI)
+over one batch of seeded synthetic frames.  Prints ONE JSON line on rank 0.
+With --impl reference the plain CPU oracle is timed instead (a slow, obviously correct
+program: a reported baseline, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "frames/sec for 6x2048 binarized DNN forward on 1 B200; XNOR-GEMM binary-op/s vs roofline"
+UNIT = "frames/s"
+L2_BYTES = 126 * 1024 * 1024
+SMS = 148
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="wsj", choices=["tiny", "wsj", "wsj_bw", "ami"])
+    ap.add_argument("--frames", type=int, default=None, help="override the batch size (frames per step)")
+    ap.add_argument("--cpu-frames", type=int, default=2048, help="frames of the workload the CPU oracle is timed on")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def workload_name(cfg, frames):
+    return "%s: %d frames x %d -> %d x %d -> %d log-softmax, %s" % (
+        cfg.name, frames, cfg.in_dim, cfg.n_hidden, cfg.hidden, cfg.classes,
+        "binary weights+activations" if cfg.act == 1 else "binary weights, hardtanh activations")
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                    sm_max_mhz=p.get("sm_max_mhz", 1965.0), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, sm_max_mhz=1965.0,
+                source="fallback")
+
+
+# ------------------------------------------------------------------ CPU oracle arm
+def oracle_step(cfg, net, X):
+    from oracle import bnn_oracle as o
+    return o.forward(X, net.W, net.scale, net.shift, net.Wout, net.bout,
+                     o.ACT_SIGN if cfg.act == 1 else o.ACT_HARDTANH, o.SIGN_ZERO_POS)
+
+
+def run_reference(args):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import bnn_oracle as o
+    from paper_1706_09453_b200 import workloads as wl
+    cfg = wl.CONFIGS[args.config]
+    frames = args.frames or cfg.frames
+    sample = min(frames, 256)       # frames per step: ~1.2 s of CPU work at WSJ scale on 8 cores
+    net = wl.make_model(cfg)
+    X = wl.make_frames(cfg, sample)
+    steps, warmup = max(1, min(args.steps, 40)), max(1, min(args.warmup, 3))
+    for _ in range(warmup):
+        oracle_step(cfg, net, X)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(cfg, net, X)
+    dt = time.perf_counter() - t0
+    fps = sample * steps / dt
+    desc = "first %d frames of the batch per step, %d steps" % (sample, steps)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(cfg, frames), "sample": desc},
+        "cpu_baseline": {"value": fps, "unit": UNIT, "cores": o.num_threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": fps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, torch, device_index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = torch.cuda.get_device_properties(device_index).uuid
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-%s" % uuid).encode())
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # NVML missing: report that, do not guess
+            self.nv, self.err = None, repr(e)
+
+    def _loop(self):
+        nv = self.nv
+        # NVML clocks-event (throttle) reason bits
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                 0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def start(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread:
+            self._stop.set()
+            self._thread.join()
+
+    def summary(self):
+        if not self.nv:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "error": self.err}
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": float(self.max_mhz), "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ roofline bookkeeping
+def layer_table(cfg, frames, peaks, sm_mhz):
+    """Per layer: algorithmic work, the pipe that bounds the kernel and its peak.
+
+    Algorithmic work: 2 binary ops per bit-MAC for XNOR layers, 2 flop per add/sub or MAC for
+    the real-valued layers.  Peaks of the integer / FP32 pipes are derived from unit counts:
+    per SM and clock 16 popcount lanes (x 32 bits x 2 bop) and 128 FP32 FMA lanes (x 2 flop),
+    at the maximum SM clock.
+    """
+    clk = peaks["sm_max_mhz"] * 1e6
+    popc_peak = SMS * 16 * 32 * 2 * clk / 1e12      # Tbop/s on the popcount pipe
+    fp32_peak = SMS * 128 * 2 * clk / 1e12          # TFLOP/s on the FP32 pipe
+    rows = []
+    k = cfg.in_dim
+    for l in range(cfg.n_hidden):
+        xnor = cfg.act == 1 and l > 0
+        work = 2.0 * frames * cfg.hidden * k
+        if xnor:
+            rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_popc_kernel", work=work, unit="Tbop/s",
+                             bound="alu", peak=popc_peak))
+        else:
+            rows.append(dict(name="signw_%d" % (l + 1), kernel="real_gemm_kernel", work=work, unit="TFLOP/s",
+                             bound="alu", peak=fp32_peak))
+        k = cfg.hidden
+    rows.append(dict(name="output", kernel="real_gemm_kernel+log_softmax_rows_kernel",
+                     work=2.0 * frames * cfg.classes * cfg.hidden, unit="TFLOP/s", bound="alu", peak=fp32_peak))
+    return rows
+
+
+def hbm_bytes_per_step(cfg, frames):
+    """Algorithmic HBM bytes of one forward: input, log-probs, weights once, activations."""
+    from paper_1706_09453_b200 import workloads as wl
+    b = frames * cfg.in_dim * 4 + frames * cfg.classes * 4
+    k = cfg.in_dim
+    for _ in range(cfg.n_hidden):
+        b += cfg.hidden * ((k + 31) // 32) * 4
+        b += 2 * frames * (cfg.hidden // 8 if cfg.act == wl.ACT_SIGN else cfg.hidden * 4)
+        k = cfg.hidden
+    b += cfg.classes * cfg.hidden * 4 + cfg.classes * 4
+    return b
+
+
+# ------------------------------------------------------------------ GPU arm
+def run_ours(args):
+    import torch
+    from paper_1706_09453_b200 import build
+    build.build()
+    from paper_1706_09453_b200 import binding as B, model, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = "cuda:%d" % local
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    cfg = wl.CONFIGS[args.config]
+    frames = args.frames or cfg.frames
+    net = wl.make_model(cfg)
+    dn = model.DeviceNet(net, device=dev)
+    # Frames are independent, so ranks shard them with no exchange: each rank owns its own batch.
+    Xh = wl.make_frames(cfg, frames, seed=cfg.seed + 1000 * rank)
+    set_bytes = frames * (cfg.in_dim + cfg.classes) * 4
+    nsets = max(2, -(-2 * L2_BYTES // set_bytes))          # rotate over > 2 x L2 of inputs/outputs
+    Xd = [model.to_dev(Xh, dev) for _ in range(nsets)]
+    Ld = [torch.empty((frames, cfg.classes), dtype=torch.float32, device=dev) for _ in range(nsets)]
+    ws = dn.workspace(frames)
+    K, W = args.steps, max(args.warmup, 3)
+
+    def step(i):
+        B.bnn_forward(dn.desc, Xd[i % nsets], Ld[i % nsets], ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(W):
+        step(i)
+    clocks = ClockSampler(torch, local)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    clocks.start()
+    e0.record()
+    for i in range(K):
+        step(i)
+    e1.record()
+    barrier()
+    clocks.stop()
+    ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if dist:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    total_ms = float(ms.item())
+
+    # ---- per-layer device time over the same steps (events recorded inside the C-ABI call)
+    nl = cfg.n_hidden + 1
+    Kp = min(K, 50)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nl + 1)] for _ in range(Kp)]
+    for row in evs:
+        for e in row:
+            e.record()
+    torch.cuda.synchronize()
+    for i in range(Kp):
+        B.bnn_forward_events(dn.desc, Xd[i % nsets], Ld[i % nsets], ws, evs[i])
+    torch.cuda.synchronize()
+    layer_ms = [float(np.mean([evs[i][l].elapsed_time(evs[i][l + 1]) for i in range(Kp)])) for l in range(nl)]
+
+    # ---- end to end: pinned host input -> device, forward, log-probs -> pinned host, every step
+    Ke = max(3, min(K, 20))
+    Xp = torch.from_numpy(Xh).pin_memory()
+    Lp = torch.empty((frames, cfg.classes), dtype=torch.float32).pin_memory()
+    for i in range(2):
+        Xd[0].copy_(Xp, non_blocking=True); step(0); Lp.copy_(Ld[0], non_blocking=True)
+    barrier()
+    e0.record()
+    for i in range(Ke):
+        Xd[i % nsets].copy_(Xp, non_blocking=True)
+        step(i)
+        Lp.copy_(Ld[i % nsets], non_blocking=True)
+    e1.record()
+    barrier()
+    ems = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if dist:
+        dist.all_reduce(ems, op=dist.ReduceOp.MAX)
+    e2e_fps = world * frames * Ke / (float(ems.item()) * 1e-3)
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    ck = clocks.summary()
+    rows = layer_table(cfg, frames, peaks, ck.get("sm_mhz"))
+    for r, t in zip(rows, layer_ms):
+        r["ms"] = t
+        r["achieved"] = r["work"] / (t * 1e-3) / 1e12
+        r["frac"] = r["achieved"] / r["peak"]
+    dom = max(rows, key=lambda r: r["ms"])
+    share = dom["ms"] / sum(layer_ms)
+    roofline = {"kernel": dom["kernel"], "layer": dom["name"], "bound": dom["bound"],
+                "achieved": dom["achieved"], "peak": dom["peak"], "unit": dom["unit"],
+                "frac": dom["frac"], "traffic": None,
+                "peak_source": "derived from unit counts x max SM clock (%.0f MHz)" % peaks["sm_max_mhz"],
+                "share_of_step": share, "avg_launch_ms": dom["ms"]}
+    fps = world * frames * K / (total_ms * 1e-3)
+    xnor_work = sum(r["work"] for r in rows if r["name"].startswith("xnor"))
+    xnor_ms = sum(r["ms"] for r in rows if r["name"].startswith("xnor"))
+    hbm = hbm_bytes_per_step(cfg, frames)
+    out = {
+        "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32 popcount (hidden layers) + f32 (first and top layer)", "data": "synthetic",
+        "config": {"workload": workload_name(cfg, frames), "frames_per_gpu": frames,
+                   "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 2 x L2); weights stay hot"
+                         % (nsets, nsets * set_bytes / 1e6),
+                   "sign_zero": "+1", "seed": cfg.seed},
+        "clocks": ck,
+        "e2e": {"value": e2e_fps, "unit": UNIT, "h2d_bytes_per_step": int(Xp.numel() * 4),
+                "d2h_bytes_per_step": int(Lp.numel() * 4), "steps": Ke},
+        "gpu_launches": K * (cfg.n_hidden + 2),
+        "roofline": roofline,
+        "layers": [{k: r[k] for k in ("name", "kernel", "ms", "achieved", "peak", "unit", "frac")} for r in rows],
+        "xnor_tbops": (xnor_work / (xnor_ms * 1e-3) / 1e12) if xnor_ms else None,
+        "hbm": {"algorithmic_bytes_per_step": hbm, "achieved_gbs": hbm / (total_ms / K * 1e-3) / 1e9,
+                "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"]},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import bnn_oracle as o
+        n = min(frames, args.cpu_frames)
+        t0 = time.perf_counter()
+        oracle_step(cfg, net, Xh[:n])
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": o.num_threads(), "kind": "oracle",
+                               "sample": "first %d frames of the batch, one pass (%.1f s)" % (n, dt)}
+    print(json.dumps(out))
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

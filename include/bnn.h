@@ -1,0 +1,214 @@
+/*
+ * bnn.h -- C ABI of the B200 (sm_100a) forward pass of a feed-forward acoustic-model DNN
+ * with binary (+-1) weights and activations (Lu, arXiv 1706.09453).
+ *
+ * Every step of the forward pass runs in this library's own CUDA kernels; there is no CPU
+ * path.  The library never allocates, frees or synchronises: the caller owns every buffer
+ * and work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *
+ * Unless an argument is marked HOST, every pointer is a DEVICE pointer.
+ *
+ * Storage conventions (the paper fixes none; these are this library's):
+ *   - real matrices are fp32 row-major with a row pitch `ld*` in floats;
+ *   - a binarised matrix stores one bit per element: bit = 1 <=> +1, bit = 0 <=> -1;
+ *     element k of a row is bit k%32 of the 32-bit word k/32 (LSB first);
+ *   - packed rows have a pitch `ld*p` in 32-bit words which is a multiple of 4, and packed
+ *     base pointers are 16-byte aligned, so every row starts on a 16-byte boundary;
+ *   - kernels that WRITE a packed row write words 0 .. ceil(K/32)-1 with the unused high
+ *     bits of the last word zero; pitch words beyond that are left untouched;
+ *   - kernels that READ a packed row ignore bits at positions >= K.
+ *
+ * Every entry point returns a bnn_status.  Arguments are validated on the host before any
+ * launch; a rejected call launches nothing.  Nothing throws or aborts across this ABI.
+ */
+#ifndef BNN_H_
+#define BNN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define BNN_API __attribute__((visibility("default")))
+#else
+#define BNN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BNN_OK = 0,
+    BNN_ERR_NULL = 1,        /* a required pointer is NULL */
+    BNN_ERR_SHAPE = 2,       /* a size is < 1, too large, or a pitch is smaller than its row */
+    BNN_ERR_ALIGN = 3,       /* base pointer or pitch breaks the alignment rules above */
+    BNN_ERR_UNSUPPORTED = 4, /* a combination of options this library does not implement */
+    BNN_ERR_WORKSPACE = 5,   /* workspace missing or too small */
+    BNN_ERR_CUDA = 6         /* the CUDA runtime reported an error at launch */
+} bnn_status;
+
+/* Value of Sign at zero.  Eq. 3 of the paper reads "+1 if x > 0, -1 otherwise", i.e.
+ * BNN_SIGN_ZERO_NEG.  BNN_SIGN_ZERO_POS is the other common convention (x >= 0 -> +1).
+ * NaN maps to -1 in both modes (every comparison with NaN is false). */
+typedef enum { BNN_SIGN_ZERO_POS = 0, BNN_SIGN_ZERO_NEG = 1 } bnn_sign_mode;
+
+/* What happens to a pre-activation after the per-unit affine (Eq. 2, h = f(h_hat)). */
+typedef enum {
+    BNN_ACT_NONE = 0,      /* write the value itself */
+    BNN_ACT_SIGN_PACK = 1, /* f = Sign (Algorithm 2), written as packed bits */
+    BNN_ACT_HARDTANH = 2   /* f = clamp to [-1, 1], written as fp32 */
+} bnn_act;
+
+/*
+ * Epilogue of a GEMM: the per-unit affine y_hat[n] = scale[n]*y[n] + shift[n] (Eq. 1 has
+ * only the bias r_l, i.e. scale = 1; a per-unit scale covers a folded normalisation), and
+ * the activation.  The affine is ONE fused multiply-add in fp32.
+ *
+ *   scale, shift : [N] or NULL (NULL scale = 1, NULL shift = 0); used by bnn_signw_gemm.
+ *   thr, flip    : used by bnn_xnor_gemm with BNN_ACT_SIGN_PACK.  Because the integer dot
+ *                  product d takes few values and d -> fma(scale, d, shift) is monotone,
+ *                  Sign(fma(scale[n], d, shift[n])) == ((d >= thr[n]) XOR flipbit[n]);
+ *                  bnn_fold_thresholds computes thr [N] and flip [ceil(N/32)] (bit n%32 of
+ *                  word n/32) so that this holds for EVERY integer d in [-K, K].
+ *   out_bits     : [M][ldob] packed result of BNN_ACT_SIGN_PACK.
+ *   sign_mode    : convention for Sign(0) (bnn_signw_gemm; the integer path has it folded
+ *                  into thr).
+ */
+typedef struct bnn_epilogue {
+    int act;
+    int sign_mode;
+    const float* scale;
+    const float* shift;
+    const int32_t* thr;
+    const uint32_t* flip;
+    uint32_t* out_bits;
+    int ldob;
+} bnn_epilogue;
+
+/* ------------------------------------------------------------------------------------
+ * Binarisation, Eq. 3 (w^b = Sign(w), Algorithm 1 forward, first statement of the loop).
+ * W : fp32 [N][ldw] real-valued weights.   Wp : uint32 [N][ldwp] packed signs (written).
+ * Errors: NULL -> BNN_ERR_NULL; N,K < 1, ldw < K, ldwp < ceil(K/32) -> BNN_ERR_SHAPE;
+ * ldwp % 4 != 0 or Wp not 16-byte aligned -> BNN_ERR_ALIGN.
+ */
+BNN_API int bnn_pack_weights(const float* W, int N, int K, int ldw, uint32_t* Wp, int ldwp,
+                     int sign_mode, void* stream);
+
+/* Same operation on a matrix of activations (Section 2.2 applies Eq. 3 to activations).
+ * X : fp32 [M][ldx].   Ap : uint32 [M][ldap] (written).  Errors as bnn_pack_weights. */
+BNN_API int bnn_binarize_pack(const float* X, int M, int K, int ldx, uint32_t* Ap, int ldap,
+                      int sign_mode, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Fold the affine + Sign of a binary hidden layer into integer thresholds (see
+ * bnn_epilogue).  scale, shift : [N] or NULL.  K : fan-in of the layer (d ranges over
+ * [-K, K]).  thr : int32 [N] (written).  flip : uint32 [ceil(N/32)] (written).
+ * The paper has no counterpart: it evaluates Sign(w h + r) directly (Algorithm 2).
+ */
+BNN_API int bnn_fold_thresholds(const float* scale, const float* shift, int N, int K, int sign_mode,
+                        int32_t* thr, uint32_t* flip, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Binary weights AND binary activations (Section 2.3): the product of Eq. 1 without the
+ * bias, d[m][n] = sum_k a[m][k]*w[n][k] with a, w in {-1,+1}
+ *             = K - 2*popcount(a_bits XOR w_bits).
+ * Ap : [M][ldap] packed activations.  Wp : [N][ldwp] packed weights.  1 <= K <= 2^24.
+ * C  : int32 [M][ldc] receives d, or NULL.
+ * epi: NULL, or act = BNN_ACT_SIGN_PACK with thr, flip, out_bits set: the next layer's
+ *      packed input h = Sign(scale*d + shift) (Eq. 2 with f = Sign) is written without the
+ *      integers ever leaving the chip.  At least one of C and epi must be given.
+ * Errors: as above; epi->act other than NONE / SIGN_PACK -> BNN_ERR_UNSUPPORTED.
+ */
+BNN_API int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
+                  int M, int N, int K, int32_t* C, int ldc,
+                  const bnn_epilogue* epi, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Binary weights against real-valued activations (Section 2.1; Algorithm 1 forward):
+ * y[m][n] = sum_k w^b[n][k]*x[m][k] -- additions and subtractions only -- followed by the
+ * epilogue: y_hat = fma(scale[n], y, shift[n]); then
+ *   BNN_ACT_NONE      : Y[m][n] = y_hat
+ *   BNN_ACT_HARDTANH  : Y[m][n] = min(max(y_hat, -1), 1)
+ *   BNN_ACT_SIGN_PACK : out_bits <- Sign(y_hat)   (Y may be NULL; if given it gets y_hat)
+ * X : fp32 [M][ldx].  Wp : [N][ldwp].  Y : fp32 [M][ldy] or NULL.  epi NULL = no affine,
+ * BNN_ACT_NONE.  Accumulation is fp32.
+ */
+BNN_API int bnn_signw_gemm(const float* X, int ldx, const uint32_t* Wp, int ldwp,
+                   int M, int N, int K, float* Y, int ldy,
+                   const bnn_epilogue* epi, void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Top layer (Section 2.3: the Softmax layer keeps real-valued weights; Algorithm 2, the
+ * branch l = L): z[m][c] = sum_n Wout[c][n]*h[m][n] + b[c], logp = z - logsumexp_c(z).
+ * Exactly one of Hp (packed +-1 activations [M][ldhp]) and Hf (fp32 [M][ldhf]) is given.
+ * Wout : fp32 [C][ldw].  b : [C] or NULL.  logp : fp32 [M][ldo] (written; holds the raw
+ * logits between the two internal passes).  log_softmax = 0 leaves the logits z.
+ */
+BNN_API int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
+                     const float* Wout, int ldw, const float* b,
+                     int M, int C, int H, float* logp, int ldo, int log_softmax,
+                     void* stream);
+
+/* ------------------------------------------------------------------------------------
+ * Whole forward pass: the loops "for l = 1 to L" of Algorithms 1 and 2.
+ */
+typedef enum {
+    BNN_LAYER_SIGNW = 0,   /* +-1 weights x real input (first layer; every hidden layer of
+                              a binary-weights-only network) */
+    BNN_LAYER_XNOR = 1,    /* +-1 weights x +-1 activations */
+    BNN_LAYER_REAL_OUT = 2 /* real-valued top layer + log-softmax; must be last */
+} bnn_layer_kind;
+
+typedef struct bnn_layer {
+    int kind;
+    int K, N;              /* fan-in, fan-out */
+    const uint32_t* Wp;    /* SIGNW, XNOR: packed weights [N][ldwp] */
+    int ldwp;
+    const float* W;        /* REAL_OUT: fp32 weights [N][ldw] */
+    int ldw;
+    const float* scale;    /* SIGNW: per-unit scale or NULL */
+    const float* shift;    /* SIGNW: per-unit shift or NULL; REAL_OUT: bias or NULL */
+    const int32_t* thr;    /* XNOR: folded thresholds [N] */
+    const uint32_t* flip;  /* XNOR: [ceil(N/32)] */
+    int act;               /* SIGNW: BNN_ACT_SIGN_PACK or BNN_ACT_HARDTANH; XNOR: SIGN_PACK */
+} bnn_layer;
+
+typedef struct bnn_model {
+    int n_layers;
+    int sign_mode;
+    const bnn_layer* layers; /* HOST array of n_layers entries (device pointers inside) */
+} bnn_model;
+
+/* Bytes of scratch bnn_forward needs for M frames (two ping-pong activation buffers). */
+BNN_API size_t bnn_forward_workspace_bytes(const bnn_model* model, int M);
+
+/*
+ * model : HOST struct.  X : fp32 [M][ldx] spliced features h_0.  logp : fp32 [M][ldo].
+ * workspace : device scratch, 256-byte aligned, >= bnn_forward_workspace_bytes(model, M).
+ * layer_out : HOST array of n_layers-1 device pointers or NULL; a non-NULL entry l makes
+ *   hidden layer l write its output there instead of into the workspace (packed bits with
+ *   pitch bnn_packed_pitch(N_l) words, or fp32 [M][N_l] for HARDTANH layers), which lets a
+ *   caller inspect every layer at no cost.
+ * Layer kinds must chain: SIGNW+SIGN_PACK -> XNOR; SIGNW+HARDTANH -> SIGNW or REAL_OUT;
+ * XNOR -> XNOR or REAL_OUT; the last layer is REAL_OUT.  Otherwise BNN_ERR_UNSUPPORTED.
+ */
+BNN_API int bnn_forward(const bnn_model* model, const float* X, int ldx, int M,
+                float* logp, int ldo, void* workspace, size_t workspace_bytes,
+                void* const* layer_out, void* stream);
+
+/* bnn_forward that also records events[l] (cudaEvent_t, HOST array of n_layers+1 entries,
+ * NULL entries skipped) on `stream` before layer l and events[n_layers] after the last
+ * kernel, so a caller can time each layer where it runs.  The paper has no counterpart. */
+BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
+                               float* logp, int ldo, void* workspace, size_t workspace_bytes,
+                               void* const* layer_out, void* const* events, void* stream);
+
+/* Smallest legal packed pitch (in words) for rows of K bits: ceil(K/32) rounded up to 4. */
+BNN_API int bnn_packed_pitch(int K);
+
+BNN_API const char* bnn_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BNN_H_ */

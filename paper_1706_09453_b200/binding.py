@@ -1,0 +1,231 @@
+"""Thin ctypes binding of the C ABI in ``include/bnn.h``.
+
+Argument marshalling only: every function takes torch CUDA tensors (device memory) and the
+current torch stream, calls the entry point of the same name and raises on a non-zero
+status.  There is no CPU path; a missing library or a CPU tensor is an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+SIGN_ZERO_POS, SIGN_ZERO_NEG = 0, 1
+ACT_NONE, ACT_SIGN_PACK, ACT_HARDTANH = 0, 1, 2
+LAYER_SIGNW, LAYER_XNOR, LAYER_REAL_OUT = 0, 1, 2
+
+
+class BnnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+
+
+class Epilogue(C.Structure):
+    _fields_ = [("act", C.c_int), ("sign_mode", C.c_int),
+                ("scale", C.c_void_p), ("shift", C.c_void_p),
+                ("thr", C.c_void_p), ("flip", C.c_void_p),
+                ("out_bits", C.c_void_p), ("ldob", C.c_int)]
+
+
+class Layer(C.Structure):
+    _fields_ = [("kind", C.c_int), ("K", C.c_int), ("N", C.c_int),
+                ("Wp", C.c_void_p), ("ldwp", C.c_int),
+                ("W", C.c_void_p), ("ldw", C.c_int),
+                ("scale", C.c_void_p), ("shift", C.c_void_p),
+                ("thr", C.c_void_p), ("flip", C.c_void_p),
+                ("act", C.c_int)]
+
+
+class Model(C.Structure):
+    _fields_ = [("n_layers", C.c_int), ("sign_mode", C.c_int), ("layers", C.POINTER(Layer))]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """Load the CUDA library; fails loudly if it has not been built."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not os.path.exists(path):
+            raise ImportError("CUDA library %s is missing: run paper_1706_09453_b200.build.build() "
+                              "(there is no CPU fallback)" % path)
+        L = C.CDLL(path)
+        L.bnn_status_string.restype = C.c_char_p
+        L.bnn_status_string.argtypes = [C.c_int]
+        L.bnn_packed_pitch.restype = C.c_int
+        L.bnn_packed_pitch.argtypes = [C.c_int]
+        L.bnn_forward_workspace_bytes.restype = C.c_size_t
+        L.bnn_forward_workspace_bytes.argtypes = [C.POINTER(Model), C.c_int]
+        i, p = C.c_int, C.c_void_p
+        L.bnn_pack_weights.argtypes = [p, i, i, i, p, i, i, p]
+        L.bnn_binarize_pack.argtypes = [p, i, i, i, p, i, i, p]
+        L.bnn_fold_thresholds.argtypes = [p, p, i, i, i, p, p, p]
+        L.bnn_xnor_gemm.argtypes = [p, i, p, i, i, i, i, p, i, C.POINTER(Epilogue), p]
+        L.bnn_signw_gemm.argtypes = [p, i, p, i, i, i, i, p, i, C.POINTER(Epilogue), p]
+        L.bnn_output_layer.argtypes = [p, i, p, i, p, i, p, i, i, i, p, i, i, p]
+        L.bnn_forward.argtypes = [C.POINTER(Model), p, i, i, p, i, p, C.c_size_t, C.POINTER(p), p]
+        L.bnn_forward_events.argtypes = [C.POINTER(Model), p, i, i, p, i, p, C.c_size_t, C.POINTER(p),
+                                         C.POINTER(p), p]
+        for name in ("bnn_pack_weights", "bnn_binarize_pack", "bnn_fold_thresholds", "bnn_xnor_gemm",
+                     "bnn_signw_gemm", "bnn_output_layer", "bnn_forward", "bnn_forward_events"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().bnn_status_string(int(status)).decode()
+
+
+def packed_pitch(k: int) -> int:
+    return int(lib().bnn_packed_pitch(int(k)))
+
+
+def _ptr(t, dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise TypeError("expected a CUDA tensor (there is no CPU path)")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("expected dtype %s, got %s" % (dtype, t.dtype))
+    return t.data_ptr()
+
+
+def _ld(t):
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError("expected a 2-D tensor with contiguous rows")
+    return t.stride(0)
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(rc, where):
+    if rc != 0:
+        raise BnnError(rc, where)
+
+
+def raw_call(name, *args) -> int:
+    """Call an entry point with raw integers/pointers and return its status (for tests)."""
+    return int(getattr(lib(), name)(*args))
+
+
+def bnn_pack_weights(W, Wp, sign_mode=SIGN_ZERO_POS):
+    n, k = W.shape
+    _check(lib().bnn_pack_weights(_ptr(W, torch.float32), n, k, _ld(W), _ptr(Wp, torch.int32), _ld(Wp),
+                                  sign_mode, _stream()), "bnn_pack_weights")
+    return Wp
+
+
+def bnn_binarize_pack(X, Ap, sign_mode=SIGN_ZERO_POS):
+    m, k = X.shape
+    _check(lib().bnn_binarize_pack(_ptr(X, torch.float32), m, k, _ld(X), _ptr(Ap, torch.int32), _ld(Ap),
+                                   sign_mode, _stream()), "bnn_binarize_pack")
+    return Ap
+
+
+def bnn_fold_thresholds(scale, shift, N, K, thr, flip, sign_mode=SIGN_ZERO_POS):
+    _check(lib().bnn_fold_thresholds(_ptr(scale, torch.float32), _ptr(shift, torch.float32), N, K, sign_mode,
+                                     _ptr(thr, torch.int32), _ptr(flip, torch.int32), _stream()),
+           "bnn_fold_thresholds")
+    return thr, flip
+
+
+def _epilogue(act=ACT_NONE, sign_mode=SIGN_ZERO_POS, scale=None, shift=None, thr=None, flip=None,
+              out_bits=None):
+    e = Epilogue()
+    e.act, e.sign_mode = act, sign_mode
+    e.scale, e.shift = _ptr(scale, torch.float32), _ptr(shift, torch.float32)
+    e.thr, e.flip = _ptr(thr, torch.int32), _ptr(flip, torch.int32)
+    e.out_bits = _ptr(out_bits, torch.int32)
+    e.ldob = _ld(out_bits) if out_bits is not None else 0
+    return e
+
+
+def bnn_xnor_gemm(Ap, Wp, K, C_out=None, thr=None, flip=None, out_bits=None):
+    """Packed tensors are int32 views of the uint32 words ([rows][pitch])."""
+    m, n = Ap.shape[0], Wp.shape[0]
+    e = None
+    if out_bits is not None:
+        e = C.byref(_epilogue(ACT_SIGN_PACK, thr=thr, flip=flip, out_bits=out_bits))
+    _check(lib().bnn_xnor_gemm(_ptr(Ap, torch.int32), _ld(Ap), _ptr(Wp, torch.int32), _ld(Wp), m, n, K,
+                               _ptr(C_out, torch.int32), _ld(C_out) if C_out is not None else 0,
+                               e, _stream()), "bnn_xnor_gemm")
+
+
+def bnn_signw_gemm(X, Wp, K, Y=None, act=ACT_NONE, scale=None, shift=None, out_bits=None,
+                   sign_mode=SIGN_ZERO_POS):
+    m, n = X.shape[0], Wp.shape[0]
+    e = C.byref(_epilogue(act, sign_mode, scale, shift, out_bits=out_bits))
+    _check(lib().bnn_signw_gemm(_ptr(X, torch.float32), _ld(X), _ptr(Wp, torch.int32), _ld(Wp), m, n, K,
+                                _ptr(Y, torch.float32), _ld(Y) if Y is not None else 0, e, _stream()),
+           "bnn_signw_gemm")
+
+
+def bnn_output_layer(Wout, b, logp, H, Hp=None, Hf=None, log_softmax=True):
+    m = (Hp if Hp is not None else Hf).shape[0]
+    c = Wout.shape[0]
+    _check(lib().bnn_output_layer(_ptr(Hp, torch.int32), _ld(Hp) if Hp is not None else 0,
+                                  _ptr(Hf, torch.float32), _ld(Hf) if Hf is not None else 0,
+                                  _ptr(Wout, torch.float32), _ld(Wout), _ptr(b, torch.float32),
+                                  m, c, H, _ptr(logp, torch.float32), _ld(logp), int(log_softmax), _stream()),
+           "bnn_output_layer")
+    return logp
+
+
+class ModelDesc:
+    """Host-side bnn_model built from a list of layer dicts; keeps the tensors alive."""
+
+    def __init__(self, layers, sign_mode=SIGN_ZERO_POS):
+        self._keep = layers
+        arr = (Layer * len(layers))()
+        for a, d in zip(arr, layers):
+            a.kind, a.K, a.N, a.act = d["kind"], d["K"], d["N"], d.get("act", ACT_NONE)
+            wp, w = d.get("Wp"), d.get("W")
+            a.Wp, a.ldwp = _ptr(wp, torch.int32), (_ld(wp) if wp is not None else 0)
+            a.W, a.ldw = _ptr(w, torch.float32), (_ld(w) if w is not None else 0)
+            a.scale, a.shift = _ptr(d.get("scale"), torch.float32), _ptr(d.get("shift"), torch.float32)
+            a.thr, a.flip = _ptr(d.get("thr"), torch.int32), _ptr(d.get("flip"), torch.int32)
+        self._arr = arr
+        self.c = Model(len(layers), sign_mode, arr)
+        self.layers = layers
+
+    def workspace_bytes(self, M: int) -> int:
+        return int(lib().bnn_forward_workspace_bytes(C.byref(self.c), M))
+
+
+def bnn_forward(model: ModelDesc, X, logp, workspace, layer_out=None):
+    m = X.shape[0]
+    lo = None
+    if layer_out is not None:
+        lo = (C.c_void_p * len(layer_out))(*[(_ptr(t) if t is not None else None) for t in layer_out])
+    _check(lib().bnn_forward(C.byref(model.c), _ptr(X, torch.float32), _ld(X), m,
+                             _ptr(logp, torch.float32), _ld(logp),
+                             _ptr(workspace), workspace.numel() * workspace.element_size(),
+                             lo, _stream()), "bnn_forward")
+    return logp
+
+
+def bnn_forward_events(model: ModelDesc, X, logp, workspace, events, layer_out=None):
+    """``events``: n_layers+1 recorded-at-least-once torch.cuda.Event objects (timing enabled)."""
+    m = X.shape[0]
+    lo = None
+    if layer_out is not None:
+        lo = (C.c_void_p * len(layer_out))(*[(_ptr(t) if t is not None else None) for t in layer_out])
+    ev = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+    _check(lib().bnn_forward_events(C.byref(model.c), _ptr(X, torch.float32), _ld(X), m,
+                                    _ptr(logp, torch.float32), _ld(logp),
+                                    _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                    lo, ev, _stream()), "bnn_forward_events")
+    return logp

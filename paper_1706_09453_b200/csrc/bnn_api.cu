@@ -1,0 +1,280 @@
+// extern "C" boundary: argument validation and kernel sequencing.  No allocation, no sync.
+#include <stdint.h>
+
+#include "bnn_common.cuh"
+
+using namespace bnn;
+
+namespace {
+
+constexpr int kMaxK = 1 << 24;  // |dot| <= K stays exact in every accumulator type used
+
+inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
+
+int check_packed(const void* p, int ld, int k) {
+    if (!p) return BNN_ERR_NULL;
+    if (ld < words_for(k)) return BNN_ERR_SHAPE;
+    if (ld % 4 != 0 || !aligned16(p)) return BNN_ERR_ALIGN;
+    return BNN_OK;
+}
+
+int check_dims(int a, int b, int c) {
+    if (a < 1 || b < 1 || c < 1) return BNN_ERR_SHAPE;
+    return BNN_OK;
+}
+
+int sign_pack_checked(const float* X, int R, int K, int ldx, uint32_t* P, int ldp, int mode,
+                      void* stream) {
+    if (!X || !P) return BNN_ERR_NULL;
+    if (R < 1 || K < 1 || ldx < K) return BNN_ERR_SHAPE;
+    if (mode != BNN_SIGN_ZERO_POS && mode != BNN_SIGN_ZERO_NEG) return BNN_ERR_UNSUPPORTED;
+    int rc = check_packed(P, ldp, K);
+    if (rc) return rc;
+    return launch_sign_pack(X, R, K, ldx, P, ldp, mode, (cudaStream_t)stream);
+}
+
+// Bytes of one hidden layer's output for M frames.
+size_t layer_out_bytes(const bnn_layer& L, int M) {
+    if (L.act == BNN_ACT_SIGN_PACK) return (size_t)M * bnn_packed_pitch(L.N) * sizeof(uint32_t);
+    return (size_t)M * L.N * sizeof(float);
+}
+
+int validate_model(const bnn_model* model) {
+    if (!model || !model->layers) return BNN_ERR_NULL;
+    const int L = model->n_layers;
+    if (L < 1) return BNN_ERR_SHAPE;
+    if (model->sign_mode != BNN_SIGN_ZERO_POS && model->sign_mode != BNN_SIGN_ZERO_NEG)
+        return BNN_ERR_UNSUPPORTED;
+    int prev_act = BNN_ACT_NONE;  // real-valued input h_0
+    int prev_n = -1;
+    for (int l = 0; l < L; ++l) {
+        const bnn_layer& y = model->layers[l];
+        if (y.K < 1 || y.N < 1 || y.K > kMaxK) return BNN_ERR_SHAPE;
+        if (prev_n >= 0 && y.K != prev_n) return BNN_ERR_SHAPE;
+        const bool in_bits = prev_act == BNN_ACT_SIGN_PACK;
+        switch (y.kind) {
+            case BNN_LAYER_SIGNW:
+                if (in_bits || l == L - 1) return BNN_ERR_UNSUPPORTED;
+                if (y.act != BNN_ACT_SIGN_PACK && y.act != BNN_ACT_HARDTANH) return BNN_ERR_UNSUPPORTED;
+                if (int rc = check_packed(y.Wp, y.ldwp, y.K)) return rc;
+                break;
+            case BNN_LAYER_XNOR:
+                if (!in_bits || l == L - 1) return BNN_ERR_UNSUPPORTED;
+                if (y.act != BNN_ACT_SIGN_PACK) return BNN_ERR_UNSUPPORTED;
+                if (!y.thr || !y.flip) return BNN_ERR_NULL;
+                if (int rc = check_packed(y.Wp, y.ldwp, y.K)) return rc;
+                break;
+            case BNN_LAYER_REAL_OUT:
+                if (l != L - 1) return BNN_ERR_UNSUPPORTED;
+                if (!y.W) return BNN_ERR_NULL;
+                if (y.ldw < y.K) return BNN_ERR_SHAPE;
+                break;
+            default:
+                return BNN_ERR_UNSUPPORTED;
+        }
+        prev_act = y.act;
+        prev_n = y.N;
+    }
+    if (model->layers[L - 1].kind != BNN_LAYER_REAL_OUT) return BNN_ERR_UNSUPPORTED;
+    return BNN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int bnn_packed_pitch(int K) { return (words_for(K) + 3) & ~3; }
+
+const char* bnn_status_string(int status) {
+    switch (status) {
+        case BNN_OK: return "ok";
+        case BNN_ERR_NULL: return "a required pointer is NULL";
+        case BNN_ERR_SHAPE: return "bad size or pitch";
+        case BNN_ERR_ALIGN: return "pointer or pitch breaks the 16-byte alignment rule";
+        case BNN_ERR_UNSUPPORTED: return "unsupported combination of options";
+        case BNN_ERR_WORKSPACE: return "workspace missing or too small";
+        case BNN_ERR_CUDA: return "CUDA runtime error at launch";
+        default: return "unknown status";
+    }
+}
+
+int bnn_pack_weights(const float* W, int N, int K, int ldw, uint32_t* Wp, int ldwp,
+                     int sign_mode, void* stream) {
+    return sign_pack_checked(W, N, K, ldw, Wp, ldwp, sign_mode, stream);
+}
+
+int bnn_binarize_pack(const float* X, int M, int K, int ldx, uint32_t* Ap, int ldap,
+                      int sign_mode, void* stream) {
+    return sign_pack_checked(X, M, K, ldx, Ap, ldap, sign_mode, stream);
+}
+
+int bnn_fold_thresholds(const float* scale, const float* shift, int N, int K, int sign_mode,
+                        int32_t* thr, uint32_t* flip, void* stream) {
+    if (!thr || !flip) return BNN_ERR_NULL;
+    if (N < 1 || K < 1 || K > kMaxK) return BNN_ERR_SHAPE;
+    if (sign_mode != BNN_SIGN_ZERO_POS && sign_mode != BNN_SIGN_ZERO_NEG) return BNN_ERR_UNSUPPORTED;
+    return launch_fold_thresholds(scale, shift, N, K, sign_mode, thr, flip, (cudaStream_t)stream);
+}
+
+int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
+                  int M, int N, int K, int32_t* C, int ldc,
+                  const bnn_epilogue* epi, void* stream) {
+    if (int rc = check_dims(M, N, K)) return rc;
+    if (K > kMaxK) return BNN_ERR_SHAPE;
+    if (int rc = check_packed(Ap, ldap, K)) return rc;
+    if (int rc = check_packed(Wp, ldwp, K)) return rc;
+    if (C && ldc < N) return BNN_ERR_SHAPE;
+    const int32_t* thr = nullptr;
+    const uint32_t* flip = nullptr;
+    uint32_t* ob = nullptr;
+    int ldob = 0;
+    if (epi && epi->act != BNN_ACT_NONE) {
+        if (epi->act != BNN_ACT_SIGN_PACK) return BNN_ERR_UNSUPPORTED;
+        if (!epi->thr || !epi->flip) return BNN_ERR_NULL;
+        if (int rc = check_packed(epi->out_bits, epi->ldob, N)) return rc;
+        thr = epi->thr; flip = epi->flip; ob = epi->out_bits; ldob = epi->ldob;
+    }
+    if (!C && !ob) return BNN_ERR_NULL;
+    return launch_xnor_popc(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, ob, ldob,
+                            (cudaStream_t)stream);
+}
+
+int bnn_signw_gemm(const float* X, int ldx, const uint32_t* Wp, int ldwp,
+                   int M, int N, int K, float* Y, int ldy,
+                   const bnn_epilogue* epi, void* stream) {
+    if (int rc = check_dims(M, N, K)) return rc;
+    if (!X) return BNN_ERR_NULL;
+    if (ldx < K) return BNN_ERR_SHAPE;
+    if (int rc = check_packed(Wp, ldwp, K)) return rc;
+    if (Y && ldy < N) return BNN_ERR_SHAPE;
+    RealGemmArgs a{};
+    a.Af = X; a.lda = ldx; a.Bb = Wp; a.ldb = ldwp;
+    a.M = M; a.N = N; a.K = K;
+    a.Y = Y; a.ldy = ldy;
+    a.act = BNN_ACT_NONE; a.sign_mode = BNN_SIGN_ZERO_POS;
+    if (epi) {
+        if (epi->act != BNN_ACT_NONE && epi->act != BNN_ACT_SIGN_PACK && epi->act != BNN_ACT_HARDTANH)
+            return BNN_ERR_UNSUPPORTED;
+        if (epi->sign_mode != BNN_SIGN_ZERO_POS && epi->sign_mode != BNN_SIGN_ZERO_NEG)
+            return BNN_ERR_UNSUPPORTED;
+        a.scale = epi->scale; a.shift = epi->shift; a.act = epi->act; a.sign_mode = epi->sign_mode;
+        if (epi->act == BNN_ACT_SIGN_PACK) {
+            if (int rc = check_packed(epi->out_bits, epi->ldob, N)) return rc;
+            a.out_bits = epi->out_bits; a.ldob = epi->ldob;
+        }
+    }
+    if (!a.Y && !a.out_bits) return BNN_ERR_NULL;
+    return launch_real_gemm(a, (cudaStream_t)stream);
+}
+
+int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
+                     const float* Wout, int ldw, const float* b,
+                     int M, int C, int H, float* logp, int ldo, int log_softmax,
+                     void* stream) {
+    if (int rc = check_dims(M, C, H)) return rc;
+    if (!Wout || !logp) return BNN_ERR_NULL;
+    if ((Hp == nullptr) == (Hf == nullptr)) return Hp ? BNN_ERR_UNSUPPORTED : BNN_ERR_NULL;
+    if (ldw < H || ldo < C) return BNN_ERR_SHAPE;
+    RealGemmArgs a{};
+    if (Hp) {
+        if (int rc = check_packed(Hp, ldhp, H)) return rc;
+        a.Ab = Hp; a.lda = ldhp;
+    } else {
+        if (ldhf < H) return BNN_ERR_SHAPE;
+        a.Af = Hf; a.lda = ldhf;
+    }
+    a.Bf = Wout; a.ldb = ldw;
+    a.M = M; a.N = C; a.K = H;
+    a.shift = b;
+    a.act = BNN_ACT_NONE;
+    a.Y = logp; a.ldy = ldo;
+    if (int rc = launch_real_gemm(a, (cudaStream_t)stream)) return rc;
+    if (log_softmax) return launch_log_softmax_rows(logp, ldo, M, C, (cudaStream_t)stream);
+    return BNN_OK;
+}
+
+size_t bnn_forward_workspace_bytes(const bnn_model* model, int M) {
+    if (validate_model(model) != BNN_OK || M < 1) return 0;
+    size_t mx = 0;
+    for (int l = 0; l + 1 < model->n_layers; ++l) {
+        size_t b = layer_out_bytes(model->layers[l], M);
+        if (b > mx) mx = b;
+    }
+    return 2 * round256(mx) + 256;
+}
+
+int bnn_forward(const bnn_model* model, const float* X, int ldx, int M,
+                float* logp, int ldo, void* workspace, size_t workspace_bytes,
+                void* const* layer_out, void* stream) {
+    return bnn_forward_events(model, X, ldx, M, logp, ldo, workspace, workspace_bytes, layer_out,
+                              nullptr, stream);
+}
+
+int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
+                       float* logp, int ldo, void* workspace, size_t workspace_bytes,
+                       void* const* layer_out, void* const* events, void* stream) {
+    if (int rc = validate_model(model)) return rc;
+    if (!X || !logp) return BNN_ERR_NULL;
+    if (M < 1 || ldx < model->layers[0].K) return BNN_ERR_SHAPE;
+    const int L = model->n_layers;
+    if (ldo < model->layers[L - 1].N) return BNN_ERR_SHAPE;
+    const size_t need = bnn_forward_workspace_bytes(model, M);
+    if (L > 1) {
+        if (!workspace || workspace_bytes < need) return BNN_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(workspace) & 255u) return BNN_ERR_ALIGN;
+    }
+    char* buf[2] = {static_cast<char*>(workspace),
+                    static_cast<char*>(workspace) + (need - 256) / 2};
+    const void* in = X;
+    int in_ld = ldx;
+    bool in_bits = false;
+    for (int l = 0; l < L; ++l) {
+        const bnn_layer& y = model->layers[l];
+        if (events && events[l] &&
+            cudaEventRecord((cudaEvent_t)events[l], (cudaStream_t)stream) != cudaSuccess)
+            return BNN_ERR_CUDA;
+        if (y.kind == BNN_LAYER_REAL_OUT) {
+            int rc = bnn_output_layer(in_bits ? static_cast<const uint32_t*>(in) : nullptr, in_ld,
+                                    in_bits ? nullptr : static_cast<const float*>(in), in_ld,
+                                    y.W, y.ldw, y.shift, M, y.N, y.K, logp, ldo, 1, stream);
+            if (rc) return rc;
+            if (events && events[L] &&
+                cudaEventRecord((cudaEvent_t)events[L], (cudaStream_t)stream) != cudaSuccess)
+                return BNN_ERR_CUDA;
+            return BNN_OK;
+        }
+        void* out = (layer_out && layer_out[l]) ? layer_out[l] : buf[l & 1];
+        if (y.act == BNN_ACT_SIGN_PACK && !aligned16(out)) return BNN_ERR_ALIGN;
+        bnn_epilogue e{};
+        e.act = y.act;
+        e.sign_mode = model->sign_mode;
+        int rc;
+        if (y.kind == BNN_LAYER_SIGNW) {
+            e.scale = y.scale; e.shift = y.shift;
+            float* yf = nullptr;
+            int out_ld;
+            if (y.act == BNN_ACT_SIGN_PACK) {
+                e.out_bits = static_cast<uint32_t*>(out); e.ldob = bnn_packed_pitch(y.N);
+                out_ld = e.ldob;
+            } else {
+                yf = static_cast<float*>(out);
+                out_ld = y.N;
+            }
+            rc = bnn_signw_gemm(static_cast<const float*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
+                                yf, y.N, &e, stream);
+            in_ld = out_ld;
+        } else {
+            e.thr = y.thr; e.flip = y.flip;
+            e.out_bits = static_cast<uint32_t*>(out); e.ldob = bnn_packed_pitch(y.N);
+            rc = bnn_xnor_gemm(static_cast<const uint32_t*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
+                               nullptr, 0, &e, stream);
+            in_ld = e.ldob;
+        }
+        if (rc) return rc;
+        in = out;
+        in_bits = y.act == BNN_ACT_SIGN_PACK;
+    }
+    return BNN_OK;
+}
+
+}  // extern "C"

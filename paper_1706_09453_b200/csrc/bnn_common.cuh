@@ -1,0 +1,74 @@
+// Shared device/host helpers of the sm_100a binarised-DNN forward library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bnn.h"
+
+namespace bnn {
+
+constexpr int kSignZeroPos = BNN_SIGN_ZERO_POS;
+constexpr int kSignZeroNeg = BNN_SIGN_ZERO_NEG;
+
+// Eq. 3: +1 iff x > 0 (ZERO_NEG, as printed) or x >= 0 (ZERO_POS).  NaN -> false.
+__device__ __forceinline__ bool sign_is_pos(float x, int mode) {
+    return mode == kSignZeroNeg ? (x > 0.0f) : (x >= 0.0f);
+}
+
+__host__ __device__ __forceinline__ int words_for(int k) { return (k + 31) >> 5; }
+__host__ __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Mask that keeps the valid bits of the last word of a K-bit row.
+__host__ __device__ __forceinline__ uint32_t tail_mask(int k) {
+    int t = k & 31;
+    return t ? ((1u << t) - 1u) : 0xFFFFFFFFu;
+}
+
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem, bool valid) {
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    int bytes = valid ? 16 : 0;  // src-size 0 => the 16 destination bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline int launch_status() { return cudaGetLastError() == cudaSuccess ? BNN_OK : BNN_ERR_CUDA; }
+
+// ---- launchers implemented in the .cu files (host side, arguments already validated) ----
+int launch_sign_pack(const float* X, int M, int K, int ldx, uint32_t* P, int ldp, int mode,
+                     cudaStream_t st);
+int launch_fold_thresholds(const float* scale, const float* shift, int N, int K, int mode,
+                           int32_t* thr, uint32_t* flip, cudaStream_t st);
+int launch_xnor_popc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
+                     int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
+                     uint32_t* out_bits, int ldob, cudaStream_t st);
+
+// Real-valued GEMM on the FP32 pipe: D[m][n] = sum_k A[m][k]*B[n][k], where each operand is
+// either fp32 or packed +-1 bits.
+struct RealGemmArgs {
+    const float* Af;      // fp32 A [M][lda] or nullptr
+    const uint32_t* Ab;   // packed A [M][lda] or nullptr
+    int lda;
+    const float* Bf;      // fp32 B [N][ldb] or nullptr
+    const uint32_t* Bb;   // packed B [N][ldb] or nullptr
+    int ldb;
+    int M, N, K;
+    const float* scale;   // [N] or nullptr
+    const float* shift;   // [N] or nullptr
+    int act;              // bnn_act
+    int sign_mode;
+    float* Y;             // fp32 out [M][ldy] or nullptr
+    int ldy;
+    uint32_t* out_bits;   // packed out [M][ldob] or nullptr
+    int ldob;
+};
+int launch_real_gemm(const RealGemmArgs& a, cudaStream_t st);
+int launch_log_softmax_rows(float* Z, int ldz, int M, int C, cudaStream_t st);
+
+}  // namespace bnn

@@ -1,0 +1,147 @@
+"""End-to-end parity of bnn_forward (one C-ABI call) with the CPU oracle on the synthetic
+WSJ / AMI shaped networks.
+
+The first layer is floating point: a unit whose pre-activation lies inside the float
+tolerance band (|y_hat| <= 1e-4 * |scale| * sum|x_i|) may legitimately binarise either way.
+So: (1) outside the band the first-layer bits must equal the oracle's; (2) the oracle then
+continues from the bits the GPU actually produced, and from there on every packed bit of
+every hidden layer must be identical and the log-probabilities within 1e-4."""
+import numpy as np
+import pytest
+
+from oracle import bnn_oracle as o
+from paper_1706_09453_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+FLOAT_TOL = 1e-4
+LOGP_TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_1706_09453_b200 import build, binding, model
+    build.build()
+    return torch, binding, model
+
+
+def run_binary_net(env, cfg, frames, mode=0, sample=None):
+    """Runs bnn_forward on `frames` frames; compares the frames in `sample` (all if None)."""
+    torch, B, model = env
+    net = wl.make_model(cfg)
+    X = wl.make_frames(cfg, frames)
+    dn = model.DeviceNet(net, mode)
+    outs = dn.layer_out_buffers(frames)
+    logp = dn.forward(model.to_dev(X), layer_out=outs)
+    torch.cuda.synchronize()
+    idx = np.arange(frames) if sample is None else np.asarray(sample)
+    gbits = [model.words_to_numpy(t, cfg.hidden)[idx] for t in outs]
+    glogp = logp.cpu().numpy()[idx]
+    # the packed weights themselves (Eq. 3 on the GPU) must equal the oracle's
+    ref = o.forward(X[idx], net.W, net.scale, net.shift, net.Wout, net.bout, o.ACT_SIGN, mode,
+                    layer1_bits=gbits[0])
+    for l, wp in enumerate(dn.Wp):
+        np.testing.assert_array_equal(model.words_to_numpy(wp, net.W[l].shape[1]), ref["Wp"][l])
+    # (1) first layer: equal outside the tolerance band
+    yh = ref["pre"][0]
+    band = FLOAT_TOL * np.abs(net.scale[0])[None, :] * ref["sumabs"][:, None]
+    own = o.unpack_pm1(ref["bits_own_layer1"], cfg.hidden)
+    got = o.unpack_pm1(gbits[0], cfg.hidden)
+    decided = np.abs(yh) > band
+    np.testing.assert_array_equal(got[decided], own[decided])
+    ambiguous = 1.0 - decided.mean()
+    assert ambiguous < 5e-3, ambiguous
+    # (2) everything downstream of the GPU's own first-layer bits is bit-exact
+    for l in range(1, cfg.n_hidden):
+        np.testing.assert_array_equal(gbits[l], ref["bits"][l], err_msg="hidden layer %d" % (l + 1))
+    err = np.abs(glogp - ref["logp"]).max()
+    assert err <= LOGP_TOL, err
+    return dict(ambiguous=ambiguous, flipped=float((got != own).mean()), logp_err=float(err))
+
+
+def test_forward_tiny_config_all_frames(env):
+    r = run_binary_net(env, wl.CONFIGS["tiny"], 256)
+    assert r["flipped"] <= r["ambiguous"]
+
+
+def test_forward_tiny_config_paper_sign_convention(env):
+    run_binary_net(env, wl.CONFIGS["tiny"], 256, mode=1)
+
+
+def test_forward_ragged_frame_count(env):
+    run_binary_net(env, wl.CONFIGS["tiny"], 131)
+
+
+def test_forward_single_frame(env):
+    run_binary_net(env, wl.CONFIGS["tiny"], 1)
+
+
+def test_forward_wsj_config_full_batch_sampled_frames(env):
+    """The benchmark's launch configuration (8192 frames); the oracle checks 600 of them,
+    including the first and last tile of frames."""
+    cfg = wl.CONFIGS["wsj"]
+    rng = np.random.default_rng(0)
+    sample = np.unique(np.concatenate([np.arange(128), np.arange(cfg.frames - 128, cfg.frames),
+                                       rng.integers(0, cfg.frames, 344)]))
+    run_binary_net(env, cfg, cfg.frames, sample=sample)
+
+
+def test_forward_ami_config_full_batch_sampled_frames(env):
+    cfg = wl.CONFIGS["ami"]
+    rng = np.random.default_rng(1)
+    sample = np.unique(np.concatenate([np.arange(64), np.arange(cfg.frames - 64, cfg.frames),
+                                       rng.integers(0, cfg.frames, 128)]))
+    run_binary_net(env, cfg, cfg.frames, sample=sample)
+
+
+def test_forward_unwritten_workspace_path_equals_layer_out_path(env):
+    """Without layer_out the activations go through the workspace: same log-probabilities."""
+    torch, B, model = env
+    cfg = wl.CONFIGS["tiny"]
+    dn = model.DeviceNet(wl.make_model(cfg))
+    X = model.to_dev(wl.make_frames(cfg, 200))
+    a = dn.forward(X).clone()
+    b = dn.forward(X, layer_out=dn.layer_out_buffers(200))
+    assert torch.equal(a, b)
+
+
+def run_bw_net(env, cfg, frames, sample=None):
+    torch, B, model = env
+    net = wl.make_model(cfg)
+    X = wl.make_frames(cfg, frames)
+    dn = model.DeviceNet(net)
+    outs = dn.layer_out_buffers(frames)
+    logp = dn.forward(model.to_dev(X), layer_out=outs)
+    torch.cuda.synchronize()
+    idx = np.arange(frames) if sample is None else np.asarray(sample)
+    ref = o.forward(X[idx], net.W, net.scale, net.shift, net.Wout, net.bout, o.ACT_HARDTANH)
+    # per-layer, teacher-forced: layer l of the GPU is fed the oracle's layer l-1 output
+    prev = X[idx]
+    for l in range(cfg.n_hidden):
+        y = torch.empty((len(idx), cfg.hidden), dtype=torch.float32, device="cuda:0")
+        B.bnn_signw_gemm(model.to_dev(prev), dn.Wp[l], net.W[l].shape[1], Y=y, act=B.ACT_HARDTANH,
+                         scale=dn.scale[l], shift=dn.shift[l])
+        tol = FLOAT_TOL * np.abs(net.scale[l])[None, :] * ref["sumabs_l"][l][:, None]
+        assert (np.abs(y.cpu().numpy() - ref["h"][l]) <= tol).all(), l
+        prev = ref["h"][l].astype(np.float32)
+    # end to end
+    err = np.abs(logp.cpu().numpy()[idx] - ref["logp"]).max()
+    assert err <= LOGP_TOL, err
+    herr = np.abs(outs[-1].cpu().numpy()[idx] - ref["h"][-1]).max()
+    assert herr <= 1e-4, herr
+
+
+def test_forward_binary_weights_only_small(env):
+    import dataclasses
+    cfg = dataclasses.replace(wl.CONFIGS["wsj_bw"], hidden=512, classes=700, frames=200)
+    run_bw_net(env, cfg, 200)
+
+
+def test_forward_binary_weights_only_wsj_config_sampled(env):
+    cfg = wl.CONFIGS["wsj_bw"]
+    rng = np.random.default_rng(2)
+    sample = np.unique(np.concatenate([np.arange(64), np.arange(cfg.frames - 64, cfg.frames),
+                                       rng.integers(0, cfg.frames, 128)]))
+    run_bw_net(env, cfg, cfg.frames, sample=sample)

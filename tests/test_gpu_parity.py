@@ -1,0 +1,290 @@
+"""Parity of the CUDA path (called through the C ABI) with the CPU oracle, element by
+element on the same seeded inputs.  Integers and packed bits must be bit-exact; floats
+within 1e-4 * sum|x_i| per output (first-layer / sign-weight GEMM) and 1e-4 absolute on
+log-probabilities."""
+import numpy as np
+import pytest
+
+from oracle import bnn_oracle as o
+from paper_1706_09453_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+FLOAT_TOL = 1e-4   # x sum_k |x[m][k]| per output
+LOGP_TOL = 1e-4    # absolute, on log-probabilities
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_1706_09453_b200 import build, binding
+    build.build()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def torch_():
+    import torch
+    return torch
+
+
+def dev(a):
+    from paper_1706_09453_b200.model import to_dev
+    return to_dev(a)
+
+
+def host_words(t, k):
+    from paper_1706_09453_b200.model import words_to_numpy
+    return words_to_numpy(t, k)
+
+
+def packed_canary(torch, rows, k, B, fill=0x5A5A5A5A):
+    return torch.full((rows, B.packed_pitch(k) + 4), fill, dtype=torch.int32, device="cuda:0")
+
+
+# ------------------------------------------------------------------ Sign + pack (Eq. 3)
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("shape", [(1, 1), (3, 31), (5, 32), (7, 33), (9, 127), (130, 440), (257, 600), (64, 2048)])
+def test_pack_matches_oracle(B, torch_, mode, shape):
+    m, k = shape
+    rng = np.random.default_rng(m * 1000 + k)
+    x = rng.standard_normal((m, k + 3)).astype(np.float32)   # pitch k+3: rows not 16-byte aligned
+    x[rng.random(x.shape) < 0.1] = 0.0
+    x[0, 0] = -0.0
+    if k > 4:
+        x[0, 1], x[0, 2], x[0, 3], x[0, 4] = np.nan, np.float32(1e-45), -np.float32(1e-45), np.inf
+    xd = dev(x)[:, :k]
+    out = packed_canary(torch_, m, k, B)
+    view = out[:, :B.packed_pitch(k)]
+    (B.bnn_binarize_pack if m % 2 else B.bnn_pack_weights)(xd, view, mode)
+    torch_.cuda.synchronize()
+    got = out.cpu().numpy().view(np.uint32)
+    kw = (k + 31) // 32
+    np.testing.assert_array_equal(got[:, :kw], o.sign_pack(x[:, :k], mode))
+    np.testing.assert_array_equal(got[:, kw:], 0x5A5A5A5A)   # pitch words untouched
+
+
+def test_pack_vectorised_path_aligned_rows(B, torch_):
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((300, 440)).astype(np.float32)
+    out = packed_canary(torch_, 300, 440, B)
+    B.bnn_binarize_pack(dev(x), out[:, :16], 0)
+    got = out.cpu().numpy().view(np.uint32)
+    np.testing.assert_array_equal(got[:, :14], o.sign_pack(x, 0))
+    np.testing.assert_array_equal(got[:, 14:], 0x5A5A5A5A)
+
+
+# ------------------------------------------------------------------ threshold fold
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("k", [1, 64, 441])
+def test_fold_thresholds_exhaustive(B, torch_, mode, k):
+    """(d >= thr) xor flip == Sign(fma(scale, d, shift)) for EVERY integer d in [-K, K]."""
+    rng = np.random.default_rng(k)
+    n = 200
+    scale = rng.uniform(-1.5, 1.5, n).astype(np.float32)
+    shift = rng.normal(0, 0.3 * k, n).astype(np.float32)
+    scale[:8] = [0.0, -0.0, 1.0, -1.0, 1e-30, -1e-30, 1e30, -1e30]
+    shift[:4] = [0.0, -0.0, 0.0, 0.0]
+    shift[8:12] = [1e30, -1e30, float(k), -float(k)]
+    scale[12:16] = [1.0, 1.0, -1.0, -1.0]
+    shift[12:16] = [2.0, -2.0, 2.0, -2.0]      # exact zeros at d = -+2
+    s = np.float32(1.0) + np.float32(2.0 ** -23)
+    scale[16], shift[16] = s, -np.float32(s * np.float32(3))   # fma vs two roundings
+    thr = torch_.empty(n, dtype=torch_.int32, device="cuda:0")
+    flip = torch_.empty((n + 31) // 32, dtype=torch_.int32, device="cuda:0")
+    B.bnn_fold_thresholds(dev(scale), dev(shift), n, k, thr, flip, mode)
+    thr = thr.cpu().numpy().astype(np.int64)
+    fw = flip.cpu().numpy().view(np.uint32)
+    fb = ((fw[np.arange(n) // 32] >> (np.arange(n) % 32).astype(np.uint32)) & 1).astype(bool)
+    d = np.arange(-k, k + 1, dtype=np.int32)
+    D = np.repeat(d[:, None], n, 1)
+    want = o.unpack_pm1(o.affine_sign_pack_i32(D, scale, shift, mode), n) == 1
+    got = (D >= thr[None, :]) ^ fb[None, :]
+    np.testing.assert_array_equal(got, want)
+
+
+def test_fold_thresholds_null_scale_shift(B, torch_):
+    thr = torch_.empty(40, dtype=torch_.int32, device="cuda:0")
+    flip = torch_.empty(2, dtype=torch_.int32, device="cuda:0")
+    B.bnn_fold_thresholds(None, None, 40, 100, thr, flip, 0)
+    assert (thr.cpu().numpy() == 0).all() and (flip.cpu().numpy() == 0).all()
+    B.bnn_fold_thresholds(None, None, 40, 100, thr, flip, 1)
+    assert (thr.cpu().numpy() == 1).all()
+
+
+# ------------------------------------------------------------------ XNOR GEMM
+XNOR_SHAPES = [(1, 1, 1), (2, 3, 31), (5, 7, 32), (17, 9, 33), (129, 130, 127), (300, 257, 1000),
+               (256, 1024, 1024), (131, 1024, 440), (200, 129, 600), (640, 384, 2048)]
+
+
+@pytest.mark.parametrize("shape", XNOR_SHAPES)
+@pytest.mark.parametrize("p", [0.5, 0.1])
+def test_xnor_gemm_int32_bit_exact(B, torch_, shape, p):
+    m, n, k = shape
+    ap = wl.make_bit_planes(m, k, p, [1, m, n, k], B.packed_pitch(k))
+    wp = wl.make_bit_planes(n, k, p, [2, m, n, k], B.packed_pitch(k))
+    c = torch_.full((m, n + 5), -77, dtype=torch_.int32, device="cuda:0")
+    B.bnn_xnor_gemm(dev(ap), dev(wp), k, C_out=c[:, :n])
+    got = c.cpu().numpy()
+    np.testing.assert_array_equal(got[:, :n], o.xnor_gemm(ap, wp, k))
+    np.testing.assert_array_equal(got[:, n:], -77)
+
+
+def test_xnor_gemm_ignores_garbage_in_pad_bits(B, torch_):
+    m, n, k = 70, 90, 1000 - 13
+    pitch = B.packed_pitch(k) + 4
+    ap = wl.make_bit_planes(m, k, 0.5, 11, pitch)
+    wp = wl.make_bit_planes(n, k, 0.5, 12, pitch)
+    want = o.xnor_gemm(ap, wp, k)
+    kw = (k + 31) // 32
+    rng = np.random.default_rng(0)
+    ap2, wp2 = ap.copy(), wp.copy()
+    ap2[:, kw:] = rng.integers(0, 2**32, (m, pitch - kw), dtype=np.uint32)
+    wp2[:, kw:] = rng.integers(0, 2**32, (n, pitch - kw), dtype=np.uint32)
+    ap2[:, kw - 1] |= np.uint32(0xFFFFFFFF << (k % 32) & 0xFFFFFFFF)
+    wp2[:, kw - 1] |= rng.integers(0, 2**32, n, dtype=np.uint32) & np.uint32(0xFFFFFFFF << (k % 32) & 0xFFFFFFFF)
+    c = torch_.empty((m, n), dtype=torch_.int32, device="cuda:0")
+    B.bnn_xnor_gemm(dev(ap2), dev(wp2), k, C_out=c)
+    np.testing.assert_array_equal(c.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("shape", [(5, 7, 33), (129, 130, 127), (300, 257, 1000), (256, 1024, 1024), (131, 96, 440)])
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("with_c", [False, True])
+def test_xnor_gemm_fused_sign_pack_bit_exact(B, torch_, shape, mode, with_c):
+    m, n, k = shape
+    rng = np.random.default_rng(m + n + k)
+    ap = wl.make_bit_planes(m, k, 0.5, [3, m, n, k], B.packed_pitch(k))
+    wp = wl.make_bit_planes(n, k, 0.5, [4, m, n, k], B.packed_pitch(k))
+    scale = rng.uniform(0.5, 1.5, n).astype(np.float32)
+    shift = rng.normal(0, 0.1, n).astype(np.float32)
+    scale[::7] *= -1                      # negative scales flip the comparison
+    scale[1::11] = 0.0
+    shift[2::5] = np.round(shift[2::5] * 20)   # integer shifts with scale...
+    scale[2::5] = 1.0                          # ... 1 make exact zeros likely
+    thr = torch_.empty(n, dtype=torch_.int32, device="cuda:0")
+    flip = torch_.empty((n + 31) // 32, dtype=torch_.int32, device="cuda:0")
+    B.bnn_fold_thresholds(dev(scale), dev(shift), n, k, thr, flip, mode)
+    out = packed_canary(torch_, m, n, B)
+    c = torch_.empty((m, n), dtype=torch_.int32, device="cuda:0") if with_c else None
+    B.bnn_xnor_gemm(dev(ap), dev(wp), k, C_out=c, thr=thr, flip=flip, out_bits=out[:, :B.packed_pitch(n)])
+    d = o.xnor_gemm(ap, wp, k)
+    want = o.affine_sign_pack_i32(d, scale, shift, mode)
+    got = out.cpu().numpy().view(np.uint32)
+    nw = (n + 31) // 32
+    np.testing.assert_array_equal(got[:, :nw], want)
+    np.testing.assert_array_equal(got[:, nw:], 0x5A5A5A5A)
+    if with_c:
+        np.testing.assert_array_equal(c.cpu().numpy(), d)
+    if mode == 0 and m * n > 100000:
+        assert (d[:, 2::5].astype(np.float32) + shift[2::5] == 0).any(), "no exact zero was exercised"
+
+
+# ------------------------------------------------------------------ +-1 weights x real input
+@pytest.mark.parametrize("shape", [(1, 1, 1), (3, 5, 33), (130, 129, 440), (257, 300, 600), (64, 256, 2048)])
+def test_signw_gemm_within_tolerance(B, torch_, shape):
+    m, n, k = shape
+    rng = np.random.default_rng(m * n + k)
+    x = rng.standard_normal((m, k)).astype(np.float32)
+    w = rng.standard_normal((n, k)).astype(np.float32)
+    wp = o.sign_pack(w, 0, B.packed_pitch(k))
+    y = torch_.full((m, n + 3), 123.0, dtype=torch_.float32, device="cuda:0")
+    B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y[:, :n])
+    got = y.cpu().numpy()
+    ref, sumabs = o.signw_gemm(x, wp, k)
+    err = np.abs(got[:, :n] - ref)
+    assert (err <= FLOAT_TOL * sumabs[:, None]).all(), err.max()
+    np.testing.assert_array_equal(got[:, n:], 123.0)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_signw_gemm_sign_pack_epilogue(B, torch_, mode):
+    m, n, k = 200, 300, 440
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((m, k)).astype(np.float32)
+    wp = wl.make_bit_planes(n, k, 0.5, 21, B.packed_pitch(k))
+    scale = rng.uniform(0.5, 1.5, n).astype(np.float32)
+    scale[::9] *= -1
+    shift = rng.normal(0, 0.1, n).astype(np.float32)
+    out = packed_canary(torch_, m, n, B)
+    y = torch_.empty((m, n), dtype=torch_.float32, device="cuda:0")
+    B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y, act=B.ACT_SIGN_PACK, scale=dev(scale), shift=dev(shift),
+                     out_bits=out[:, :B.packed_pitch(n)], sign_mode=mode)
+    ref, sumabs = o.signw_gemm(x, wp, k)
+    yh, _, bits = o.affine_act_f64(ref, scale, shift, o.ACT_SIGN, mode)
+    tol = FLOAT_TOL * np.abs(scale)[None, :] * sumabs[:, None]
+    assert (np.abs(y.cpu().numpy() - yh) <= tol + 1e-6).all()
+    got = out.cpu().numpy().view(np.uint32)
+    nw = (n + 31) // 32
+    gs, ws = o.unpack_pm1(got[:, :nw], n), o.unpack_pm1(bits, n)
+    decided = np.abs(yh) > tol          # outside the band the bit is determined
+    np.testing.assert_array_equal(gs[decided], ws[decided])
+    assert decided.mean() > 0.99
+    np.testing.assert_array_equal(got[:, nw:], 0x5A5A5A5A)
+    # the bits are exactly the Sign of the fp32 values the kernel itself reports
+    yv = y.cpu().numpy()
+    own = np.where((yv > 0) if mode == 1 else (yv >= 0), 1, -1)
+    np.testing.assert_array_equal(gs, own)
+
+
+def test_signw_gemm_exact_zero_follows_sign_mode(B, torch_):
+    """Integer-valued inputs make y exactly 0 for some units; the bit must follow the mode."""
+    m, n, k = 40, 64, 64
+    rng = np.random.default_rng(3)
+    x = rng.integers(-2, 3, (m, k)).astype(np.float32)
+    wp = wl.make_bit_planes(n, k, 0.5, 22, B.packed_pitch(k))
+    ref, _ = o.signw_gemm(x, wp, k)
+    assert (ref == 0).any()
+    for mode in (0, 1):
+        out = packed_canary(torch_, m, n, B)
+        B.bnn_signw_gemm(dev(x), dev(wp), k, act=B.ACT_SIGN_PACK, out_bits=out[:, :4], sign_mode=mode)
+        _, _, bits = o.affine_act_f64(ref, None, None, o.ACT_SIGN, mode)
+        np.testing.assert_array_equal(out.cpu().numpy().view(np.uint32)[:, :2], bits)
+
+
+def test_signw_gemm_hardtanh_epilogue(B, torch_):
+    m, n, k = 150, 200, 2048
+    rng = np.random.default_rng(4)
+    x = rng.uniform(-1, 1, (m, k)).astype(np.float32)
+    wp = wl.make_bit_planes(n, k, 0.5, 23, B.packed_pitch(k))
+    scale = np.full(n, 0.05, np.float32)
+    y = torch_.empty((m, n), dtype=torch_.float32, device="cuda:0")
+    B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y, act=B.ACT_HARDTANH, scale=dev(scale))
+    ref, sumabs = o.signw_gemm(x, wp, k)
+    _, h, _ = o.affine_act_f64(ref, scale, None, o.ACT_HARDTANH)
+    got = y.cpu().numpy()
+    assert (np.abs(got - h) <= FLOAT_TOL * 0.05 * sumabs[:, None]).all()
+    assert got.min() >= -1.0 and got.max() <= 1.0 and (got == 1.0).any() and (got == -1.0).any()
+
+
+# ------------------------------------------------------------------ top layer
+@pytest.mark.parametrize("c", [10, 2000, 3307, 3972])
+def test_output_layer_bits_logp(B, torch_, c):
+    m, h = 70, 1024
+    rng = np.random.default_rng(c)
+    hp = wl.make_bit_planes(m, h, 0.5, 31, B.packed_pitch(h))
+    wout = rng.normal(0, 1 / np.sqrt(h), (c, h)).astype(np.float32)
+    b = rng.normal(0, 0.1, c).astype(np.float32)
+    z = torch_.full((m, c + 1), 9.0, dtype=torch_.float32, device="cuda:0")
+    B.bnn_output_layer(dev(wout), dev(b), z[:, :c], h, Hp=dev(hp), log_softmax=False)
+    zr = o.real_gemm_bits(hp, wout, b, h)
+    assert np.abs(z.cpu().numpy()[:, :c] - zr).max() <= FLOAT_TOL * h
+    lp = torch_.full((m, c + 1), 9.0, dtype=torch_.float32, device="cuda:0")
+    B.bnn_output_layer(dev(wout), dev(b), lp[:, :c], h, Hp=dev(hp))
+    got = lp.cpu().numpy()
+    assert np.abs(got[:, :c] - o.log_softmax(zr)).max() <= LOGP_TOL
+    np.testing.assert_array_equal(got[:, c], 9.0)
+    np.testing.assert_allclose(np.exp(got[:, :c].astype(np.float64)).sum(1), 1.0, atol=1e-4)
+
+
+def test_output_layer_real_activations(B, torch_):
+    m, h, c = 33, 300, 257
+    rng = np.random.default_rng(8)
+    hf = rng.uniform(-1, 1, (m, h)).astype(np.float32)
+    wout = rng.normal(0, 1 / np.sqrt(h), (c, h)).astype(np.float32)
+    b = rng.normal(0, 0.1, c).astype(np.float32)
+    lp = torch_.empty((m, c), dtype=torch_.float32, device="cuda:0")
+    B.bnn_output_layer(dev(wout), dev(b), lp, h, Hf=dev(hf))
+    want = o.log_softmax(o.real_gemm_f32(hf, wout, b))
+    assert np.abs(lp.cpu().numpy() - want).max() <= LOGP_TOL
