@@ -39,6 +39,8 @@ def parse_args():
     ap.add_argument("--frames", type=int, default=None, help="override the batch size (frames per step)")
     ap.add_argument("--cpu-frames", type=int, default=2048, help="frames of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--xnor-path", default="tensor", choices=["tensor", "popc"],
+                    help="kernel of the binary hidden layers: tcgen05 tensor core or integer-pipe popcount")
     return ap.parse_args()
 
 
@@ -151,7 +153,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ roofline bookkeeping
-def layer_table(cfg, frames, peaks, sm_mhz):
+def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor"):
     """Per layer: algorithmic work, the pipe that bounds the kernel and its peak.
 
     Algorithmic work: 2 binary ops per bit-MAC for XNOR layers, 2 flop per add/sub or MAC for
@@ -167,7 +169,12 @@ def layer_table(cfg, frames, peaks, sm_mhz):
     for l in range(cfg.n_hidden):
         xnor = cfg.act == 1 and l > 0
         work = 2.0 * frames * cfg.hidden * k
-        if xnor:
+        if xnor and xnor_path == "tensor":
+            # u8 x u8 tensor-core MACs: 2 x the measured bf16 rate (nominal ratio), sustained
+            # figure because the kernel is timed inside a long step; 1 bit-MAC = 2 bop
+            rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_tc_kernel", work=work, unit="Tbop/s",
+                             bound="tensor", peak=2.0 * peaks["bf16_tflops_sustained"]))
+        elif xnor:
             rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_popc_kernel", work=work, unit="Tbop/s",
                              bound="alu", peak=popc_peak))
         else:
@@ -214,6 +221,7 @@ def run_ours(args):
     cfg = wl.CONFIGS[args.config]
     frames = args.frames or cfg.frames
     net = wl.make_model(cfg)
+    B.bnn_set_xnor_path(B.XNOR_TENSOR if args.xnor_path == "tensor" else B.XNOR_POPC)
     dn = model.DeviceNet(net, device=dev)
     # Frames are independent, so ranks shard them with no exchange: each rank owns its own batch.
     Xh = wl.make_frames(cfg, frames, seed=cfg.seed + 1000 * rank)
@@ -289,7 +297,7 @@ def run_ours(args):
 
     peaks = load_peaks()
     ck = clocks.summary()
-    rows = layer_table(cfg, frames, peaks, ck.get("sm_mhz"))
+    rows = layer_table(cfg, frames, peaks, ck.get("sm_mhz"), args.xnor_path)
     for r, t in zip(rows, layer_ms):
         r["ms"] = t
         r["achieved"] = r["work"] / (t * 1e-3) / 1e12
@@ -299,7 +307,9 @@ def run_ours(args):
     roofline = {"kernel": dom["kernel"], "layer": dom["name"], "bound": dom["bound"],
                 "achieved": dom["achieved"], "peak": dom["peak"], "unit": dom["unit"],
                 "frac": dom["frac"], "traffic": None,
-                "peak_source": "derived from unit counts x max SM clock (%.0f MHz)" % peaks["sm_max_mhz"],
+                "peak_source": ("2 x bf16_tflops_sustained of MEASURED_PEAKS.json (%s)" % peaks["source"])
+                if dom["bound"] == "tensor" else
+                "derived from unit counts x max SM clock (%.0f MHz)" % peaks["sm_max_mhz"],
                 "share_of_step": share, "avg_launch_ms": dom["ms"]}
     fps = world * frames * K / (total_ms * 1e-3)
     xnor_work = sum(r["work"] for r in rows if r["name"].startswith("xnor"))
@@ -308,7 +318,9 @@ def run_ours(args):
     out = {
         "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32 popcount (hidden layers) + f32 (first and top layer)", "data": "synthetic",
+        "dtype": "%s (hidden layers) + f32 (first and top layer)"
+                 % ("u8 tensor-core MMA, s32 accumulate" if args.xnor_path == "tensor" else "int32 popcount"),
+        "device_status": B.bnn_device_status(), "data": "synthetic",
         "config": {"workload": workload_name(cfg, frames), "frames_per_gpu": frames,
                    "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 2 x L2); weights stay hot"
                          % (nsets, nsets * set_bytes / 1e6),

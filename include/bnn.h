@@ -203,6 +203,20 @@ BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, 
                                float* logp, int ldo, void* workspace, size_t workspace_bytes,
                                void* const* layer_out, void* const* events, void* stream);
 
+/* Which kernel bnn_xnor_gemm (and the XNOR layers of bnn_forward) use.  Both compute the
+ * same integers: BNN_XNOR_POPC is the XOR/popcount kernel on the integer pipes,
+ * BNN_XNOR_TENSOR the tcgen05 tensor-core kernel (needs K <= 2^22; larger K falls back to
+ * popcount).  BNN_XNOR_AUTO picks the faster one as measured on B200 (tensor).
+ * Process-wide setting; returns the previous value, or -1 for an unknown `path`. */
+typedef enum { BNN_XNOR_AUTO = 0, BNN_XNOR_POPC = 1, BNN_XNOR_TENSOR = 2 } bnn_xnor_path;
+BNN_API int bnn_set_xnor_path(int path);
+
+/* Tensor-core kernels bound every wait they perform; a CTA whose wait runs out stops, frees
+ * its tensor memory and sets a status word.  This call SYNCHRONISES the device and stores
+ * that word in *status (HOST pointer): 0 = no kernel gave up, 1 = one did (results of the
+ * affected launch are invalid).  The paper has no counterpart. */
+BNN_API int bnn_device_status(int* status);
+
 /* Smallest legal packed pitch (in words) for rows of K bits: ceil(K/32) rounded up to 4. */
 BNN_API int bnn_packed_pitch(int K);
 

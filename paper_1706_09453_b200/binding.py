@@ -64,6 +64,10 @@ def lib():
         L.bnn_status_string.argtypes = [C.c_int]
         L.bnn_packed_pitch.restype = C.c_int
         L.bnn_packed_pitch.argtypes = [C.c_int]
+        L.bnn_set_xnor_path.argtypes = [C.c_int]
+        L.bnn_set_xnor_path.restype = C.c_int
+        L.bnn_device_status.argtypes = [C.POINTER(C.c_int)]
+        L.bnn_device_status.restype = C.c_int
         L.bnn_forward_workspace_bytes.restype = C.c_size_t
         L.bnn_forward_workspace_bytes.argtypes = [C.POINTER(Model), C.c_int]
         i, p = C.c_int, C.c_void_p
@@ -89,6 +93,23 @@ def status_string(status: int) -> str:
 
 def packed_pitch(k: int) -> int:
     return int(lib().bnn_packed_pitch(int(k)))
+
+
+XNOR_AUTO, XNOR_POPC, XNOR_TENSOR = 0, 1, 2
+
+
+def bnn_set_xnor_path(path: int) -> int:
+    prev = int(lib().bnn_set_xnor_path(int(path)))
+    if prev < 0:
+        raise ValueError("unknown XNOR path %r" % path)
+    return prev
+
+
+def bnn_device_status() -> int:
+    """Synchronises the device; 0 unless a tensor-core kernel gave up on a bounded wait."""
+    st = C.c_int(-1)
+    _check(lib().bnn_device_status(C.byref(st)), "bnn_device_status")
+    return st.value
 
 
 def _ptr(t, dtype=None):

@@ -7,7 +7,8 @@ using namespace bnn;
 
 namespace {
 
-constexpr int kMaxK = 1 << 24;  // |dot| <= K stays exact in every accumulator type used
+constexpr int kMaxK = 1 << 24;
+int g_xnor_path = BNN_XNOR_AUTO;  // |dot| <= K stays exact in every accumulator type used
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -85,6 +86,18 @@ extern "C" {
 
 int bnn_packed_pitch(int K) { return (words_for(K) + 3) & ~3; }
 
+int bnn_set_xnor_path(int path) {
+    if (path != BNN_XNOR_AUTO && path != BNN_XNOR_POPC && path != BNN_XNOR_TENSOR) return -1;
+    const int prev = g_xnor_path;
+    g_xnor_path = path;
+    return prev;
+}
+
+int bnn_device_status(int* status) {
+    if (!status) return BNN_ERR_NULL;
+    return read_tc_status(status);
+}
+
 const char* bnn_status_string(int status) {
     switch (status) {
         case BNN_OK: return "ok";
@@ -135,8 +148,9 @@ int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
         thr = epi->thr; flip = epi->flip; ob = epi->out_bits; ldob = epi->ldob;
     }
     if (!C && !ob) return BNN_ERR_NULL;
-    return launch_xnor_popc(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, ob, ldob,
-                            (cudaStream_t)stream);
+    const bool tensor = g_xnor_path != BNN_XNOR_POPC && K <= kMaxKTensor;
+    return (tensor ? launch_xnor_tc : launch_xnor_popc)(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip,
+                                                        ob, ldob, (cudaStream_t)stream);
 }
 
 int bnn_signw_gemm(const float* X, int ldx, const uint32_t* Wp, int ldwp,

@@ -49,6 +49,14 @@ int launch_xnor_popc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
                      int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
                      uint32_t* out_bits, int ldob, cudaStream_t st);
 
+// Tensor-core (tcgen05) XNOR GEMM; same contract as launch_xnor_popc.  K <= kMaxKTensor.
+constexpr int kMaxKTensor = 1 << 22;
+int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
+                   int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
+                   uint32_t* out_bits, int ldob, cudaStream_t st);
+// Reads (synchronously) the word that a tensor-core kernel sets when a bounded wait ran out.
+int read_tc_status(int* out);
+
 // Real-valued GEMM on the FP32 pipe: D[m][n] = sum_k A[m][k]*B[n][k], where each operand is
 // either fp32 or packed +-1 bits.
 struct RealGemmArgs {

@@ -1,0 +1,369 @@
+// XNOR GEMM on the 5th-generation tensor cores (tcgen05, kind::i8, accumulators in TMEM).
+//
+// Identity used: with bits a, w in {0,1} standing for -1/+1,
+//     dot = K - 2 popc(a) - 2 popc(w) + 4 popc(a AND w),
+// and popc(a AND w) is an ordinary integer dot product of the bit vectors, i.e. a dense
+// contraction the tensor core can do.  Packed bits stay 1 bit per element in HBM/L2; they
+// are widened to bytes only inside the SM, on the way into shared memory:
+//   - the contraction index may be permuted freely as long as A and W use the same
+//     permutation, so byte j of output word (w_i, t) is simply bit 8j+t of packed word w_i:
+//     one AND with the mask 0x01010101 << t widens 4 bits to 4 bytes;
+//   - that leaves the byte holding 2^t instead of 1.  A keeps 2^t, W is bit-reversed within
+//     bytes first so its byte holds 2^(7-t); every product is then 2^7 * a * w and the
+//     accumulator is exactly 128 * popc(a AND w) (u8 x u8 -> s32).
+//
+// One persistent CTA per SM, tile 128 frames x 256 units, 128 bits of K per pipeline stage.
+// Warp roles: warps 0-3 epilogue (TMEM -> thresholds -> packed bits / int32), warp 4 issues
+// the MMAs, warps 5-16 are producers (one packed row each per stage).  Two accumulator
+// buffers in TMEM (2 x 256 columns) let the epilogue of tile i overlap the MMAs of tile i+1.
+#include "bnn_common.cuh"
+#include "tcgen05.cuh"
+
+namespace bnn {
+
+__device__ int g_tc_status = 0;  // set to 1 by a CTA whose bounded wait ran out
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 256, BK = 128;  // BK: bits of K per stage = bytes per widened row
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int EPI_WARPS = 4, MMA_WARP = 4, PROD_WARP0 = 5, PROD_WARPS = 12;
+constexpr int THREADS = (PROD_WARP0 + PROD_WARPS) * 32;  // 544
+constexpr int PREFETCH = 3;                              // packed words in flight per producer
+constexpr uint32_t TMEM_COLS = 512;
+
+struct Control {
+    int T[BN];              // per-unit constant of the epilogue (threshold or 2 popc(w) - K)
+    uint32_t flipw[BN / 32];
+    uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + (int)sizeof(Control) + 128;
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// AND of a predicate over the 128 epilogue threads (named barrier 2)
+__device__ __forceinline__ bool epi_all(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "barrier.red.and.pred q, 2, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"((uint32_t)pred) : "memory");
+    return r != 0;
+}
+
+// One lane waits, the whole warp gets the same answer.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+}
+
+// popcount of the valid bits of one packed row
+__device__ __forceinline__ int row_popc(const uint32_t* __restrict__ row, int kw, uint32_t tmask) {
+    int s = 0;
+    const int full4 = (kw - 1) >> 2;  // 16-byte chunks that lie entirely before the last word
+    for (int q = 0; q < full4; ++q) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(row) + q);
+        s += __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
+    }
+    for (int k = full4 << 2; k < kw; ++k) {
+        uint32_t v = __ldg(row + k);
+        if (k == kw - 1) v &= tmask;
+        s += __popc(v);
+    }
+    return s;
+}
+
+template <bool STORE_C, bool SIGN_PACK>
+__global__ void __launch_bounds__(THREADS, 1)
+xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __restrict__ Wp, int ldwp,
+               int M, int N, int K, int32_t* __restrict__ C, int ldc,
+               const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
+               uint32_t* __restrict__ out_bits, int ldob) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES);
+    volatile int* abort_flag = &ctl->abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int kw = words_for(K);
+    const uint32_t tmask = tail_mask(K);
+    const int nks = ceil_div(K, BK);
+    const int m_tiles = ceil_div(M, BM), n_tiles = ceil_div(N, BN);
+    const int tiles = m_tiles * n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), PROD_WARPS);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
+        }
+        ctl->abort = 0;
+        mbar_init_fence();
+    }
+    if (warp == MMA_WARP) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ctl->tmem_base;
+
+    if (warp >= PROD_WARP0) {
+        // ---------------- producers: packed words -> widened byte tiles in shared memory
+        const int p = threadIdx.x - PROD_WARP0 * 32;  // 0..383
+        const bool is_a = p < BM;
+        const int r = is_a ? p : p - BM;
+        const uint32_t* base = is_a ? Ap : Wp;
+        const int ld = is_a ? ldap : ldwp;
+        const int rows = is_a ? M : N;
+        const int rows_tile = is_a ? BM : BN;
+        const uint32_t dst_off = (is_a ? 0 : A_BYTES) + r * 16;
+        const int my_tiles = (tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
+        const int total = my_tiles * nks;  // stages this CTA runs
+
+        // prefetch cursor: stage `pf_ks` of this CTA's tile number `pf_tl`
+        int pf_i = 0, pf_ks = 0, pf_tile = blockIdx.x;
+        auto fetch = [&]() -> uint4 {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (pf_i < total) {
+                const int row = (is_a ? (pf_tile % m_tiles) * BM : (pf_tile / m_tiles) * BN) + r;
+                const int k0 = pf_ks * 4;  // first word of this stage
+                if (row < rows && k0 < kw) {
+                    v = __ldg(reinterpret_cast<const uint4*>(base + (size_t)row * ld + k0));
+                    const int last = kw - 1 - k0;  // index of the last valid word in this chunk
+                    if (last == 0) { v.x &= tmask; v.y = 0u; v.z = 0u; v.w = 0u; }
+                    else if (last == 1) { v.y &= tmask; v.z = 0u; v.w = 0u; }
+                    else if (last == 2) { v.z &= tmask; v.w = 0u; }
+                    else if (last == 3) { v.w &= tmask; }
+                }
+                ++pf_i;
+                if (++pf_ks == nks) { pf_ks = 0; pf_tile += gridDim.x; }
+            }
+            return v;
+        };
+
+        uint4 ring[PREFETCH];
+#pragma unroll
+        for (int j = 0; j < PREFETCH; ++j) ring[j] = fetch();
+        for (int it = 0; it < total; ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (uint32_t)((it / STAGES) & 1);
+            uint4 v = ring[0];
+#pragma unroll
+            for (int j = 0; j + 1 < PREFETCH; ++j) ring[j] = ring[j + 1];
+            ring[PREFETCH - 1] = fetch();
+            if (!is_a) {  // reverse the bits inside each byte
+                v.x = __brev(__byte_perm(v.x, 0, 0x0123));
+                v.y = __brev(__byte_perm(v.y, 0, 0x0123));
+                v.z = __brev(__byte_perm(v.z, 0, 0x0123));
+                v.w = __brev(__byte_perm(v.w, 0, 0x0123));
+            }
+            if (!warp_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag, lane)) break;
+            uint8_t* dst = smem + s * STAGE_BYTES + dst_off;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const uint32_t mk = is_a ? (0x01010101u << t) : (0x01010101u << (7 - t));
+                *reinterpret_cast<uint4*>(dst + t * (rows_tile * 16)) =
+                    make_uint4(v.x & mk, v.y & mk, v.z & mk, v.w & mk);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
+        }
+    } else if (warp == MMA_WARP) {
+        // ---------------- MMA issue: one thread
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc(kAccS32, kFmtU8, kFmtU8, BM, BN);
+            int it = 0;
+            int tl = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
+                const int b = tl & 1;
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), (uint32_t)(((tl >> 1) & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t d = tmem + (uint32_t)(b * BN);
+                for (int ks = 0; ks < nks; ++ks, ++it) {
+                    const int s = it % STAGES;
+                    ok = mbar_wait(smem_u32(&ctl->full[s]), (uint32_t)((it / STAGES) & 1), abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t a0 = smem_u32(smem + s * STAGE_BYTES);
+                    const uint32_t b0 = a0 + A_BYTES;
+#pragma unroll
+                    for (int j = 0; j < BK / 32; ++j) {
+                        const uint64_t da = smem_desc_kmajor(a0 + 2 * j * (BM * 16), BM * 16, 128);
+                        const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (BN * 16), BN * 16, 128);
+                        mma_i8(d, da, db, idesc, (ks | j) != 0);
+                    }
+                    mma_commit(smem_u32(&ctl->empty[s]));
+                }
+                if (ok) mma_commit(smem_u32(&ctl->acc_full[b]));
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue: 128 threads, thread = one frame (TMEM lane)
+        const int row_in_tile = warp * 32 + lane;
+        int tl = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
+            const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+            const int m = m0 + row_in_tile;
+            // per-frame and per-unit popcounts of this tile (overlaps the MMAs of the tile)
+            const int pa = m < M ? row_popc(Ap + (size_t)m * ldap, kw, tmask) : 0;
+            epi_bar_sync();  // previous tile's readers of T are done
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int nl = row_in_tile + h * 128, n = n0 + nl;
+                int t = 0;
+                if (n < N) {
+                    const int pw = row_popc(Wp + (size_t)n * ldwp, kw, tmask);
+                    t = (SIGN_PACK && !STORE_C) ? 32 * (thr[n] + 2 * pw - K) : 2 * pw - K;
+                }
+                ctl->T[nl] = t;
+            }
+            if (SIGN_PACK && row_in_tile < BN / 32) {
+                const int wi = (n0 >> 5) + row_in_tile;
+                ctl->flipw[row_in_tile] = wi < words_for(N) ? flip[wi] : 0u;
+            }
+            epi_bar_sync();
+            const int b = tl & 1;
+            // all four epilogue warps take the same decision, so none is left at a barrier
+            ok = epi_all(warp_wait(smem_u32(&ctl->acc_full[b]), (uint32_t)((tl >> 1) & 1), abort_flag, lane));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * BN);
+            uint32_t words[BN / 32];
+#pragma unroll
+            for (int g = 0; g < BN / 32; ++g) {
+                uint32_t acc[32];
+                tmem_ld32(taddr + g * 32, acc);
+                tmem_ld_wait();
+                const int nb = n0 + g * 32;
+                if (STORE_C) {
+                    // dot = 4 popc(a&w) - 2 popc(a) - (2 popc(w) - K), acc = 128 popc(a&w)
+                    int d[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) d[j] = (int)(acc[j] >> 5) - 2 * pa - ctl->T[g * 32 + j];
+                    if (m < M) {
+                        int32_t* dst = C + (size_t)m * ldc + nb;
+                        const bool vec = (ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && nb + 31 < N;
+                        if (vec) {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                reinterpret_cast<int4*>(dst)[q] = make_int4(d[4 * q], d[4 * q + 1], d[4 * q + 2], d[4 * q + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (nb + j < N) dst[j] = d[j];
+                        }
+                    }
+                    if (SIGN_PACK) {
+                        uint32_t wd = 0u;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int n = nb + j;
+                            const bool bit = n < N && (d[j] >= __ldg(thr + (n < N ? n : 0)));
+                            wd |= (uint32_t)bit << j;
+                        }
+                        words[g] = wd ^ ctl->flipw[g];
+                    }
+                } else {
+                    // bit = (acc - 64 popc(a) - T[n] >= 0); the sign bits are shifted in from the
+                    // top, element 31 first, so element j ends up in bit j, inverted.
+                    const int cm = 64 * pa;
+                    uint32_t wd = 0u;
+#pragma unroll
+                    for (int j = 31; j >= 0; --j) {
+                        const int v = (int)acc[j] - cm - ctl->T[g * 32 + j];
+                        wd = __funnelshift_l((uint32_t)v, wd, 1);
+                    }
+                    words[g] = ~wd ^ ctl->flipw[g];
+                }
+                if (SIGN_PACK) {
+                    const int valid = N - nb;  // columns of this word that exist
+                    if (valid < 32) words[g] = valid > 0 ? (words[g] & ((1u << valid) - 1u)) : 0u;
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+            if (SIGN_PACK && m < M) {
+                const int nw = words_for(N), w0 = n0 >> 5;
+                uint32_t* dst = out_bits + (size_t)m * ldob + w0;
+                if (w0 + BN / 32 <= nw) {
+                    reinterpret_cast<uint4*>(dst)[0] = make_uint4(words[0], words[1], words[2], words[3]);
+                    reinterpret_cast<uint4*>(dst)[1] = make_uint4(words[4], words[5], words[6], words[7]);
+                } else {
+#pragma unroll
+                    for (int g = 0; g < BN / 32; ++g)
+                        if (w0 + g < nw) dst[g] = words[g];
+                }
+            }
+        }
+    }
+
+    // ---------------- teardown: every thread arrives here, also after an aborted wait
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == MMA_WARP) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
+    if (threadIdx.x == 0 && ctl->abort) atomicExch(&g_tc_status, 1);
+}
+
+int g_sm_count = 0;
+
+template <bool STORE_C, bool SIGN_PACK>
+int launch_variant(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N, int K,
+                   int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
+                   uint32_t* out_bits, int ldob, cudaStream_t st) {
+    auto kern = xnor_tc_kernel<STORE_C, SIGN_PACK>;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return BNN_ERR_CUDA;
+        configured = true;
+    }
+    if (g_sm_count == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return BNN_ERR_CUDA;
+    }
+    const int tiles = ceil_div(M, BM) * ceil_div(N, BN);
+    const int grid = tiles < g_sm_count ? tiles : g_sm_count;
+    kern<<<grid, THREADS, SMEM_BYTES, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob);
+    return launch_status();
+}
+
+}  // namespace
+
+int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
+                   int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
+                   uint32_t* out_bits, int ldob, cudaStream_t st) {
+    const bool sp = out_bits != nullptr;
+    if (C && sp) return launch_variant<true, true>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
+    if (C) return launch_variant<true, false>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
+    return launch_variant<false, true>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
+}
+
+int read_tc_status(int* out) {
+    return cudaMemcpyFromSymbol(out, g_tc_status, sizeof(int)) == cudaSuccess ? BNN_OK : BNN_ERR_CUDA;
+}
+
+}  // namespace bnn

@@ -64,6 +64,16 @@ def run_binary_net(env, cfg, frames, mode=0, sample=None):
 def test_forward_tiny_config_all_frames(env):
     r = run_binary_net(env, wl.CONFIGS["tiny"], 256)
     assert r["flipped"] <= r["ambiguous"]
+    assert env[1].bnn_device_status() == 0
+
+
+def test_forward_tiny_config_popcount_path(env):
+    B = env[1]
+    prev = B.bnn_set_xnor_path(B.XNOR_POPC)
+    try:
+        run_binary_net(env, wl.CONFIGS["tiny"], 256)
+    finally:
+        B.bnn_set_xnor_path(prev)
 
 
 def test_forward_tiny_config_paper_sign_convention(env):

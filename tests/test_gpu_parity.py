@@ -29,6 +29,15 @@ def torch_():
     return torch
 
 
+@pytest.fixture(params=["popc", "tensor"])
+def xnor_path(request, B):
+    """Runs a test once per XNOR kernel (integer-pipe popcount, tcgen05 tensor core)."""
+    prev = B.bnn_set_xnor_path(B.XNOR_POPC if request.param == "popc" else B.XNOR_TENSOR)
+    yield request.param
+    B.bnn_set_xnor_path(prev)
+    assert B.bnn_device_status() == 0, "a tensor-core kernel gave up on a bounded wait"
+
+
 def dev(a):
     from paper_1706_09453_b200.model import to_dev
     return to_dev(a)
@@ -115,12 +124,13 @@ def test_fold_thresholds_null_scale_shift(B, torch_):
 
 # ------------------------------------------------------------------ XNOR GEMM
 XNOR_SHAPES = [(1, 1, 1), (2, 3, 31), (5, 7, 32), (17, 9, 33), (129, 130, 127), (300, 257, 1000),
-               (256, 1024, 1024), (131, 1024, 440), (200, 129, 600), (640, 384, 2048)]
+               (256, 1024, 1024), (131, 1024, 440), (200, 129, 600), (640, 384, 2048), (100, 520, 4100),
+               (20000, 256, 96)]
 
 
 @pytest.mark.parametrize("shape", XNOR_SHAPES)
 @pytest.mark.parametrize("p", [0.5, 0.1])
-def test_xnor_gemm_int32_bit_exact(B, torch_, shape, p):
+def test_xnor_gemm_int32_bit_exact(B, torch_, xnor_path, shape, p):
     m, n, k = shape
     ap = wl.make_bit_planes(m, k, p, [1, m, n, k], B.packed_pitch(k))
     wp = wl.make_bit_planes(n, k, p, [2, m, n, k], B.packed_pitch(k))
@@ -131,7 +141,7 @@ def test_xnor_gemm_int32_bit_exact(B, torch_, shape, p):
     np.testing.assert_array_equal(got[:, n:], -77)
 
 
-def test_xnor_gemm_ignores_garbage_in_pad_bits(B, torch_):
+def test_xnor_gemm_ignores_garbage_in_pad_bits(B, torch_, xnor_path):
     m, n, k = 70, 90, 1000 - 13
     pitch = B.packed_pitch(k) + 4
     ap = wl.make_bit_planes(m, k, 0.5, 11, pitch)
@@ -149,10 +159,11 @@ def test_xnor_gemm_ignores_garbage_in_pad_bits(B, torch_):
     np.testing.assert_array_equal(c.cpu().numpy(), want)
 
 
-@pytest.mark.parametrize("shape", [(5, 7, 33), (129, 130, 127), (300, 257, 1000), (256, 1024, 1024), (131, 96, 440)])
+@pytest.mark.parametrize("shape", [(5, 7, 33), (129, 130, 127), (300, 257, 1000), (256, 1024, 1024), (131, 96, 440),
+                                   (19100, 300, 160)])
 @pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("with_c", [False, True])
-def test_xnor_gemm_fused_sign_pack_bit_exact(B, torch_, shape, mode, with_c):
+def test_xnor_gemm_fused_sign_pack_bit_exact(B, torch_, xnor_path, shape, mode, with_c):
     m, n, k = shape
     rng = np.random.default_rng(m + n + k)
     ap = wl.make_bit_planes(m, k, 0.5, [3, m, n, k], B.packed_pitch(k))
