@@ -39,6 +39,8 @@ def parse_args():
     ap.add_argument("--frames", type=int, default=None, help="override the batch size (frames per step)")
     ap.add_argument("--cpu-frames", type=int, default=2048, help="frames of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--real-path", default="tensor", choices=["tensor", "fp32"],
+                    help="kernel of the real-valued layers: tcgen05 with split operands or the FP32 pipe")
     ap.add_argument("--xnor-path", default="tensor", choices=["tensor", "popc"],
                     help="kernel of the binary hidden layers: tcgen05 tensor core or integer-pipe popcount")
     return ap.parse_args()
@@ -153,7 +155,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ roofline bookkeeping
-def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor"):
+def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tensor"):
     """Per layer: algorithmic work, the pipe that bounds the kernel and its peak.
 
     Algorithmic work: 2 binary ops per bit-MAC for XNOR layers, 2 flop per add/sub or MAC for
@@ -177,12 +179,25 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor"):
         elif xnor:
             rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_popc_kernel", work=work, unit="Tbop/s",
                              bound="alu", peak=popc_peak))
+        elif real_path == "tensor":
+            # bf16 tensor-core MMAs, one pass per bf16 term of the real operand (2 terms);
+            # algorithmic flops count the product once
+            rows.append(dict(name="signw_%d" % (l + 1), kernel="signw_tc_kernel", work=work, unit="TFLOP/s",
+                             bound="tensor", peak=peaks["bf16_tflops_sustained"], passes=2))
         else:
             rows.append(dict(name="signw_%d" % (l + 1), kernel="real_gemm_kernel", work=work, unit="TFLOP/s",
                              bound="alu", peak=fp32_peak))
         k = cfg.hidden
-    rows.append(dict(name="output", kernel="real_gemm_kernel+log_softmax_rows_kernel",
-                     work=2.0 * frames * cfg.classes * cfg.hidden, unit="TFLOP/s", bound="alu", peak=fp32_peak))
+    owork = 2.0 * frames * cfg.classes * cfg.hidden
+    if real_path == "tensor" and cfg.act == 1:
+        rows.append(dict(name="output_gemm", kernel="out_tc_kernel", work=owork, unit="TFLOP/s", bound="tensor",
+                         peak=peaks["bf16_tflops_sustained"], passes=2))
+    else:
+        rows.append(dict(name="output_gemm", kernel="real_gemm_kernel", work=owork, unit="TFLOP/s", bound="alu",
+                         peak=fp32_peak))
+    # log-softmax: one read and one write of the [frames][classes] fp32 matrix
+    rows.append(dict(name="log_softmax", kernel="log_softmax_rows_kernel", work=2.0 * frames * cfg.classes * 4,
+                     unit="GB/s", bound="hbm", peak=peaks["hbm_gbs"], scale=1e9))
     return rows
 
 
@@ -222,6 +237,7 @@ def run_ours(args):
     frames = args.frames or cfg.frames
     net = wl.make_model(cfg)
     B.bnn_set_xnor_path(B.XNOR_TENSOR if args.xnor_path == "tensor" else B.XNOR_POPC)
+    B.bnn_set_option(B.OPT_REAL_PATH, B.PATH_TENSOR if args.real_path == "tensor" else B.PATH_CUDA_CORE)
     dn = model.DeviceNet(net, device=dev)
     # Frames are independent, so ranks shard them with no exchange: each rank owns its own batch.
     Xh = wl.make_frames(cfg, frames, seed=cfg.seed + 1000 * rank)
@@ -261,7 +277,7 @@ def run_ours(args):
     # ---- per-layer device time over the same steps (events recorded inside the C-ABI call)
     nl = cfg.n_hidden + 1
     Kp = min(K, 50)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nl + 1)] for _ in range(Kp)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nl + 2)] for _ in range(Kp)]
     for row in evs:
         for e in row:
             e.record()
@@ -269,7 +285,10 @@ def run_ours(args):
     for i in range(Kp):
         B.bnn_forward_events(dn.desc, Xd[i % nsets], Ld[i % nsets], ws, evs[i])
     torch.cuda.synchronize()
-    layer_ms = [float(np.mean([evs[i][l].elapsed_time(evs[i][l + 1]) for i in range(Kp)])) for l in range(nl)]
+    # event order in time: 0 .. nl-1 (before each layer), nl+1 (after the top GEMM), nl (end)
+    order = list(range(nl)) + [nl + 1, nl]
+    layer_ms = [float(np.mean([evs[i][order[l]].elapsed_time(evs[i][order[l + 1]]) for i in range(Kp)]))
+                for l in range(nl + 1)]
 
     # ---- end to end: pinned host input -> device, forward, log-probs -> pinned host, every step
     Ke = max(3, min(K, 20))
@@ -297,11 +316,13 @@ def run_ours(args):
 
     peaks = load_peaks()
     ck = clocks.summary()
-    rows = layer_table(cfg, frames, peaks, ck.get("sm_mhz"), args.xnor_path)
+    rows = layer_table(cfg, frames, peaks, ck.get("sm_mhz"), args.xnor_path, args.real_path)
+    assert len(rows) == len(layer_ms)
     for r, t in zip(rows, layer_ms):
         r["ms"] = t
-        r["achieved"] = r["work"] / (t * 1e-3) / 1e12
+        r["achieved"] = r["work"] / (t * 1e-3) / r.get("scale", 1e12)
         r["frac"] = r["achieved"] / r["peak"]
+        r["pipe_util"] = r["frac"] * r.get("passes", 1)
     dom = max(rows, key=lambda r: r["ms"])
     share = dom["ms"] / sum(layer_ms)
     roofline = {"kernel": dom["kernel"], "layer": dom["name"], "bound": dom["bound"],
@@ -318,8 +339,9 @@ def run_ours(args):
     out = {
         "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "%s (hidden layers) + f32 (first and top layer)"
-                 % ("u8 tensor-core MMA, s32 accumulate" if args.xnor_path == "tensor" else "int32 popcount"),
+        "dtype": "%s (hidden layers) + %s (first and top layer)"
+                 % ("u8 tensor-core MMA, s32 accumulate" if args.xnor_path == "tensor" else "int32 popcount",
+                    "split bf16/fp16 tensor-core MMA, f32 accumulate" if args.real_path == "tensor" else "f32"),
         "device_status": B.bnn_device_status(), "data": "synthetic",
         "config": {"workload": workload_name(cfg, frames), "frames_per_gpu": frames,
                    "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 2 x L2); weights stay hot"
@@ -329,8 +351,10 @@ def run_ours(args):
         "e2e": {"value": e2e_fps, "unit": UNIT, "h2d_bytes_per_step": int(Xp.numel() * 4),
                 "d2h_bytes_per_step": int(Lp.numel() * 4), "steps": Ke},
         "gpu_launches": K * (cfg.n_hidden + 2),
+        "paths": {"xnor": args.xnor_path, "real": args.real_path},
         "roofline": roofline,
-        "layers": [{k: r[k] for k in ("name", "kernel", "ms", "achieved", "peak", "unit", "frac")} for r in rows],
+        "layers": [{k: r[k] for k in ("name", "kernel", "bound", "ms", "achieved", "peak", "unit", "frac", "pipe_util")}
+                   for r in rows],
         "xnor_tbops": (xnor_work / (xnor_ms * 1e-3) / 1e12) if xnor_ms else None,
         "hbm": {"algorithmic_bytes_per_step": hbm, "achieved_gbs": hbm / (total_ms / K * 1e-3) / 1e9,
                 "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"]},

@@ -143,11 +143,22 @@ BNN_API int bnn_signw_gemm(const float* X, int ldx, const uint32_t* Wp, int ldwp
  * Exactly one of Hp (packed +-1 activations [M][ldhp]) and Hf (fp32 [M][ldhf]) is given.
  * Wout : fp32 [C][ldw].  b : [C] or NULL.  logp : fp32 [M][ldo] (written; holds the raw
  * logits between the two internal passes).  log_softmax = 0 leaves the logits z.
+ * prepared : NULL, or the image bnn_output_prepare made from the SAME Wout; with it and
+ * packed activations the product runs on the tensor cores, otherwise on the FP32 pipe.
  */
 BNN_API int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
-                     const float* Wout, int ldw, const float* b,
+                     const float* Wout, int ldw, const float* b, const void* prepared,
                      int M, int C, int H, float* logp, int ldo, int log_softmax,
                      void* stream);
+
+/* One-time preparation of the top layer's weights for the tensor cores: each class row is
+ * scaled by a power of two and split into two fp16 terms (about 22 significant bits), stored
+ * in the order the MMA reads shared memory.  prepared : device buffer, 256-byte aligned, of
+ * at least bnn_output_prepared_bytes(C, H) bytes.  The paper has no counterpart (it keeps
+ * this layer in full precision; Section 2.3). */
+BNN_API size_t bnn_output_prepared_bytes(int C, int H);
+BNN_API int bnn_output_prepare(const float* Wout, int ldw, int C, int H,
+                               void* prepared, size_t prepared_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------
  * Whole forward pass: the loops "for l = 1 to L" of Algorithms 1 and 2.
@@ -166,6 +177,7 @@ typedef struct bnn_layer {
     int ldwp;
     const float* W;        /* REAL_OUT: fp32 weights [N][ldw] */
     int ldw;
+    const void* W_prepared;/* REAL_OUT: bnn_output_prepare image of W, or NULL */
     const float* scale;    /* SIGNW: per-unit scale or NULL */
     const float* shift;    /* SIGNW: per-unit shift or NULL; REAL_OUT: bias or NULL */
     const int32_t* thr;    /* XNOR: folded thresholds [N] */
@@ -196,20 +208,29 @@ BNN_API int bnn_forward(const bnn_model* model, const float* X, int ldx, int M,
                 float* logp, int ldo, void* workspace, size_t workspace_bytes,
                 void* const* layer_out, void* stream);
 
-/* bnn_forward that also records events[l] (cudaEvent_t, HOST array of n_layers+1 entries,
- * NULL entries skipped) on `stream` before layer l and events[n_layers] after the last
- * kernel, so a caller can time each layer where it runs.  The paper has no counterpart. */
+/* bnn_forward that also records events on `stream` so a caller can time each layer where it
+ * runs.  events : HOST array of n_layers+2 cudaEvent_t (NULL entries skipped): events[l] is
+ * recorded before layer l, events[n_layers] after the last kernel, events[n_layers+1]
+ * between the top layer's GEMM and its log-softmax.  The paper has no counterpart. */
 BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                                float* logp, int ldo, void* workspace, size_t workspace_bytes,
                                void* const* layer_out, void* const* events, void* stream);
 
-/* Which kernel bnn_xnor_gemm (and the XNOR layers of bnn_forward) use.  Both compute the
- * same integers: BNN_XNOR_POPC is the XOR/popcount kernel on the integer pipes,
- * BNN_XNOR_TENSOR the tcgen05 tensor-core kernel (needs K <= 2^22; larger K falls back to
- * popcount).  BNN_XNOR_AUTO picks the faster one as measured on B200 (tensor).
- * Process-wide setting; returns the previous value, or -1 for an unknown `path`. */
-typedef enum { BNN_XNOR_AUTO = 0, BNN_XNOR_POPC = 1, BNN_XNOR_TENSOR = 2 } bnn_xnor_path;
-BNN_API int bnn_set_xnor_path(int path);
+/* Process-wide choice of kernels; bnn_set_option returns the previous value or -1 for an
+ * unknown option/value.  Every choice computes the same function (integers identical, floats
+ * within the documented bounds); the options exist so that the paths can be measured against
+ * each other.
+ *   BNN_OPT_XNOR_PATH  : BNN_PATH_AUTO | BNN_PATH_CUDA_CORE (XOR/popcount on the integer
+ *                        pipes) | BNN_PATH_TENSOR (tcgen05; needs K <= 2^22, larger K falls
+ *                        back to popcount).  AUTO = TENSOR, the faster one on B200.
+ *   BNN_OPT_REAL_PATH  : same values, for bnn_signw_gemm and bnn_output_layer: FP32 pipe or
+ *                        tcgen05 with split bf16/fp16 operands.  AUTO = TENSOR.
+ *   BNN_OPT_SIGNW_TERMS: 2 (default) or 3 bf16 terms for the real operand of bnn_signw_gemm
+ *                        on the tensor path: |error| <= 2^-17 sum|x_i| with 2, fp32-exact
+ *                        products with 3. */
+typedef enum { BNN_OPT_XNOR_PATH = 0, BNN_OPT_REAL_PATH = 1, BNN_OPT_SIGNW_TERMS = 2 } bnn_option;
+typedef enum { BNN_PATH_AUTO = 0, BNN_PATH_CUDA_CORE = 1, BNN_PATH_TENSOR = 2 } bnn_path;
+BNN_API int bnn_set_option(int option, int value);
 
 /* Tensor-core kernels bound every wait they perform; a CTA whose wait runs out stops, frees
  * its tensor memory and sets a status word.  This call SYNCHRONISES the device and stores

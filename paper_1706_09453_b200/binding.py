@@ -34,7 +34,7 @@ class Epilogue(C.Structure):
 class Layer(C.Structure):
     _fields_ = [("kind", C.c_int), ("K", C.c_int), ("N", C.c_int),
                 ("Wp", C.c_void_p), ("ldwp", C.c_int),
-                ("W", C.c_void_p), ("ldw", C.c_int),
+                ("W", C.c_void_p), ("ldw", C.c_int), ("W_prepared", C.c_void_p),
                 ("scale", C.c_void_p), ("shift", C.c_void_p),
                 ("thr", C.c_void_p), ("flip", C.c_void_p),
                 ("act", C.c_int)]
@@ -64,8 +64,12 @@ def lib():
         L.bnn_status_string.argtypes = [C.c_int]
         L.bnn_packed_pitch.restype = C.c_int
         L.bnn_packed_pitch.argtypes = [C.c_int]
-        L.bnn_set_xnor_path.argtypes = [C.c_int]
-        L.bnn_set_xnor_path.restype = C.c_int
+        L.bnn_set_option.argtypes = [C.c_int, C.c_int]
+        L.bnn_set_option.restype = C.c_int
+        L.bnn_output_prepared_bytes.argtypes = [C.c_int, C.c_int]
+        L.bnn_output_prepared_bytes.restype = C.c_size_t
+        L.bnn_output_prepare.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.bnn_output_prepare.restype = C.c_int
         L.bnn_device_status.argtypes = [C.POINTER(C.c_int)]
         L.bnn_device_status.restype = C.c_int
         L.bnn_forward_workspace_bytes.restype = C.c_size_t
@@ -76,7 +80,7 @@ def lib():
         L.bnn_fold_thresholds.argtypes = [p, p, i, i, i, p, p, p]
         L.bnn_xnor_gemm.argtypes = [p, i, p, i, i, i, i, p, i, C.POINTER(Epilogue), p]
         L.bnn_signw_gemm.argtypes = [p, i, p, i, i, i, i, p, i, C.POINTER(Epilogue), p]
-        L.bnn_output_layer.argtypes = [p, i, p, i, p, i, p, i, i, i, p, i, i, p]
+        L.bnn_output_layer.argtypes = [p, i, p, i, p, i, p, p, i, i, i, p, i, i, p]
         L.bnn_forward.argtypes = [C.POINTER(Model), p, i, i, p, i, p, C.c_size_t, C.POINTER(p), p]
         L.bnn_forward_events.argtypes = [C.POINTER(Model), p, i, i, p, i, p, C.c_size_t, C.POINTER(p),
                                          C.POINTER(p), p]
@@ -95,14 +99,20 @@ def packed_pitch(k: int) -> int:
     return int(lib().bnn_packed_pitch(int(k)))
 
 
-XNOR_AUTO, XNOR_POPC, XNOR_TENSOR = 0, 1, 2
+OPT_XNOR_PATH, OPT_REAL_PATH, OPT_SIGNW_TERMS = 0, 1, 2
+PATH_AUTO, PATH_CUDA_CORE, PATH_TENSOR = 0, 1, 2
+XNOR_AUTO, XNOR_POPC, XNOR_TENSOR = PATH_AUTO, PATH_CUDA_CORE, PATH_TENSOR
+
+
+def bnn_set_option(option: int, value: int) -> int:
+    prev = int(lib().bnn_set_option(int(option), int(value)))
+    if prev < 0:
+        raise ValueError("unknown option/value %r/%r" % (option, value))
+    return prev
 
 
 def bnn_set_xnor_path(path: int) -> int:
-    prev = int(lib().bnn_set_xnor_path(int(path)))
-    if prev < 0:
-        raise ValueError("unknown XNOR path %r" % path)
-    return prev
+    return bnn_set_option(OPT_XNOR_PATH, path)
 
 
 def bnn_device_status() -> int:
@@ -194,13 +204,24 @@ def bnn_signw_gemm(X, Wp, K, Y=None, act=ACT_NONE, scale=None, shift=None, out_b
            "bnn_signw_gemm")
 
 
-def bnn_output_layer(Wout, b, logp, H, Hp=None, Hf=None, log_softmax=True):
+def bnn_output_prepared_bytes(C_, H) -> int:
+    return int(lib().bnn_output_prepared_bytes(int(C_), int(H)))
+
+
+def bnn_output_prepare(Wout, prepared):
+    c, h = Wout.shape
+    _check(lib().bnn_output_prepare(_ptr(Wout, torch.float32), _ld(Wout), c, h, _ptr(prepared),
+                                    prepared.numel() * prepared.element_size(), _stream()), "bnn_output_prepare")
+    return prepared
+
+
+def bnn_output_layer(Wout, b, logp, H, Hp=None, Hf=None, log_softmax=True, prepared=None):
     m = (Hp if Hp is not None else Hf).shape[0]
     c = Wout.shape[0]
     _check(lib().bnn_output_layer(_ptr(Hp, torch.int32), _ld(Hp) if Hp is not None else 0,
                                   _ptr(Hf, torch.float32), _ld(Hf) if Hf is not None else 0,
                                   _ptr(Wout, torch.float32), _ld(Wout), _ptr(b, torch.float32),
-                                  m, c, H, _ptr(logp, torch.float32), _ld(logp), int(log_softmax), _stream()),
+                                  _ptr(prepared), m, c, H, _ptr(logp, torch.float32), _ld(logp), int(log_softmax), _stream()),
            "bnn_output_layer")
     return logp
 
@@ -216,6 +237,7 @@ class ModelDesc:
             wp, w = d.get("Wp"), d.get("W")
             a.Wp, a.ldwp = _ptr(wp, torch.int32), (_ld(wp) if wp is not None else 0)
             a.W, a.ldw = _ptr(w, torch.float32), (_ld(w) if w is not None else 0)
+            a.W_prepared = _ptr(d.get("W_prepared"))
             a.scale, a.shift = _ptr(d.get("scale"), torch.float32), _ptr(d.get("shift"), torch.float32)
             a.thr, a.flip = _ptr(d.get("thr"), torch.int32), _ptr(d.get("flip"), torch.int32)
         self._arr = arr
@@ -239,7 +261,7 @@ def bnn_forward(model: ModelDesc, X, logp, workspace, layer_out=None):
 
 
 def bnn_forward_events(model: ModelDesc, X, logp, workspace, events, layer_out=None):
-    """``events``: n_layers+1 recorded-at-least-once torch.cuda.Event objects (timing enabled)."""
+    """``events``: n_layers+2 recorded-at-least-once torch.cuda.Event objects (timing enabled)."""
     m = X.shape[0]
     lo = None
     if layer_out is not None:

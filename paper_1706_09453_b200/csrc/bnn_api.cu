@@ -8,7 +8,9 @@ using namespace bnn;
 namespace {
 
 constexpr int kMaxK = 1 << 24;
-int g_xnor_path = BNN_XNOR_AUTO;  // |dot| <= K stays exact in every accumulator type used
+int g_xnor_path = BNN_PATH_AUTO;
+int g_real_path = BNN_PATH_AUTO;
+int g_signw_terms = 2;  // |dot| <= K stays exact in every accumulator type used
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -86,10 +88,21 @@ extern "C" {
 
 int bnn_packed_pitch(int K) { return (words_for(K) + 3) & ~3; }
 
-int bnn_set_xnor_path(int path) {
-    if (path != BNN_XNOR_AUTO && path != BNN_XNOR_POPC && path != BNN_XNOR_TENSOR) return -1;
-    const int prev = g_xnor_path;
-    g_xnor_path = path;
+int bnn_set_option(int option, int value) {
+    int* slot = nullptr;
+    switch (option) {
+        case BNN_OPT_XNOR_PATH: slot = &g_xnor_path; break;
+        case BNN_OPT_REAL_PATH: slot = &g_real_path; break;
+        case BNN_OPT_SIGNW_TERMS: slot = &g_signw_terms; break;
+        default: return -1;
+    }
+    if (option == BNN_OPT_SIGNW_TERMS) {
+        if (value != 2 && value != 3) return -1;
+    } else if (value != BNN_PATH_AUTO && value != BNN_PATH_CUDA_CORE && value != BNN_PATH_TENSOR) {
+        return -1;
+    }
+    const int prev = *slot;
+    *slot = value;
     return prev;
 }
 
@@ -148,7 +161,7 @@ int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
         thr = epi->thr; flip = epi->flip; ob = epi->out_bits; ldob = epi->ldob;
     }
     if (!C && !ob) return BNN_ERR_NULL;
-    const bool tensor = g_xnor_path != BNN_XNOR_POPC && K <= kMaxKTensor;
+    const bool tensor = g_xnor_path != BNN_PATH_CUDA_CORE && K <= kMaxKTensor;
     return (tensor ? launch_xnor_tc : launch_xnor_popc)(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip,
                                                         ob, ldob, (cudaStream_t)stream);
 }
@@ -178,13 +191,28 @@ int bnn_signw_gemm(const float* X, int ldx, const uint32_t* Wp, int ldwp,
         }
     }
     if (!a.Y && !a.out_bits) return BNN_ERR_NULL;
+    if (g_real_path != BNN_PATH_CUDA_CORE) return launch_signw_tc(a, g_signw_terms, (cudaStream_t)stream);
     return launch_real_gemm(a, (cudaStream_t)stream);
 }
 
-int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
-                     const float* Wout, int ldw, const float* b,
-                     int M, int C, int H, float* logp, int ldo, int log_softmax,
-                     void* stream) {
+size_t bnn_output_prepared_bytes(int C, int H) {
+    if (C < 1 || H < 1) return 0;
+    return out_prepared_bytes(C, H);
+}
+
+int bnn_output_prepare(const float* Wout, int ldw, int C, int H,
+                       void* prepared, size_t prepared_bytes, void* stream) {
+    if (!Wout || !prepared) return BNN_ERR_NULL;
+    if (C < 1 || H < 1 || ldw < H) return BNN_ERR_SHAPE;
+    if (prepared_bytes < out_prepared_bytes(C, H)) return BNN_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(prepared) & 255u) return BNN_ERR_ALIGN;
+    return launch_out_prepare(Wout, ldw, C, H, prepared, (cudaStream_t)stream);
+}
+
+static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
+                             const float* Wout, int ldw, const float* b, const void* prepared,
+                             int M, int C, int H, float* logp, int ldo, int log_softmax,
+                             void* mid_event, void* stream) {
     if (int rc = check_dims(M, C, H)) return rc;
     if (!Wout || !logp) return BNN_ERR_NULL;
     if ((Hp == nullptr) == (Hf == nullptr)) return Hp ? BNN_ERR_UNSUPPORTED : BNN_ERR_NULL;
@@ -202,9 +230,25 @@ int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
     a.shift = b;
     a.act = BNN_ACT_NONE;
     a.Y = logp; a.ldy = ldo;
-    if (int rc = launch_real_gemm(a, (cudaStream_t)stream)) return rc;
+    if (prepared && (reinterpret_cast<uintptr_t>(prepared) & 255u)) return BNN_ERR_ALIGN;
+    int rc;
+    if (Hp && prepared && g_real_path != BNN_PATH_CUDA_CORE)
+        rc = launch_out_tc(Hp, ldhp, prepared, b, M, C, H, logp, ldo, (cudaStream_t)stream);
+    else
+        rc = launch_real_gemm(a, (cudaStream_t)stream);
+    if (rc) return rc;
+    if (mid_event && cudaEventRecord((cudaEvent_t)mid_event, (cudaStream_t)stream) != cudaSuccess)
+        return BNN_ERR_CUDA;
     if (log_softmax) return launch_log_softmax_rows(logp, ldo, M, C, (cudaStream_t)stream);
     return BNN_OK;
+}
+
+int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
+                     const float* Wout, int ldw, const float* b, const void* prepared,
+                     int M, int C, int H, float* logp, int ldo, int log_softmax,
+                     void* stream) {
+    return output_layer_impl(Hp, ldhp, Hf, ldhf, Wout, ldw, b, prepared, M, C, H, logp, ldo,
+                             log_softmax, nullptr, stream);
 }
 
 size_t bnn_forward_workspace_bytes(const bnn_model* model, int M) {
@@ -248,9 +292,10 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
             cudaEventRecord((cudaEvent_t)events[l], (cudaStream_t)stream) != cudaSuccess)
             return BNN_ERR_CUDA;
         if (y.kind == BNN_LAYER_REAL_OUT) {
-            int rc = bnn_output_layer(in_bits ? static_cast<const uint32_t*>(in) : nullptr, in_ld,
-                                    in_bits ? nullptr : static_cast<const float*>(in), in_ld,
-                                    y.W, y.ldw, y.shift, M, y.N, y.K, logp, ldo, 1, stream);
+            int rc = output_layer_impl(in_bits ? static_cast<const uint32_t*>(in) : nullptr, in_ld,
+                                       in_bits ? nullptr : static_cast<const float*>(in), in_ld,
+                                       y.W, y.ldw, y.shift, y.W_prepared, M, y.N, y.K, logp, ldo, 1,
+                                       events ? events[L + 1] : nullptr, stream);
             if (rc) return rc;
             if (events && events[L] &&
                 cudaEventRecord((cudaEvent_t)events[L], (cudaStream_t)stream) != cudaSuccess)

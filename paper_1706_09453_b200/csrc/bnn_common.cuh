@@ -56,6 +56,8 @@ int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, i
                    uint32_t* out_bits, int ldob, cudaStream_t st);
 // Reads (synchronously) the word that a tensor-core kernel sets when a bounded wait ran out.
 int read_tc_status(int* out);
+// Device address of that word, passed to every tensor-core kernel (nullptr on failure).
+int* tc_status_ptr();
 
 // Real-valued GEMM on the FP32 pipe: D[m][n] = sum_k A[m][k]*B[n][k], where each operand is
 // either fp32 or packed +-1 bits.
@@ -77,6 +79,13 @@ struct RealGemmArgs {
     int ldob;
 };
 int launch_real_gemm(const RealGemmArgs& a, cudaStream_t st);
+// Tensor-core versions: +-1 weights x real input (A fp32, B bits; `terms` bf16 terms), and
+// the top layer on packed activations with prepared fp16 weight terms.
+int launch_signw_tc(const RealGemmArgs& a, int terms, cudaStream_t st);
+size_t out_prepared_bytes(int C, int H);
+int launch_out_prepare(const float* W, int ldw, int C, int H, void* prepared, cudaStream_t st);
+int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const float* bias,
+                  int M, int C, int H, float* Z, int ldz, cudaStream_t st);
 int launch_log_softmax_rows(float* Z, int ldz, int M, int C, cudaStream_t st);
 
 }  // namespace bnn

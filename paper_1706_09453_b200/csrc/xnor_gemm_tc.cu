@@ -22,6 +22,7 @@
 namespace bnn {
 
 __device__ int g_tc_status = 0;  // set to 1 by a CTA whose bounded wait ran out
+int* tc_status_ptr();
 
 namespace {
 
@@ -86,7 +87,7 @@ __global__ void __launch_bounds__(THREADS, 1)
 xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __restrict__ Wp, int ldwp,
                int M, int N, int K, int32_t* __restrict__ C, int ldc,
                const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
-               uint32_t* __restrict__ out_bits, int ldob) {
+               uint32_t* __restrict__ out_bits, int ldob, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES);
@@ -323,7 +324,7 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (threadIdx.x == 0 && ctl->abort) atomicExch(&g_tc_status, 1);
+    if (threadIdx.x == 0 && ctl->abort) atomicExch(status, 1);
 }
 
 int g_sm_count = 0;
@@ -347,7 +348,9 @@ int launch_variant(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, i
     }
     const int tiles = ceil_div(M, BM) * ceil_div(N, BN);
     const int grid = tiles < g_sm_count ? tiles : g_sm_count;
-    kern<<<grid, THREADS, SMEM_BYTES, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob);
+    int* status = tc_status_ptr();
+    if (!status) return BNN_ERR_CUDA;
+    kern<<<grid, THREADS, SMEM_BYTES, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, status);
     return launch_status();
 }
 
@@ -360,6 +363,13 @@ int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, i
     if (C && sp) return launch_variant<true, true>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
     if (C) return launch_variant<true, false>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
     return launch_variant<false, true>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
+}
+
+// Device address of the status word (one per device would need a table; one device is used).
+int* tc_status_ptr() {
+    static int* ptr = nullptr;
+    if (!ptr && cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_tc_status) != cudaSuccess) ptr = nullptr;
+    return ptr;
 }
 
 int read_tc_status(int* out) {

@@ -52,8 +52,11 @@ class DeviceNet:
                 layers.append(dict(kind=B.LAYER_XNOR, K=k, N=n, Wp=wp, thr=thr, flip=flip,
                                    act=B.ACT_SIGN_PACK))
         self.Wout, self.bout = to_dev(net.Wout, device), to_dev(net.bout, device)
+        self.Wout_prepared = torch.empty(B.bnn_output_prepared_bytes(cfg.classes, cfg.hidden),
+                                         dtype=torch.uint8, device=device)
+        B.bnn_output_prepare(self.Wout, self.Wout_prepared)
         layers.append(dict(kind=B.LAYER_REAL_OUT, K=cfg.hidden, N=cfg.classes, W=self.Wout,
-                           shift=self.bout))
+                           W_prepared=self.Wout_prepared, shift=self.bout))
         self.desc = B.ModelDesc(layers, sign_mode)
         self._ws = None
 

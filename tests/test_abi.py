@@ -68,8 +68,16 @@ def test_bad_arguments_are_rejected_without_a_launch(lib):
     # signw / output layer
     assert rc("bnn_signw_gemm", None, 4, fake, 4, 1, 1, 4, fake, 1, None, None) == 1
     assert rc("bnn_signw_gemm", fake, 4, fake, 4, 1, 1, 4, None, 0, None, None) == 1        # no output
-    assert rc("bnn_output_layer", fake, 4, fake, 4, fake, 4, None, 1, 1, 4, fake, 1, 1, None) == 4
-    assert rc("bnn_output_layer", None, 0, None, 0, fake, 4, None, 1, 1, 4, fake, 1, 1, None) == 1
+    assert rc("bnn_output_layer", fake, 4, fake, 4, fake, 4, None, None, 1, 1, 4, fake, 1, 1, None) == 4
+    assert rc("bnn_output_layer", None, 0, None, 0, fake, 4, None, None, 1, 1, 4, fake, 1, 1, None) == 1
+    assert rc("bnn_output_layer", fake, 4, None, 0, fake, 4, None, fake + 16, 1, 1, 4, fake, 1, 1, None) == 3
+    assert rc("bnn_output_prepare", fake, 4, 1, 4, None, 1 << 20, None) == 1
+    assert rc("bnn_output_prepare", fake, 4, 1, 4, fake, 16, None) == 5
+    assert B.bnn_output_prepared_bytes(3400, 2048) == 27 * 64 * 16384 + 27 * 128 * 4
+    # options
+    assert B.bnn_set_option(B.OPT_XNOR_PATH, B.PATH_CUDA_CORE) == 0
+    assert B.bnn_set_option(B.OPT_XNOR_PATH, B.PATH_AUTO) == 1
+    assert rc("bnn_set_option", 9, 0) == -1 and rc("bnn_set_option", 2, 4) == -1
     assert rc("bnn_fold_thresholds", None, None, 4, 4, 0, None, fake, None) == 1
 
 

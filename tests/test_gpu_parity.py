@@ -38,6 +38,15 @@ def xnor_path(request, B):
     assert B.bnn_device_status() == 0, "a tensor-core kernel gave up on a bounded wait"
 
 
+@pytest.fixture(params=["fp32", "tensor"])
+def real_path(request, B):
+    """Runs a test once per real-valued GEMM kernel (FP32 pipe, tcgen05 with split operands)."""
+    prev = B.bnn_set_option(B.OPT_REAL_PATH, B.PATH_CUDA_CORE if request.param == "fp32" else B.PATH_TENSOR)
+    yield request.param
+    B.bnn_set_option(B.OPT_REAL_PATH, prev)
+    assert B.bnn_device_status() == 0, "a tensor-core kernel gave up on a bounded wait"
+
+
 def dev(a):
     from paper_1706_09453_b200.model import to_dev
     return to_dev(a)
@@ -193,8 +202,9 @@ def test_xnor_gemm_fused_sign_pack_bit_exact(B, torch_, xnor_path, shape, mode, 
 
 
 # ------------------------------------------------------------------ +-1 weights x real input
-@pytest.mark.parametrize("shape", [(1, 1, 1), (3, 5, 33), (130, 129, 440), (257, 300, 600), (64, 256, 2048)])
-def test_signw_gemm_within_tolerance(B, torch_, shape):
+@pytest.mark.parametrize("shape", [(1, 1, 1), (3, 5, 33), (130, 129, 440), (257, 300, 600), (64, 256, 2048),
+                                   (20000, 260, 70)])
+def test_signw_gemm_within_tolerance(B, torch_, real_path, shape):
     m, n, k = shape
     rng = np.random.default_rng(m * n + k)
     x = rng.standard_normal((m, k)).astype(np.float32)
@@ -210,7 +220,7 @@ def test_signw_gemm_within_tolerance(B, torch_, shape):
 
 
 @pytest.mark.parametrize("mode", [0, 1])
-def test_signw_gemm_sign_pack_epilogue(B, torch_, mode):
+def test_signw_gemm_sign_pack_epilogue(B, torch_, real_path, mode):
     m, n, k = 200, 300, 440
     rng = np.random.default_rng(9)
     x = rng.standard_normal((m, k)).astype(np.float32)
@@ -239,7 +249,7 @@ def test_signw_gemm_sign_pack_epilogue(B, torch_, mode):
     np.testing.assert_array_equal(gs, own)
 
 
-def test_signw_gemm_exact_zero_follows_sign_mode(B, torch_):
+def test_signw_gemm_exact_zero_follows_sign_mode(B, torch_, real_path):
     """Integer-valued inputs make y exactly 0 for some units; the bit must follow the mode."""
     m, n, k = 40, 64, 64
     rng = np.random.default_rng(3)
@@ -254,7 +264,7 @@ def test_signw_gemm_exact_zero_follows_sign_mode(B, torch_):
         np.testing.assert_array_equal(out.cpu().numpy().view(np.uint32)[:, :2], bits)
 
 
-def test_signw_gemm_hardtanh_epilogue(B, torch_):
+def test_signw_gemm_hardtanh_epilogue(B, torch_, real_path):
     m, n, k = 150, 200, 2048
     rng = np.random.default_rng(4)
     x = rng.uniform(-1, 1, (m, k)).astype(np.float32)
@@ -270,19 +280,23 @@ def test_signw_gemm_hardtanh_epilogue(B, torch_):
 
 
 # ------------------------------------------------------------------ top layer
-@pytest.mark.parametrize("c", [10, 2000, 3307, 3972])
-def test_output_layer_bits_logp(B, torch_, c):
-    m, h = 70, 1024
+@pytest.mark.parametrize("c,m,h", [(10, 70, 1024), (2000, 70, 1024), (3307, 70, 1024), (3972, 70, 1024),
+                                   (300, 1100, 1000), (129, 513, 33)])
+def test_output_layer_bits_logp(B, torch_, real_path, c, m, h):
     rng = np.random.default_rng(c)
     hp = wl.make_bit_planes(m, h, 0.5, 31, B.packed_pitch(h))
     wout = rng.normal(0, 1 / np.sqrt(h), (c, h)).astype(np.float32)
     b = rng.normal(0, 0.1, c).astype(np.float32)
+    prep = None
+    if real_path == "tensor":
+        prep = torch_.empty(B.bnn_output_prepared_bytes(c, h), dtype=torch_.uint8, device="cuda:0")
+        B.bnn_output_prepare(dev(wout), prep)
     z = torch_.full((m, c + 1), 9.0, dtype=torch_.float32, device="cuda:0")
-    B.bnn_output_layer(dev(wout), dev(b), z[:, :c], h, Hp=dev(hp), log_softmax=False)
+    B.bnn_output_layer(dev(wout), dev(b), z[:, :c], h, Hp=dev(hp), log_softmax=False, prepared=prep)
     zr = o.real_gemm_bits(hp, wout, b, h)
     assert np.abs(z.cpu().numpy()[:, :c] - zr).max() <= FLOAT_TOL * h
     lp = torch_.full((m, c + 1), 9.0, dtype=torch_.float32, device="cuda:0")
-    B.bnn_output_layer(dev(wout), dev(b), lp[:, :c], h, Hp=dev(hp))
+    B.bnn_output_layer(dev(wout), dev(b), lp[:, :c], h, Hp=dev(hp), prepared=prep)
     got = lp.cpu().numpy()
     assert np.abs(got[:, :c] - o.log_softmax(zr)).max() <= LOGP_TOL
     np.testing.assert_array_equal(got[:, c], 9.0)
@@ -299,3 +313,43 @@ def test_output_layer_real_activations(B, torch_):
     B.bnn_output_layer(dev(wout), dev(b), lp, h, Hf=dev(hf))
     want = o.log_softmax(o.real_gemm_f32(hf, wout, b))
     assert np.abs(lp.cpu().numpy() - want).max() <= LOGP_TOL
+
+
+def test_output_layer_wide_dynamic_range_weights(B, torch_):
+    """Rows whose magnitudes differ by many orders: the per-row power-of-two scaling of the
+    prepared fp16 terms must keep every row accurate."""
+    m, h, c = 64, 512, 200
+    rng = np.random.default_rng(12)
+    hp = wl.make_bit_planes(m, h, 0.5, 41, B.packed_pitch(h))
+    wout = rng.normal(0, 1, (c, h)).astype(np.float32)
+    wout *= (10.0 ** rng.uniform(-12, 6, (c, 1))).astype(np.float32)
+    wout[5] = 0.0
+    prep = torch_.empty(B.bnn_output_prepared_bytes(c, h), dtype=torch_.uint8, device="cuda:0")
+    B.bnn_output_prepare(dev(wout), prep)
+    z = torch_.empty((m, c), dtype=torch_.float32, device="cuda:0")
+    B.bnn_output_layer(dev(wout), None, z, h, Hp=dev(hp), log_softmax=False, prepared=prep)
+    zr = o.real_gemm_bits(hp, wout, None, h)
+    bound = 2.0 ** -20 * np.abs(wout.astype(np.float64)).sum(1)[None, :]
+    assert (np.abs(z.cpu().numpy() - zr) <= bound).all()
+    assert B.bnn_device_status() == 0
+
+
+@pytest.mark.parametrize("terms", [2, 3])
+def test_signw_gemm_tensor_error_bound_by_terms(B, torch_, terms):
+    """2 bf16 terms: |err| <= 2^-16 sum|x|; 3 terms: products exact, only fp32 accumulation."""
+    m, n, k = 300, 256, 440
+    rng = np.random.default_rng(13)
+    x = (rng.standard_normal((m, k)) * 10.0 ** rng.uniform(-3, 3, (m, 1))).astype(np.float32)
+    wp = wl.make_bit_planes(n, k, 0.5, 42, B.packed_pitch(k))
+    prev_p = B.bnn_set_option(B.OPT_REAL_PATH, B.PATH_TENSOR)
+    prev_t = B.bnn_set_option(B.OPT_SIGNW_TERMS, terms)
+    try:
+        y = torch_.empty((m, n), dtype=torch_.float32, device="cuda:0")
+        B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y)
+        ref, sumabs = o.signw_gemm(x, wp, k)
+        err = np.abs(y.cpu().numpy() - ref) / sumabs[:, None]
+        assert err.max() <= (2.0 ** -16 if terms == 2 else 2.0 ** -21), err.max()
+    finally:
+        B.bnn_set_option(B.OPT_SIGNW_TERMS, prev_t)
+        B.bnn_set_option(B.OPT_REAL_PATH, prev_p)
+    assert B.bnn_device_status() == 0
