@@ -44,21 +44,6 @@ struct Control {
 };
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + (int)sizeof(Control) + 128;
 
-__device__ __forceinline__ bool epi_all(bool pred) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 p, %1, 0;\n\t"
-        "barrier.red.and.pred q, 2, 128, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r) : "r"((uint32_t)pred) : "memory");
-    return r != 0;
-}
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int lane) {
-    int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
-    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
-}
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -130,8 +115,6 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
     volatile int* abort_flag = &ctl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int kw = words_for(H);
-    const uint32_t tmask = tail_mask(H);
     const int nks = ceil_div(H, BK);
     const int c_tiles = ceil_div(C, BC), f_tiles = ceil_div(M, FN);
     const int tiles = c_tiles * f_tiles;
@@ -161,38 +144,40 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
         const int p = threadIdx.x - PROD_WARP0 * 32;  // 0..255
         const int my_tiles = (tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
         const int total = my_tiles * nks;
-        int pf_i = 0, pf_ks = 0, pf_tile = blockIdx.x;
-        auto fetch = [&](uint32_t (&o)[2]) {
-            o[0] = 0u; o[1] = 0u;
-            if (pf_i >= total) return;
+        // Packed rows are read 16 bytes (4 stages) at a time, one group ahead of use.  Words at
+        // or beyond ceil(H/32) may hold anything: the weight image is zero there.
+        const int ngroups = ceil_div(nks, 4);
+        int pf_g = 0, pf_tile = blockIdx.x, pf_left = my_tiles;
+        auto fetch = [&](uint4 (&o)[2]) {
+            o[0] = make_uint4(0u, 0u, 0u, 0u);
+            o[1] = o[0];
+            if (pf_left == 0) return;
             const int f0 = (pf_tile / c_tiles) * FN;
-            if (pf_ks < kw) {
 #pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    const int f = f0 + p + 256 * q;
-                    if (f < M) {
-                        uint32_t w = __ldg(Hp + (size_t)f * ldhp + pf_ks);
-                        if (pf_ks == kw - 1) w &= tmask;  // pad bits widen to -1, against zero weights
-                        o[q] = w;
-                    }
-                }
+            for (int q = 0; q < 2; ++q) {
+                const int f = f0 + p + 256 * q;
+                if (f < M) o[q] = __ldg(reinterpret_cast<const uint4*>(Hp + (size_t)f * ldhp) + pf_g);
             }
-            ++pf_i;
-            if (++pf_ks == nks) { pf_ks = 0; pf_tile += gridDim.x; }
+            if (++pf_g == ngroups) { pf_g = 0; pf_tile += gridDim.x; --pf_left; }
         };
-        uint32_t cur[2], nxt[2];
-        fetch(cur);
+        uint4 grp[2], nxt[2];
+        fetch(grp);
+        fetch(nxt);
         int ks = 0, tile = blockIdx.x;
         for (int it = 0; it < total; ++it) {
-            fetch(nxt);
             const int s = it % STAGES;
             const uint32_t ph = (uint32_t)((it / STAGES) & 1);
+            const int sub = ks & 3;
+            uint32_t cur[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q)
+                cur[q] = sub == 0 ? grp[q].x : sub == 1 ? grp[q].y : sub == 2 ? grp[q].z : grp[q].w;
             if (!warp_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag, lane)) break;
-            uint8_t* st = smem + s * STAGE_BYTES;
+            const uint32_t st = smem_u32(smem) + s * STAGE_BYTES;
             if (p == 0) {
                 const int ct = tile % c_tiles;
                 mbar_expect_tx(smem_u32(&ctl->full[s]), A_BYTES);
-                bulk_g2s(smem_u32(st), img + ((size_t)ct * nks + ks) * A_BYTES, A_BYTES, smem_u32(&ctl->full[s]));
+                bulk_g2s(st, img + ((size_t)ct * nks + ks) * A_BYTES, A_BYTES, smem_u32(&ctl->full[s]));
             }
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
@@ -202,14 +187,17 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
                 for (int t = 0; t < 16; ++t) wv[t] = ((nw << (15 - t)) & 0x80008000u) | 0x3C003C00u;
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
-                    *reinterpret_cast<uint4*>(st + A_BYTES + (c * FN + p + 256 * q) * 16) =
-                        make_uint4(wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
+                    sts128(st + A_BYTES + (c * FN + p + 256 * q) * 16, wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
             }
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
-            cur[0] = nxt[0]; cur[1] = nxt[1];
-            if (++ks == nks) { ks = 0; tile += gridDim.x; }
+            ++ks;
+            if ((ks & 3) == 0 || ks == nks) {   // group used up: take the prefetched one
+                grp[0] = nxt[0]; grp[1] = nxt[1];
+                fetch(nxt);
+            }
+            if (ks == nks) { ks = 0; tile += gridDim.x; }
         }
     } else if (warp == MMA_WARP) {
         if (lane == 0) {

@@ -198,11 +198,33 @@ real_gemm_kernel(RealGemmArgs g) {
     }
 }
 
-// One CTA per row: online (max, sum exp) in one sweep, then z - logsumexp in a second.
+// Block-wide (max, sum of exp) combination used by both log-softmax kernels.
+__device__ __forceinline__ float block_logsumexp(float mx, float s, float* sm, float* ss) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float m2 = __shfl_xor_sync(0xFFFFFFFFu, mx, o);
+        const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        const float mn = fmaxf(mx, m2);
+        s = s * expf(mx - mn) + s2 * expf(m2 - mn);
+        mx = mn;
+    }
+    if (lane == 0) { sm[w] = mx; ss[w] = s; }
+    __syncthreads();
+    float gm = sm[0], gs = ss[0];
+    for (int i = 1; i < 8; ++i) {
+        const float mn = fmaxf(gm, sm[i]);
+        gs = gs * expf(gm - mn) + ss[i] * expf(sm[i] - mn);
+        gm = mn;
+    }
+    __syncthreads();
+    return gm + logf(gs);
+}
+
+// One CTA per row, any C: online (max, sum exp) in one sweep, then z - logsumexp in a second.
 __global__ void __launch_bounds__(256)
 log_softmax_rows_kernel(float* __restrict__ Z, int ldz, int M, int C) {
     __shared__ float sm[8], ss[8];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     for (int row = blockIdx.x; row < M; row += gridDim.x) {
         float* z = Z + (size_t)row * ldz;
         float mx = -FLT_MAX, s = 0.f;
@@ -211,25 +233,39 @@ log_softmax_rows_kernel(float* __restrict__ Z, int ldz, int M, int C) {
             if (v > mx) { s *= expf(mx - v); mx = v; }
             s += expf(v - mx);
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, mx, o);
-            const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, o);
-            const float mn = fmaxf(mx, m2);
-            s = s * expf(mx - mn) + s2 * expf(m2 - mn);
-            mx = mn;
-        }
-        if (lane == 0) { sm[w] = mx; ss[w] = s; }
-        __syncthreads();
-        float gm = sm[0], gs = ss[0];
-        for (int i = 1; i < 8; ++i) {
-            const float mn = fmaxf(gm, sm[i]);
-            gs = gs * expf(gm - mn) + ss[i] * expf(sm[i] - mn);
-            gm = mn;
-        }
-        const float lse = gm + logf(gs);
+        const float lse = block_logsumexp(mx, s, sm, ss);
         for (int c = threadIdx.x; c < C; c += blockDim.x) z[c] -= lse;
-        __syncthreads();
+    }
+}
+
+// Same result with the whole row held in registers (C <= 256*4*V, 16-byte aligned rows):
+// every logit is read from memory once and written once.
+template <int V>
+__global__ void __launch_bounds__(256)
+log_softmax_rows_reg_kernel(float* __restrict__ Z, int ldz, int M, int C) {
+    __shared__ float sm[8], ss[8];
+    const int c4 = C >> 2;  // C % 4 == 0
+    for (int row = blockIdx.x; row < M; row += gridDim.x) {
+        float4* z = reinterpret_cast<float4*>(Z + (size_t)row * ldz);
+        float4 v[V];
+        float mx = -FLT_MAX;
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const int c = threadIdx.x + i * 256;
+            v[i] = c < c4 ? z[c] : make_float4(-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX);
+            mx = fmaxf(fmaxf(mx, fmaxf(v[i].x, v[i].y)), fmaxf(v[i].z, v[i].w));
+        }
+        float s = 0.f;
+#pragma unroll
+        for (int i = 0; i < V; ++i)
+            if (threadIdx.x + i * 256 < c4)
+                s += expf(v[i].x - mx) + expf(v[i].y - mx) + expf(v[i].z - mx) + expf(v[i].w - mx);
+        const float lse = block_logsumexp(mx, s, sm, ss);
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const int c = threadIdx.x + i * 256;
+            if (c < c4) z[c] = make_float4(v[i].x - lse, v[i].y - lse, v[i].z - lse, v[i].w - lse);
+        }
     }
 }
 
@@ -249,8 +285,14 @@ int launch_real_gemm(const RealGemmArgs& a, cudaStream_t st) {
 }
 
 int launch_log_softmax_rows(float* Z, int ldz, int M, int C, cudaStream_t st) {
-    int blocks = M < 148 * 8 ? M : 148 * 8;
-    log_softmax_rows_kernel<<<blocks, 256, 0, st>>>(Z, ldz, M, C);
+    const int blocks = M < 148 * 8 ? M : 148 * 8;
+    const bool reg = (C % 4 == 0) && (ldz % 4 == 0) && aligned16(Z) && C <= 256 * 4 * 4;
+    if (reg && C <= 256 * 4 * 2)
+        log_softmax_rows_reg_kernel<2><<<blocks, 256, 0, st>>>(Z, ldz, M, C);
+    else if (reg)
+        log_softmax_rows_reg_kernel<4><<<blocks, 256, 0, st>>>(Z, ldz, M, C);
+    else
+        log_softmax_rows_kernel<<<blocks, 256, 0, st>>>(Z, ldz, M, C);
     return launch_status();
 }
 

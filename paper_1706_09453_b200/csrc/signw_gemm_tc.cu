@@ -42,22 +42,6 @@ struct Control {
     int abort;
 };
 
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-__device__ __forceinline__ bool epi_all(bool pred) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 p, %1, 0;\n\t"
-        "barrier.red.and.pred q, 2, 128, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r) : "r"((uint32_t)pred) : "memory");
-    return r != 0;
-}
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int lane) {
-    int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
-    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
-}
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -182,17 +166,16 @@ __global__ void __launch_bounds__(THREADS, 1) signw_tc_kernel(Args g) {
             for (int t = 0; t < 16; ++t) wv[t] = ((nw << (15 - t)) & 0x80008000u) | 0x3F803F80u;
 
             if (!warp_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag, lane)) break;
-            uint8_t* st = smem + s * C::STAGE_BYTES;
+            const uint32_t st = smem_u32(smem) + s * C::STAGE_BYTES;
 #pragma unroll
             for (int q = 0; q < NT; ++q)
 #pragma unroll
                 for (int c = 0; c < 2; ++c)
-                    *reinterpret_cast<uint4*>(st + q * A_PLANE + ((h * 2 + c) * BM + ra) * 16) =
-                        make_uint4(term[q][4 * c], term[q][4 * c + 1], term[q][4 * c + 2], term[q][4 * c + 3]);
+                    sts128(st + q * A_PLANE + ((h * 2 + c) * BM + ra) * 16,
+                           term[q][4 * c], term[q][4 * c + 1], term[q][4 * c + 2], term[q][4 * c + 3]);
 #pragma unroll
             for (int c = 0; c < 4; ++c)
-                *reinterpret_cast<uint4*>(st + NT * A_PLANE + (c * BN + p) * 16) =
-                    make_uint4(wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
+                sts128(st + NT * A_PLANE + (c * BN + p) * 16, wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));

@@ -16,6 +16,9 @@
 // Warp roles: warps 0-3 epilogue (TMEM -> thresholds -> packed bits / int32), warp 4 issues
 // the MMAs, warps 5-16 are producers (one packed row each per stage).  Two accumulator
 // buffers in TMEM (2 x 256 columns) let the epilogue of tile i overlap the MMAs of tile i+1.
+// The row popcounts the identity needs cost nothing extra: each producer thread sees every
+// word of its row anyway, sums their popcounts and hands the total to the epilogue through a
+// small ring in shared memory.
 #include "bnn_common.cuh"
 #include "tcgen05.cuh"
 
@@ -36,50 +39,111 @@ constexpr int THREADS = (PROD_WARP0 + PROD_WARPS) * 32;  // 544
 constexpr int PREFETCH = 3;                              // packed words in flight per producer
 constexpr uint32_t TMEM_COLS = 512;
 
+// Producers may run up to STAGES tiles ahead of the MMA warp (when a tile is a single stage)
+// and the MMA warp up to 2 tiles ahead of the epilogue, hence the depth of the popcount ring.
+constexpr int RING = 8;
+
 struct Control {
     int T[BN];              // per-unit constant of the epilogue (threshold or 2 popc(w) - K)
     uint32_t flipw[BN / 32];
-    uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
+    int popc[RING][BM + BN];  // per tile: popcount of each frame row, then of each unit row
+    uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], popc_ready[RING];
     uint32_t tmem_base;
     int abort;
 };
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + (int)sizeof(Control) + 128;
 
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// AND of a predicate over the 128 epilogue threads (named barrier 2)
-__device__ __forceinline__ bool epi_all(bool pred) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 p, %1, 0;\n\t"
-        "barrier.red.and.pred q, 2, 128, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r) : "r"((uint32_t)pred) : "memory");
-    return r != 0;
-}
 
-// One lane waits, the whole warp gets the same answer.
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int lane) {
-    int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
-    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
-}
 
-// popcount of the valid bits of one packed row
-__device__ __forceinline__ int row_popc(const uint32_t* __restrict__ row, int kw, uint32_t tmask) {
-    int s = 0;
-    const int full4 = (kw - 1) >> 2;  // 16-byte chunks that lie entirely before the last word
-    for (int q = 0; q < full4; ++q) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(row) + q);
-        s += __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
+struct ProducerArgs {
+    uint32_t smem;        // shared-space address of stage 0
+    Control* ctl;
+    volatile int* abort_flag;
+    int tiles, m_tiles, nks, kw;
+    uint32_t tmask;
+    int lane;
+};
+
+// Producer loop of one thread: row `r` of every tile of this CTA, stage by stage.  IS_A picks
+// the operand (frames / units): tile height, byte weights 2^t / 2^(7-t) and the slot in the
+// popcount ring are compile-time, so a stage is ~80 instructions.
+template <bool IS_A>
+__device__ __forceinline__ void produce(const ProducerArgs& a, const uint32_t* __restrict__ base, int ld,
+                                        int rows, int r) {
+    constexpr int ROWS = IS_A ? BM : BN;
+    Control* ctl = a.ctl;
+    const int my_tiles = (a.tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
+    const int total = my_tiles * a.nks;
+    const uint32_t dst0 = a.smem + (IS_A ? 0 : A_BYTES) + r * 16;
+
+    // prefetch cursor: the divisions happen once per tile, not per stage
+    int pf_left = total, pf_ks = 0, pf_tile = blockIdx.x;
+    const uint4* pf_ptr = nullptr;
+    auto set_row = [&]() {
+        const int row = (IS_A ? (pf_tile % a.m_tiles) * BM : (pf_tile / a.m_tiles) * BN) + r;
+        pf_ptr = row < rows ? reinterpret_cast<const uint4*>(base + (size_t)row * ld) : nullptr;
+    };
+    set_row();
+    auto fetch = [&]() -> uint4 {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (pf_left > 0) {
+            --pf_left;
+            if (pf_ptr) v = __ldg(pf_ptr + pf_ks);
+            if (++pf_ks == a.nks) {      // last stage of the row: clear the bits at positions >= K
+                const int last = a.kw - 1 - 4 * (a.nks - 1);
+                if (last == 0) { v.x &= a.tmask; v.y = 0u; v.z = 0u; v.w = 0u; }
+                else if (last == 1) { v.y &= a.tmask; v.z = 0u; v.w = 0u; }
+                else if (last == 2) { v.z &= a.tmask; v.w = 0u; }
+                else { v.w &= a.tmask; }
+                pf_ks = 0;
+                pf_tile += gridDim.x;
+                set_row();
+            }
+        }
+        return v;
+    };
+
+    uint4 ring[PREFETCH];
+#pragma unroll
+    for (int j = 0; j < PREFETCH; ++j) ring[j] = fetch();
+    int pc = 0, ks = 0, slot = 0, s = 0;
+    uint32_t ph = 1;  // parity to wait for on `empty`: a fresh barrier passes parity 1
+    for (int it = 0; it < total; ++it) {
+        uint4 v = ring[0];
+#pragma unroll
+        for (int j = 0; j + 1 < PREFETCH; ++j) ring[j] = ring[j + 1];
+        ring[PREFETCH - 1] = fetch();
+        pc += __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
+        if (!IS_A) {  // reverse the bits inside each byte, so that bit t carries weight 2^(7-t)
+            v.x = __brev(__byte_perm(v.x, 0, 0x0123));
+            v.y = __brev(__byte_perm(v.y, 0, 0x0123));
+            v.z = __brev(__byte_perm(v.z, 0, 0x0123));
+            v.w = __brev(__byte_perm(v.w, 0, 0x0123));
+        }
+        if (!warp_wait(smem_u32(&ctl->empty[s]), ph, a.abort_flag, a.lane)) break;
+        const uint32_t dst = dst0 + s * STAGE_BYTES;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            constexpr uint32_t one = 0x01010101u;
+            const uint32_t mk = IS_A ? (one << t) : (one << (7 - t));
+            sts128(dst + t * (ROWS * 16), v.x & mk, v.y & mk, v.z & mk, v.w & mk);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (a.lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
+        if (++ks == a.nks) {  // row finished: publish its popcount for this tile
+            // The slot was last read by the epilogue of the tile RING tiles back, which is done:
+            // this tile's stages could only be filled after the MMAs of the tile STAGES back had
+            // run, and those waited for the epilogue two tiles before that.
+            ctl->popc[slot][(IS_A ? 0 : BM) + r] = pc;
+            __syncwarp();
+            if (a.lane == 0) mbar_arrive(smem_u32(&ctl->popc_ready[slot]));
+            pc = 0; ks = 0;
+            slot = (slot + 1) % RING;
+        }
     }
-    for (int k = full4 << 2; k < kw; ++k) {
-        uint32_t v = __ldg(row + k);
-        if (k == kw - 1) v &= tmask;
-        s += __popc(v);
-    }
-    return s;
 }
 
 template <bool STORE_C, bool SIGN_PACK>
@@ -109,6 +173,7 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
         }
+        for (int b = 0; b < RING; ++b) mbar_init(smem_u32(&ctl->popc_ready[b]), PROD_WARPS);
         ctl->abort = 0;
         mbar_init_fence();
     }
@@ -123,66 +188,10 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
 
     if (warp >= PROD_WARP0) {
         // ---------------- producers: packed words -> widened byte tiles in shared memory
-        const int p = threadIdx.x - PROD_WARP0 * 32;  // 0..383
-        const bool is_a = p < BM;
-        const int r = is_a ? p : p - BM;
-        const uint32_t* base = is_a ? Ap : Wp;
-        const int ld = is_a ? ldap : ldwp;
-        const int rows = is_a ? M : N;
-        const int rows_tile = is_a ? BM : BN;
-        const uint32_t dst_off = (is_a ? 0 : A_BYTES) + r * 16;
-        const int my_tiles = (tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
-        const int total = my_tiles * nks;  // stages this CTA runs
-
-        // prefetch cursor: stage `pf_ks` of this CTA's tile number `pf_tl`
-        int pf_i = 0, pf_ks = 0, pf_tile = blockIdx.x;
-        auto fetch = [&]() -> uint4 {
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (pf_i < total) {
-                const int row = (is_a ? (pf_tile % m_tiles) * BM : (pf_tile / m_tiles) * BN) + r;
-                const int k0 = pf_ks * 4;  // first word of this stage
-                if (row < rows && k0 < kw) {
-                    v = __ldg(reinterpret_cast<const uint4*>(base + (size_t)row * ld + k0));
-                    const int last = kw - 1 - k0;  // index of the last valid word in this chunk
-                    if (last == 0) { v.x &= tmask; v.y = 0u; v.z = 0u; v.w = 0u; }
-                    else if (last == 1) { v.y &= tmask; v.z = 0u; v.w = 0u; }
-                    else if (last == 2) { v.z &= tmask; v.w = 0u; }
-                    else if (last == 3) { v.w &= tmask; }
-                }
-                ++pf_i;
-                if (++pf_ks == nks) { pf_ks = 0; pf_tile += gridDim.x; }
-            }
-            return v;
-        };
-
-        uint4 ring[PREFETCH];
-#pragma unroll
-        for (int j = 0; j < PREFETCH; ++j) ring[j] = fetch();
-        for (int it = 0; it < total; ++it) {
-            const int s = it % STAGES;
-            const uint32_t ph = (uint32_t)((it / STAGES) & 1);
-            uint4 v = ring[0];
-#pragma unroll
-            for (int j = 0; j + 1 < PREFETCH; ++j) ring[j] = ring[j + 1];
-            ring[PREFETCH - 1] = fetch();
-            if (!is_a) {  // reverse the bits inside each byte
-                v.x = __brev(__byte_perm(v.x, 0, 0x0123));
-                v.y = __brev(__byte_perm(v.y, 0, 0x0123));
-                v.z = __brev(__byte_perm(v.z, 0, 0x0123));
-                v.w = __brev(__byte_perm(v.w, 0, 0x0123));
-            }
-            if (!warp_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag, lane)) break;
-            uint8_t* dst = smem + s * STAGE_BYTES + dst_off;
-#pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const uint32_t mk = is_a ? (0x01010101u << t) : (0x01010101u << (7 - t));
-                *reinterpret_cast<uint4*>(dst + t * (rows_tile * 16)) =
-                    make_uint4(v.x & mk, v.y & mk, v.z & mk, v.w & mk);
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
-        }
+        const int p = threadIdx.x - PROD_WARP0 * 32;  // 0..383; a warp is all-A or all-W
+        ProducerArgs pa{smem_u32(smem), ctl, abort_flag, tiles, m_tiles, nks, kw, tmask, lane};
+        if (p < BM) produce<true>(pa, Ap, ldap, M, p);
+        else produce<false>(pa, Wp, ldwp, N, p - BM);
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issue: one thread
         if (lane == 0) {
@@ -223,15 +232,18 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
         for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
             const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
             const int m = m0 + row_in_tile;
-            // per-frame and per-unit popcounts of this tile (overlaps the MMAs of the tile)
-            const int pa = m < M ? row_popc(Ap + (size_t)m * ldap, kw, tmask) : 0;
+            // row popcounts of this tile, published by the producers
+            ok = epi_all(warp_wait(smem_u32(&ctl->popc_ready[tl % RING]), (uint32_t)((tl / RING) & 1), abort_flag, lane));
+            if (!ok) break;
+            const int* pcs = ctl->popc[tl % RING];
+            const int pa = pcs[row_in_tile];
             epi_bar_sync();  // previous tile's readers of T are done
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int nl = row_in_tile + h * 128, n = n0 + nl;
                 int t = 0;
                 if (n < N) {
-                    const int pw = row_popc(Wp + (size_t)n * ldwp, kw, tmask);
+                    const int pw = pcs[BM + nl];
                     t = (SIGN_PACK && !STORE_C) ? 32 * (thr[n] + 2 * pw - K) : 2 * pw - K;
                 }
                 ctl->T[nl] = t;
