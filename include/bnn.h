@@ -208,6 +208,28 @@ BNN_API int bnn_forward(const bnn_model* model, const float* X, int ldx, int M,
                 float* logp, int ldo, void* workspace, size_t workspace_bytes,
                 void* const* layer_out, void* stream);
 
+/* The forward pass for callers that cannot allocate device memory -- for instance a
+ * real-time decoding thread (cudaMalloc stalls the whole device), a plug-in whose host
+ * program fixes its memory budget at start-up, or a process that has given all device memory
+ * to another pool.  Same result as bnn_forward, but the scratch is a fixed array of
+ * BNN_STATIC_WORKSPACE_BYTES inside the library image instead of a caller buffer; every GPU
+ * that loads the library holds those bytes until the process exits.  The paper has no
+ * counterpart.
+ *   - Inputs and outputs (model, X, logp) are still the caller's.
+ *   - Limit: bnn_forward_workspace_bytes(model, M) must not exceed the array; otherwise the
+ *     call launches nothing and returns BNN_ERR_WORKSPACE.  (8 MiB holds 16384 frames of a
+ *     2048-wide binary-activation network, or 512 frames with fp32 hardtanh activations.)
+ *   - This call makes no cudaMalloc/cudaFree and uses no allocating library routine.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside of any stream capture.
+ *   - All calls share the one array, which keeps whatever the last call left in it (nothing
+ *     needs clearing: each layer only reads what the previous layer wrote in the same call).
+ *     Two calls whose kernels can overlap on the GPU -- different streams, or several host
+ *     threads -- race on it: run them one after the other. */
+#define BNN_STATIC_WORKSPACE_BYTES (8u << 20)
+BNN_API int bnn_forward_static(const bnn_model* model, const float* X, int ldx, int M,
+                               float* logp, int ldo, void* stream);
+
 /* bnn_forward that also records events on `stream` so a caller can time each layer where it
  * runs.  events : HOST array of n_layers+2 cudaEvent_t (NULL entries skipped): events[l] is
  * recorded before layer l, events[n_layers] after the last kernel, events[n_layers+1]

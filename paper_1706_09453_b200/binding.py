@@ -82,6 +82,8 @@ def lib():
         L.bnn_signw_gemm.argtypes = [p, i, p, i, i, i, i, p, i, C.POINTER(Epilogue), p]
         L.bnn_output_layer.argtypes = [p, i, p, i, p, i, p, p, i, i, i, p, i, i, p]
         L.bnn_forward.argtypes = [C.POINTER(Model), p, i, i, p, i, p, C.c_size_t, C.POINTER(p), p]
+        L.bnn_forward_static.argtypes = [C.POINTER(Model), p, i, i, p, i, p]
+        L.bnn_forward_static.restype = C.c_int
         L.bnn_forward_events.argtypes = [C.POINTER(Model), p, i, i, p, i, p, C.c_size_t, C.POINTER(p),
                                          C.POINTER(p), p]
         for name in ("bnn_pack_weights", "bnn_binarize_pack", "bnn_fold_thresholds", "bnn_xnor_gemm",
@@ -271,4 +273,16 @@ def bnn_forward_events(model: ModelDesc, X, logp, workspace, events, layer_out=N
                                     _ptr(logp, torch.float32), _ld(logp),
                                     _ptr(workspace), workspace.numel() * workspace.element_size(),
                                     lo, ev, _stream()), "bnn_forward_events")
+    return logp
+
+
+STATIC_WORKSPACE_BYTES = 8 << 20
+
+
+def bnn_forward_static(model: ModelDesc, X, logp):
+    """Forward pass that allocates nothing: its scratch is a fixed array inside the library
+    (for callers that may not call cudaMalloc).  Raises BnnError(status 5) when the batch
+    needs more than STATIC_WORKSPACE_BYTES of scratch."""
+    _check(lib().bnn_forward_static(C.byref(model.c), _ptr(X, torch.float32), _ld(X), X.shape[0],
+                                    _ptr(logp, torch.float32), _ld(logp), _stream()), "bnn_forward_static")
     return logp
