@@ -37,7 +37,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="wsj", choices=["tiny", "wsj", "wsj_bw", "ami"])
     ap.add_argument("--frames", type=int, default=None, help="override the batch size (frames per step)")
-    ap.add_argument("--cpu-frames", type=int, default=2048, help="frames of the workload the CPU oracle is timed on")
+    ap.add_argument("--cpu-frames", type=int, default=16384, help="frames of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--real-path", default="tensor", choices=["tensor", "fp32"],
                     help="kernel of the real-valued layers: tcgen05 with split operands or the FP32 pipe")
@@ -214,6 +214,22 @@ def hbm_bytes_per_step(cfg, frames):
     return b
 
 
+def ncu_traffic(kernel):
+    """DRAM bytes (read + write) per launch of `kernel` from the committed ncu capture, or
+    None when there is none or the kernel's source has changed since it was taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    rec = json.load(open(path)).get(kernel)
+    if not rec:
+        return None
+    src = os.path.join(ROOT, "paper_1706_09453_b200", "csrc", rec["source"])
+    if not os.path.exists(src) or hashlib.sha256(open(src, "rb").read()).hexdigest() != rec["source_sha256"]:
+        return None
+    return rec["dram_bytes_per_launch"]
+
+
 # ------------------------------------------------------------------ GPU arm
 def run_ours(args):
     import torch
@@ -323,15 +339,28 @@ def run_ours(args):
         r["achieved"] = r["work"] / (t * 1e-3) / r.get("scale", 1e12)
         r["frac"] = r["achieved"] / r["peak"]
         r["pipe_util"] = r["frac"] * r.get("passes", 1)
-    dom = max(rows, key=lambda r: r["ms"])
-    share = dom["ms"] / sum(layer_ms)
-    roofline = {"kernel": dom["kernel"], "layer": dom["name"], "bound": dom["bound"],
-                "achieved": dom["achieved"], "peak": dom["peak"], "unit": dom["unit"],
-                "frac": dom["frac"], "traffic": None,
-                "peak_source": ("2 x bf16_tflops_sustained of MEASURED_PEAKS.json (%s)" % peaks["source"])
-                if dom["bound"] == "tensor" else
-                "derived from unit counts x max SM clock (%.0f MHz)" % peaks["sm_max_mhz"],
-                "share_of_step": share, "avg_launch_ms": dom["ms"]}
+    # dominant KERNEL: group the layers by the kernel that runs them (the five binary hidden
+    # layers are five launches of one kernel) and take the largest share of the step
+    groups = {}
+    for r in rows:
+        gk = groups.setdefault(r["kernel"], dict(ms=0.0, work=0.0, n=0, row=r))
+        gk["ms"] += r["ms"]; gk["work"] += r["work"]; gk["n"] += 1
+    dk, dg = max(groups.items(), key=lambda kv: kv[1]["ms"])
+    dom = dg["row"]
+    achieved = dg["work"] / (dg["ms"] * 1e-3) / dom.get("scale", 1e12)
+    roofline = {"kernel": dk, "launches_per_step": dg["n"], "bound": dom["bound"],
+                "achieved": achieved, "peak": dom["peak"], "unit": dom["unit"],
+                "frac": achieved / dom["peak"], "traffic": ncu_traffic(dk),
+                "peak_source": ("2 x bf16_tflops_sustained of MEASURED_PEAKS.json (%s): u8 MMA = 2 x bf16 (nominal ratio), "
+                                "sustained figure because the kernel is timed inside a long step; of measured"
+                                % peaks["source"]) if dk == "xnor_tc_kernel" else
+                               ("bf16_tflops_sustained of MEASURED_PEAKS.json (%s); of measured" % peaks["source"])
+                               if dom["bound"] == "tensor" else
+                               ("hbm_gbs of MEASURED_PEAKS.json (%s); of measured" % peaks["source"])
+                               if dom["bound"] == "hbm" else
+                               "derived from unit counts x max SM clock (%.0f MHz)" % peaks["sm_max_mhz"],
+                "algorithmic_work_per_launch": dg["work"] / dg["n"],
+                "share_of_step": dg["ms"] / sum(layer_ms), "avg_launch_ms": dg["ms"] / dg["n"]}
     fps = world * frames * K / (total_ms * 1e-3)
     xnor_work = sum(r["work"] for r in rows if r["name"].startswith("xnor"))
     xnor_ms = sum(r["ms"] for r in rows if r["name"].startswith("xnor"))
