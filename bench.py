@@ -39,6 +39,9 @@ def parse_args():
     ap.add_argument("--frames", type=int, default=None, help="override the batch size (frames per step)")
     ap.add_argument("--cpu-frames", type=int, default=16384, help="frames of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="isolated XNOR GEMM sweep (M x K x N x bit density), one JSON line per point")
+    ap.add_argument("--sweep-quick", action="store_true", help="only the corner points of the sweep")
     ap.add_argument("--real-path", default="tensor", choices=["tensor", "fp32"],
                     help="kernel of the real-valued layers: tcgen05 with split operands or the FP32 pipe")
     ap.add_argument("--xnor-path", default="tensor", choices=["tensor", "popc"],
@@ -401,9 +404,91 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Isolated XNOR-popcount GEMM, int32 output, on both kernels; binary-op/s and GB/s per point
+    against max(bytes / HBM bandwidth, bops / tensor peak).  Inputs are drawn on the device and
+    packed with the library's own bnn_binarize_pack; a few rows of every point are checked
+    against the CPU oracle."""
+    import torch
+    from paper_1706_09453_b200 import build
+    build.build()
+    from paper_1706_09453_b200 import binding as B, model, workloads as wl
+    from oracle import bnn_oracle as o
+    peaks = load_peaks()
+    dev = "cuda:0"
+    Ms, Ks, Ns = wl.SWEEP_M, wl.SWEEP_K, wl.SWEEP_N
+    if args.sweep_quick:
+        Ms, Ks, Ns = (Ms[0], Ms[-1]), (Ks[0], Ks[-1]), (Ns[0], Ns[-1])
+    gen = torch.Generator(device=dev)
+
+    def planes(rows, k, p, seed):
+        gen.manual_seed(seed)
+        out = model.packed_empty(rows, k, dev)
+        step = max(1, (1 << 28) // k)      # pack in slabs of <= 1 GiB of floats
+        for r0 in range(0, rows, step):
+            r1 = min(rows, r0 + step)
+            x = torch.rand((r1 - r0, k), device=dev, generator=gen)
+            x = (p - x)                      # >= 0 with probability p  ->  bit 1
+            B.bnn_binarize_pack(x, out[r0:r1], B.SIGN_ZERO_NEG)
+        return out
+
+    def timeit(fn, n):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    for p in wl.SWEEP_P:
+        for M in Ms:
+            for K in Ks:
+                A = planes(M, K, p, 1000 + M + K)
+                for N in Ns:
+                    W = planes(N, K, p, 2000 + N + K)
+                    # rotate over enough output buffers that C is never found in L2
+                    cbytes = M * N * 4
+                    nbuf = max(1, min(4, -(-2 * L2_BYTES // cbytes)))
+                    Cs = [torch.empty((M, N), dtype=torch.int32, device=dev) for _ in range(nbuf)]
+                    bops = 2.0 * M * N * K
+                    nbytes = M * K / 8 + N * K / 8 + cbytes
+                    rec = {"sweep": True, "M": M, "K": K, "N": N, "p": p, "bops": bops, "bytes": nbytes}
+                    it = [0]
+                    for name, path in (("tensor", B.XNOR_TENSOR), ("popc", B.XNOR_POPC)):
+                        B.bnn_set_xnor_path(path)
+                        def call():
+                            B.bnn_xnor_gemm(A, W, K, C_out=Cs[it[0] % nbuf]); it[0] += 1
+                        reps = 5 if bops > 1e12 else 20
+                        if name == "popc" and bops > 2e12:
+                            reps = 2
+                        ms = timeit(call, reps)
+                        rec[name] = {"ms": ms, "tbops": bops / ms / 1e9, "gbs": nbytes / ms / 1e6}
+                    t_roof = max(nbytes / (peaks["hbm_gbs"] * 1e9), bops / (2 * peaks["bf16_tflops"] * 1e12))
+                    rec["bound"] = "hbm" if nbytes / (peaks["hbm_gbs"] * 1e9) > bops / (2 * peaks["bf16_tflops"] * 1e12) else "tensor"
+                    rec["roofline_frac_tensor_kernel"] = t_roof / (rec["tensor"]["ms"] * 1e-3)
+                    # parity on sampled rows (first, last, two in between)
+                    B.bnn_set_xnor_path(B.XNOR_TENSOR)
+                    B.bnn_xnor_gemm(A, W, K, C_out=Cs[0])
+                    rows = sorted({0, M // 3, (2 * M) // 3, M - 1})
+                    got = Cs[0][rows].cpu().numpy()
+                    want = o.xnor_gemm(model.words_to_numpy(A[rows], K), model.words_to_numpy(W, K), K)
+                    rec["parity_rows_checked"] = len(rows)
+                    rec["parity_ok"] = bool((got == want).all())
+                    rec["device_status"] = B.bnn_device_status()
+                    print(json.dumps(rec), flush=True)
+                    del Cs, W
+                del A
+
+
 if __name__ == "__main__":
     a = parse_args()
-    if a.impl == "reference":
+    if a.sweep:
+        run_sweep(a)
+    elif a.impl == "reference":
         run_reference(a)
     else:
         run_ours(a)
