@@ -12,10 +12,14 @@
 //     bytes first so its byte holds 2^(7-t); every product is then 2^7 * a * w and the
 //     accumulator is exactly 128 * popc(a AND w) (u8 x u8 -> s32).
 //
-// One persistent CTA per SM, tile 128 frames x 256 units, 128 bits of K per pipeline stage.
+// One persistent CTA per SM, tile 128 frames x 192 units, 128 bits of K per pipeline stage.
 // Warp roles: warps 0-3 epilogue (TMEM -> thresholds -> packed bits / int32), warp 4 issues
-// the MMAs, warps 5-16 are producers (one packed row each per stage).  Two accumulator
-// buffers in TMEM (2 x 256 columns) let the epilogue of tile i overlap the MMAs of tile i+1.
+// the MMAs, warps 5-8 widen the frame rows and warps 9-14 the unit rows (one packed row per
+// thread and stage).  The kernel is bound by the shared-memory pipe, not by the tensor pipe,
+// so the frame operand never touches shared memory: its producers write the widened bytes
+// straight into tensor memory (tcgen05.st, lane = frame) and the MMA reads A from there.
+// TMEM budget (512 columns): two 192-column accumulators, so that the epilogue of tile i
+// overlaps the MMAs of tile i+1, plus 4 stages x 32 columns of A.
 // The row popcounts the identity needs cost nothing extra: each producer thread sees every
 // word of its row anyway, sums their popcounts and hands the total to the epilogue through a
 // small ring in shared memory.
@@ -31,11 +35,14 @@ namespace {
 
 using namespace tc;
 
-constexpr int BM = 128, BN = 256, BK = 128;  // BK: bits of K per stage = bytes per widened row
+constexpr int BM = 128, BN = 192, BK = 128;  // BK: bits of K per stage = bytes per widened row
 constexpr int STAGES = 4;
-constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int EPI_WARPS = 4, MMA_WARP = 4, PROD_WARP0 = 5, PROD_WARPS = 12;
-constexpr int THREADS = (PROD_WARP0 + PROD_WARPS) * 32;  // 544
+constexpr int B_BYTES = BN * BK, STAGE_BYTES = B_BYTES;  // only the unit operand lives in shared memory
+constexpr int EPI_WARPS = 4, MMA_WARP = 4, PROD_WARP0 = 5, A_WARPS = 4, B_WARPS = BN / 32;
+constexpr int PROD_WARPS = A_WARPS + B_WARPS;
+constexpr int THREADS = (PROD_WARP0 + PROD_WARPS) * 32;  // 480
+constexpr uint32_t TMEM_A_COL = 2 * BN;                  // A stages start after the two accumulators
+constexpr uint32_t A_COLS = BK / 4;                      // 32-bit columns per A stage
 constexpr int PREFETCH = 3;                              // packed words in flight per producer
 constexpr uint32_t TMEM_COLS = 512;
 
@@ -58,6 +65,7 @@ constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + (int)sizeof(Control) + 128;
 
 struct ProducerArgs {
     uint32_t smem;        // shared-space address of stage 0
+    uint32_t tmem;        // base of the tensor-memory allocation
     Control* ctl;
     volatile int* abort_flag;
     int tiles, m_tiles, nks, kw;
@@ -71,11 +79,12 @@ struct ProducerArgs {
 template <bool IS_A>
 __device__ __forceinline__ void produce(const ProducerArgs& a, const uint32_t* __restrict__ base, int ld,
                                         int rows, int r) {
-    constexpr int ROWS = IS_A ? BM : BN;
     Control* ctl = a.ctl;
     const int my_tiles = (a.tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
     const int total = my_tiles * a.nks;
-    const uint32_t dst0 = a.smem + (IS_A ? 0 : A_BYTES) + r * 16;
+    const uint32_t dst0 = a.smem + r * 16;
+    // TMEM lane of this thread's frame row: a warp may only touch lanes 32*(warp%4)..+31
+    const uint32_t tdst0 = a.tmem + ((uint32_t)(r & ~31) << 16) + TMEM_A_COL;
 
     // prefetch cursor: the divisions happen once per tile, not per stage
     int pf_left = total, pf_ks = 0, pf_tile = blockIdx.x;
@@ -122,14 +131,28 @@ __device__ __forceinline__ void produce(const ProducerArgs& a, const uint32_t* _
             v.w = __brev(__byte_perm(v.w, 0, 0x0123));
         }
         if (!warp_wait(smem_u32(&ctl->empty[s]), ph, a.abort_flag, a.lane)) break;
-        const uint32_t dst = dst0 + s * STAGE_BYTES;
+        if (IS_A) {
+            // column 4t+i of the stage holds bytes 16t+4i .. 16t+4i+3 of K: the same order as
+            // the 16-byte chunks of the unit operand in shared memory
+            uint32_t wr[32];
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            constexpr uint32_t one = 0x01010101u;
-            const uint32_t mk = IS_A ? (one << t) : (one << (7 - t));
-            sts128(dst + t * (ROWS * 16), v.x & mk, v.y & mk, v.z & mk, v.w & mk);
+            for (int t = 0; t < 8; ++t) {
+                const uint32_t mk = 0x01010101u << t;
+                wr[4 * t + 0] = v.x & mk; wr[4 * t + 1] = v.y & mk;
+                wr[4 * t + 2] = v.z & mk; wr[4 * t + 3] = v.w & mk;
+            }
+            tmem_st32(tdst0 + s * A_COLS, wr);
+            tmem_st_wait();
+            tc_fence_before_sync();
+        } else {
+            const uint32_t dst = dst0 + s * STAGE_BYTES;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const uint32_t mk = 0x01010101u << (7 - t);
+                sts128(dst + t * (BN * 16), v.x & mk, v.y & mk, v.z & mk, v.w & mk);
+            }
+            fence_proxy_async_smem();
         }
-        fence_proxy_async_smem();
         __syncwarp();
         if (a.lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
         if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -188,10 +211,9 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
 
     if (warp >= PROD_WARP0) {
         // ---------------- producers: packed words -> widened byte tiles in shared memory
-        const int p = threadIdx.x - PROD_WARP0 * 32;  // 0..383; a warp is all-A or all-W
-        ProducerArgs pa{smem_u32(smem), ctl, abort_flag, tiles, m_tiles, nks, kw, tmask, lane};
-        if (p < BM) produce<true>(pa, Ap, ldap, M, p);
-        else produce<false>(pa, Wp, ldwp, N, p - BM);
+        ProducerArgs pa{smem_u32(smem), tmem, ctl, abort_flag, tiles, m_tiles, nks, kw, tmask, lane};
+        if (warp < PROD_WARP0 + A_WARPS) produce<true>(pa, Ap, ldap, M, (warp & 3) * 32 + lane);
+        else produce<false>(pa, Wp, ldwp, N, (warp - PROD_WARP0 - A_WARPS) * 32 + lane);
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issue: one thread
         if (lane == 0) {
@@ -210,13 +232,12 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
                     ok = mbar_wait(smem_u32(&ctl->full[s]), (uint32_t)((it / STAGES) & 1), abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t a0 = smem_u32(smem + s * STAGE_BYTES);
-                    const uint32_t b0 = a0 + A_BYTES;
+                    const uint32_t b0 = smem_u32(smem + s * STAGE_BYTES);
+                    const uint32_t ta = tmem + TMEM_A_COL + s * A_COLS;
 #pragma unroll
-                    for (int j = 0; j < BK / 32; ++j) {
-                        const uint64_t da = smem_desc_kmajor(a0 + 2 * j * (BM * 16), BM * 16, 128);
+                    for (int j = 0; j < BK / 32; ++j) {   // 32 bytes of K = 8 TMEM columns of A per MMA
                         const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (BN * 16), BN * 16, 128);
-                        mma_i8(d, da, db, idesc, (ks | j) != 0);
+                        mma_i8_ts(d, ta + 8 * j, db, idesc, (ks | j) != 0);
                     }
                     mma_commit(smem_u32(&ctl->empty[s]));
                 }
@@ -241,12 +262,14 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int nl = row_in_tile + h * 128, n = n0 + nl;
-                int t = 0;
-                if (n < N) {
-                    const int pw = pcs[BM + nl];
-                    t = (SIGN_PACK && !STORE_C) ? 32 * (thr[n] + 2 * pw - K) : 2 * pw - K;
+                if (nl < BN) {
+                    int t = 0;
+                    if (n < N) {
+                        const int pw = pcs[BM + nl];
+                        t = (SIGN_PACK && !STORE_C) ? 32 * (thr[n] + 2 * pw - K) : 2 * pw - K;
+                    }
+                    ctl->T[nl] = t;
                 }
-                ctl->T[nl] = t;
             }
             if (SIGN_PACK && row_in_tile < BN / 32) {
                 const int wi = (n0 >> 5) + row_in_tile;
@@ -317,9 +340,10 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
             if (SIGN_PACK && m < M) {
                 const int nw = words_for(N), w0 = n0 >> 5;
                 uint32_t* dst = out_bits + (size_t)m * ldob + w0;
-                if (w0 + BN / 32 <= nw) {
-                    reinterpret_cast<uint4*>(dst)[0] = make_uint4(words[0], words[1], words[2], words[3]);
-                    reinterpret_cast<uint4*>(dst)[1] = make_uint4(words[4], words[5], words[6], words[7]);
+                if (w0 + BN / 32 <= nw) {   // 6 words; rows are 16-byte aligned, n0/32 is a multiple of 6
+#pragma unroll
+                    for (int q = 0; q < BN / 64; ++q)
+                        reinterpret_cast<uint2*>(dst)[q] = make_uint2(words[2 * q], words[2 * q + 1]);
                 } else {
 #pragma unroll
                     for (int g = 0; g < BN / 32; ++g)
