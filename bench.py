@@ -240,17 +240,13 @@ def run_ours(args):
     build.build()
     from paper_1706_09453_b200 import binding as B, model, workloads as wl
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_1706_09453_b200 import dist as D
+    rank, world, local = D.env_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
     torch.cuda.set_device(local)
     dev = "cuda:%d" % local
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    dist = D.init("nccl", torch.device(dev))
 
     cfg = wl.CONFIGS[args.config]
     frames = args.frames or cfg.frames
@@ -259,7 +255,7 @@ def run_ours(args):
     B.bnn_set_option(B.OPT_REAL_PATH, B.PATH_TENSOR if args.real_path == "tensor" else B.PATH_CUDA_CORE)
     dn = model.DeviceNet(net, device=dev)
     # Frames are independent, so ranks shard them with no exchange: each rank owns its own batch.
-    Xh = wl.make_frames(cfg, frames, seed=cfg.seed + 1000 * rank)
+    Xh = wl.make_frames(cfg, frames, seed=D.frames_seed(cfg.seed, rank))
     set_bytes = frames * (cfg.in_dim + cfg.classes) * 4
     nsets = max(2, -(-2 * L2_BYTES // set_bytes))          # rotate over > 2 x L2 of inputs/outputs
     Xd = [model.to_dev(Xh, dev) for _ in range(nsets)]
@@ -288,10 +284,7 @@ def run_ours(args):
     e1.record()
     barrier()
     clocks.stop()
-    ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    total_ms = float(ms.item())
+    total_ms = D.max_over_ranks(dist, e0.elapsed_time(e1), dev)
 
     # ---- per-layer device time over the same steps (events recorded inside the C-ABI call)
     nl = cfg.n_hidden + 1
@@ -323,10 +316,7 @@ def run_ours(args):
         Lp.copy_(Ld[i % nsets], non_blocking=True)
     e1.record()
     barrier()
-    ems = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(ems, op=dist.ReduceOp.MAX)
-    e2e_fps = world * frames * Ke / (float(ems.item()) * 1e-3)
+    e2e_fps = D.aggregate_rate(frames, world, Ke, D.max_over_ranks(dist, e0.elapsed_time(e1), dev))
 
     if rank != 0:
         if dist:
@@ -364,7 +354,7 @@ def run_ours(args):
                                "derived from unit counts x max SM clock (%.0f MHz)" % peaks["sm_max_mhz"],
                 "algorithmic_work_per_launch": dg["work"] / dg["n"],
                 "share_of_step": dg["ms"] / sum(layer_ms), "avg_launch_ms": dg["ms"] / dg["n"]}
-    fps = world * frames * K / (total_ms * 1e-3)
+    fps = D.aggregate_rate(frames, world, K, total_ms)
     xnor_work = sum(r["work"] for r in rows if r["name"].startswith("xnor"))
     xnor_ms = sum(r["ms"] for r in rows if r["name"].startswith("xnor"))
     hbm = hbm_bytes_per_step(cfg, frames)
