@@ -185,7 +185,7 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
         elif real_path == "tensor":
             # bf16 tensor-core MMAs, one pass per bf16 term of the real operand (2 terms);
             # algorithmic flops count the product once
-            rows.append(dict(name="signw_%d" % (l + 1), kernel="signw_tc_kernel", work=work, unit="TFLOP/s",
+            rows.append(dict(name="signw_%d" % (l + 1), kernel="x_split_kernel+signw_img_kernel", work=work, unit="TFLOP/s",
                              bound="tensor", peak=peaks["bf16_tflops_sustained"], passes=2))
         else:
             rows.append(dict(name="signw_%d" % (l + 1), kernel="real_gemm_kernel", work=work, unit="TFLOP/s",
@@ -372,7 +372,9 @@ def run_ours(args):
         "clocks": ck,
         "e2e": {"value": e2e_fps, "unit": UNIT, "h2d_bytes_per_step": int(Xp.numel() * 4),
                 "d2h_bytes_per_step": int(Lp.numel() * 4), "steps": Ke},
-        "gpu_launches": K * (cfg.n_hidden + 2),
+        # per step: one kernel per binary hidden layer, two per sign-weight layer (split + GEMM),
+        # top-layer GEMM and log-softmax
+        "gpu_launches": K * (cfg.n_hidden + 2 + (1 if cfg.act == 1 else cfg.n_hidden) * (1 if args.real_path == "tensor" else 0)),
         "paths": {"xnor": args.xnor_path, "real": args.real_path},
         "roofline": roofline,
         "layers": [{k: r[k] for k in ("name", "kernel", "bound", "ms", "achieved", "peak", "unit", "frac", "pipe_util")}

@@ -74,6 +74,13 @@ def lib():
         L.bnn_device_status.restype = C.c_int
         L.bnn_forward_workspace_bytes.restype = C.c_size_t
         L.bnn_forward_workspace_bytes.argtypes = [C.POINTER(Model), C.c_int]
+        L.bnn_forward_min_workspace_bytes.restype = C.c_size_t
+        L.bnn_forward_min_workspace_bytes.argtypes = [C.POINTER(Model), C.c_int]
+        L.bnn_signw_workspace_bytes.restype = C.c_size_t
+        L.bnn_signw_workspace_bytes.argtypes = [C.c_int, C.c_int]
+        L.bnn_signw_gemm_ws.restype = C.c_int
+        L.bnn_signw_gemm_ws.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                        C.c_int, C.POINTER(Epilogue), C.c_void_p, C.c_size_t, C.c_void_p]
         i, p = C.c_int, C.c_void_p
         L.bnn_pack_weights.argtypes = [p, i, i, i, p, i, i, p]
         L.bnn_binarize_pack.argtypes = [p, i, i, i, p, i, i, p]
@@ -197,10 +204,21 @@ def bnn_xnor_gemm(Ap, Wp, K, C_out=None, thr=None, flip=None, out_bits=None):
                                e, _stream()), "bnn_xnor_gemm")
 
 
+def bnn_signw_workspace_bytes(M, K) -> int:
+    return int(lib().bnn_signw_workspace_bytes(int(M), int(K)))
+
+
 def bnn_signw_gemm(X, Wp, K, Y=None, act=ACT_NONE, scale=None, shift=None, out_bits=None,
-                   sign_mode=SIGN_ZERO_POS):
+                   sign_mode=SIGN_ZERO_POS, workspace=None):
+    """With ``workspace`` (uint8 CUDA tensor) this calls bnn_signw_gemm_ws."""
     m, n = X.shape[0], Wp.shape[0]
     e = C.byref(_epilogue(act, sign_mode, scale, shift, out_bits=out_bits))
+    if workspace is not None:
+        _check(lib().bnn_signw_gemm_ws(_ptr(X, torch.float32), _ld(X), _ptr(Wp, torch.int32), _ld(Wp), m, n, K,
+                                       _ptr(Y, torch.float32), _ld(Y) if Y is not None else 0, e,
+                                       _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+               "bnn_signw_gemm_ws")
+        return
     _check(lib().bnn_signw_gemm(_ptr(X, torch.float32), _ld(X), _ptr(Wp, torch.int32), _ld(Wp), m, n, K,
                                 _ptr(Y, torch.float32), _ld(Y) if Y is not None else 0, e, _stream()),
            "bnn_signw_gemm")
@@ -248,6 +266,9 @@ class ModelDesc:
 
     def workspace_bytes(self, M: int) -> int:
         return int(lib().bnn_forward_workspace_bytes(C.byref(self.c), M))
+
+    def min_workspace_bytes(self, M: int) -> int:
+        return int(lib().bnn_forward_min_workspace_bytes(C.byref(self.c), M))
 
 
 def bnn_forward(model: ModelDesc, X, logp, workspace, layer_out=None):

@@ -166,9 +166,21 @@ int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
                                                         ob, ldob, (cudaStream_t)stream);
 }
 
+size_t bnn_signw_workspace_bytes(int M, int K) {
+    if (M < 1 || K < 1) return 0;
+    return signw_image_bytes(M, K, g_signw_terms);
+}
+
 int bnn_signw_gemm(const float* X, int ldx, const uint32_t* Wp, int ldwp,
                    int M, int N, int K, float* Y, int ldy,
                    const bnn_epilogue* epi, void* stream) {
+    return bnn_signw_gemm_ws(X, ldx, Wp, ldwp, M, N, K, Y, ldy, epi, nullptr, 0, stream);
+}
+
+int bnn_signw_gemm_ws(const float* X, int ldx, const uint32_t* Wp, int ldwp,
+                      int M, int N, int K, float* Y, int ldy,
+                      const bnn_epilogue* epi, void* workspace, size_t workspace_bytes,
+                      void* stream) {
     if (int rc = check_dims(M, N, K)) return rc;
     if (!X) return BNN_ERR_NULL;
     if (ldx < K) return BNN_ERR_SHAPE;
@@ -191,7 +203,12 @@ int bnn_signw_gemm(const float* X, int ldx, const uint32_t* Wp, int ldwp,
         }
     }
     if (!a.Y && !a.out_bits) return BNN_ERR_NULL;
-    if (g_real_path != BNN_PATH_CUDA_CORE) return launch_signw_tc(a, g_signw_terms, (cudaStream_t)stream);
+    if (g_real_path != BNN_PATH_CUDA_CORE) {
+        if (workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255u) &&
+            workspace_bytes >= signw_image_bytes(M, K, g_signw_terms))
+            return launch_signw_img(a, g_signw_terms, workspace, (cudaStream_t)stream);
+        return launch_signw_tc(a, g_signw_terms, (cudaStream_t)stream);
+    }
     return launch_real_gemm(a, (cudaStream_t)stream);
 }
 
@@ -251,7 +268,7 @@ int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
                              log_softmax, nullptr, stream);
 }
 
-size_t bnn_forward_workspace_bytes(const bnn_model* model, int M) {
+size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M) {
     if (validate_model(model) != BNN_OK || M < 1) return 0;
     size_t mx = 0;
     for (int l = 0; l + 1 < model->n_layers; ++l) {
@@ -259,6 +276,18 @@ size_t bnn_forward_workspace_bytes(const bnn_model* model, int M) {
         if (b > mx) mx = b;
     }
     return 2 * round256(mx) + 256;
+}
+
+size_t bnn_forward_workspace_bytes(const bnn_model* model, int M) {
+    const size_t base = bnn_forward_min_workspace_bytes(model, M);
+    if (base == 0) return 0;
+    size_t img = 0;
+    for (int l = 0; l < model->n_layers; ++l)
+        if (model->layers[l].kind == BNN_LAYER_SIGNW) {
+            const size_t b = signw_image_bytes(M, model->layers[l].K, 3);  // room for either term count
+            if (b > img) img = b;
+        }
+    return base + round256(img);
 }
 
 int bnn_forward(const bnn_model* model, const float* X, int ldx, int M,
@@ -276,13 +305,16 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
     if (M < 1 || ldx < model->layers[0].K) return BNN_ERR_SHAPE;
     const int L = model->n_layers;
     if (ldo < model->layers[L - 1].N) return BNN_ERR_SHAPE;
-    const size_t need = bnn_forward_workspace_bytes(model, M);
+    const size_t need = bnn_forward_min_workspace_bytes(model, M);
     if (L > 1) {
         if (!workspace || workspace_bytes < need) return BNN_ERR_WORKSPACE;
         if (reinterpret_cast<uintptr_t>(workspace) & 255u) return BNN_ERR_ALIGN;
     }
     char* buf[2] = {static_cast<char*>(workspace),
                     static_cast<char*>(workspace) + (need - 256) / 2};
+    // whatever lies beyond the two activation buffers serves the sign-weight layers' image
+    char* img = static_cast<char*>(workspace) + (need - 256);
+    const size_t img_bytes = workspace_bytes > need - 256 ? workspace_bytes - (need - 256) : 0;
     const void* in = X;
     int in_ld = ldx;
     bool in_bits = false;
@@ -319,8 +351,8 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                 yf = static_cast<float*>(out);
                 out_ld = y.N;
             }
-            rc = bnn_signw_gemm(static_cast<const float*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
-                                yf, y.N, &e, stream);
+            rc = bnn_signw_gemm_ws(static_cast<const float*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
+                                   yf, y.N, &e, img, img_bytes, stream);
             in_ld = out_ld;
         } else {
             e.thr = y.thr; e.flip = y.flip;

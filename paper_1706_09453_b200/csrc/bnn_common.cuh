@@ -82,6 +82,10 @@ int launch_real_gemm(const RealGemmArgs& a, cudaStream_t st);
 // Tensor-core versions: +-1 weights x real input (A fp32, B bits; `terms` bf16 terms), and
 // the top layer on packed activations with prepared fp16 weight terms.
 int launch_signw_tc(const RealGemmArgs& a, int terms, cudaStream_t st);
+// Same product with the activations split once into a scratch image (see signw_img_tc.cu):
+// `workspace` must hold signw_image_bytes(M, K, terms) bytes, 256-byte aligned.
+size_t signw_image_bytes(int M, int K, int terms);
+int launch_signw_img(const RealGemmArgs& a, int terms, void* workspace, cudaStream_t st);
 size_t out_prepared_bytes(int C, int H);
 int launch_out_prepare(const float* W, int ldw, int C, int H, void* prepared, cudaStream_t st);
 int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const float* bias,

@@ -36,7 +36,7 @@ extern "C" int bnn_forward_static(const bnn_model* model, const float* X, int ld
                                   float* logp, int ldo, void* stream) {
     if (!model) return BNN_ERR_NULL;
     if (M < 1) return BNN_ERR_SHAPE;
-    const size_t need = bnn_forward_workspace_bytes(model, M);
+    const size_t need = bnn_forward_min_workspace_bytes(model, M);
     // need == 0 means the model itself is invalid: bnn_forward reports which way.
     if (need > (size_t)BNN_STATIC_WORKSPACE_BYTES) return BNN_ERR_WORKSPACE;
     void* ws = static_workspace_for_current_device();

@@ -1,0 +1,376 @@
+// Binary weights x real-valued activations on the tensor cores, with the activations split
+// ONCE per call into bf16 terms (instead of once per tile of units):
+//
+//   1. x_split_kernel writes x = x_hi + x_lo (+ x_lo2) as bf16 planes into a scratch "image"
+//      that is stored in exactly the order the MMA reads shared memory (a memory-bound pass:
+//      every fp32 input is read once);
+//   2. signw_img_kernel runs the GEMM: a pipeline stage of activations is ONE bulk asynchronous
+//      copy of the image (no tensor map, no multicast), the packed +-1 weights are widened to
+//      bf16 on chip, one MMA per term accumulates in fp32 in tensor memory.
+//
+// Frames are on the M side (TMEM lane = frame), units on the N side.  A CTA tile is 128 frames
+// x 512 units (two 256-column accumulators fed by the same activation stage).  The epilogue
+// thread owns a frame: per-unit affine (one fma), then Sign + pack (16 words per row and
+// tile) and/or fp32 stores of 128 contiguous bytes.
+//
+// |result - exact| <= 2^-17 * sum_k |x[m][k]| with 2 terms (products exact with 3), plus fp32
+// accumulation rounding.  The contraction index is permuted inside each group of 32 exactly
+// as in the other sign-weight kernel: word t of a K step holds k = t and k = t + 16.
+#include <cuda_bf16.h>
+
+#include "bnn_common.cuh"
+#include "tcgen05.cuh"
+
+namespace bnn {
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128;           // frames per tile
+constexpr int UN = 512;           // units per tile (2 x 256)
+constexpr int BK = 32;            // k per stage
+constexpr int A_PLANE = BM * BK * 2;        // 8 KB per bf16 term
+constexpr int B_BYTES = UN * BK * 2;        // 32 KB
+constexpr int MMA_WARP = 4, PROD_WARP0 = 5, PROD_WARPS = 8, EPI_WARPS = 4;
+constexpr int THREADS = (PROD_WARP0 + PROD_WARPS) * 32;
+constexpr uint32_t TMEM_COLS = 512;
+
+template <int NT> struct Cfg {
+    static constexpr int A_BYTES = NT * A_PLANE;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = NT == 2 ? 4 : 3;
+};
+
+struct Control {
+    float sc[UN], sh[UN];
+    uint64_t full[4], empty[4], acc_full, acc_empty;
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16_lo_as_float(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi_as_float(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// ---- split: one CTA per (frame tile, stage): 128 rows x 32 floats -> NT planes of 8 KB ------
+template <int NT>
+__global__ void __launch_bounds__(256)
+x_split_kernel(const float* __restrict__ X, int ldx, int M, int K, int nks, uint8_t* __restrict__ img) {
+    __shared__ float raw[BM][BK + 1];
+    const int mt = blockIdx.x / nks, ks = blockIdx.x % nks;
+    const int t = threadIdx.x;
+    // coalesced read: 8 consecutive threads fetch the 32 floats of one row segment
+    const bool vec = (ldx % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = (t >> 3) + 32 * i, m = mt * BM + row;
+        const int c4 = (t & 7) * 4, k = ks * BK + c4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (m < M) {
+            const float* src = X + (size_t)m * ldx + k;
+            if (vec && k + 3 < K) {
+                v = __ldg(reinterpret_cast<const float4*>(src));
+            } else {
+                if (k + 0 < K) v.x = __ldg(src + 0);
+                if (k + 1 < K) v.y = __ldg(src + 1);
+                if (k + 2 < K) v.z = __ldg(src + 2);
+                if (k + 3 < K) v.w = __ldg(src + 3);
+            }
+        }
+        raw[row][c4 + 0] = v.x; raw[row][c4 + 1] = v.y; raw[row][c4 + 2] = v.z; raw[row][c4 + 3] = v.w;
+    }
+    __syncthreads();
+    // coalesced write: consecutive threads write consecutive 16-byte chunks (consecutive rows)
+    uint8_t* blk = img + ((size_t)mt * nks + ks) * (NT * A_PLANE);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int chunk = t + 256 * i;          // 0..511 = (K step j, half-step cc, row)
+        const int row = chunk & (BM - 1), jc = chunk >> 7;   // jc = 2j + cc
+        uint32_t w[NT][4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {           // word e pairs k = 4jc + e with k + 16
+            float a = raw[row][4 * jc + e], b = raw[row][4 * jc + e + 16];
+#pragma unroll
+            for (int q = 0; q < NT; ++q) {
+                const uint32_t p = pack_bf16x2(a, b);
+                w[q][e] = p;
+                if (q + 1 < NT) { a -= bf16_lo_as_float(p); b -= bf16_hi_as_float(p); }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < NT; ++q)
+            *reinterpret_cast<uint4*>(blk + q * A_PLANE + (size_t)chunk * 16) = make_uint4(w[q][0], w[q][1], w[q][2], w[q][3]);
+    }
+}
+
+struct Args {
+    const uint8_t* img;
+    const uint32_t* Wp; int ldwp;
+    int M, N, K;
+    const float* scale; const float* shift;
+    int act, sign_mode;
+    float* Y; int ldy;
+    uint32_t* out_bits; int ldob;
+    int* status;
+};
+
+template <int NT>
+__global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
+    using C = Cfg<NT>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    Control* ctl = reinterpret_cast<Control*>(smem + C::STAGES * C::STAGE_BYTES);
+    volatile int* abort_flag = &ctl->abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int M = g.M, N = g.N;
+    const int nks = ceil_div(g.K, BK);
+    const int m_tiles = ceil_div(M, BM), n_tiles = ceil_div(N, UN);
+    const int tiles = m_tiles * n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), PROD_WARPS);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        mbar_init(smem_u32(&ctl->acc_full), 1);
+        mbar_init(smem_u32(&ctl->acc_empty), EPI_WARPS);
+        ctl->abort = 0;
+        mbar_init_fence();
+    }
+    if (warp == MMA_WARP) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ctl->tmem_base;
+
+    if (warp >= PROD_WARP0) {
+        // ---------------- producers: thread p widens packed weight rows p and p+256 of the unit
+        // tile; the first producer thread also starts the bulk copy of the activation stage.
+        const int p = threadIdx.x - PROD_WARP0 * 32;  // 0..255
+        const int my_tiles = (tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
+        const int total = my_tiles * nks;
+        // Packed rows are read 16 bytes (4 stages) at a time, one group ahead of use.  Bits at
+        // positions >= K may hold anything: the activation image is zero there.
+        const int ngroups = ceil_div(nks, 4);
+        int pf_g = 0, pf_tile = blockIdx.x, pf_left = my_tiles;
+        auto fetch = [&](uint4 (&o)[2]) {
+            o[0] = make_uint4(0u, 0u, 0u, 0u);
+            o[1] = o[0];
+            if (pf_left == 0) return;
+            const int n0 = (pf_tile / m_tiles) * UN;
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const int n = n0 + p + 256 * q;
+                if (n < N) o[q] = __ldg(reinterpret_cast<const uint4*>(g.Wp + (size_t)n * g.ldwp) + pf_g);
+            }
+            if (++pf_g == ngroups) { pf_g = 0; pf_tile += gridDim.x; --pf_left; }
+        };
+        uint4 grp[2], nxt[2];
+        fetch(grp);
+        fetch(nxt);
+        int ks = 0, tile = blockIdx.x, s = 0;
+        uint32_t ph = 1;  // parity to wait for on `empty`: a fresh barrier passes parity 1
+        for (int it = 0; it < total; ++it) {
+            const int sub = ks & 3;
+            uint32_t cur[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q)
+                cur[q] = sub == 0 ? grp[q].x : sub == 1 ? grp[q].y : sub == 2 ? grp[q].z : grp[q].w;
+            if (!warp_wait(smem_u32(&ctl->empty[s]), ph, abort_flag, lane)) break;
+            const uint32_t st = smem_u32(smem) + s * C::STAGE_BYTES;
+            if (p == 0) {
+                const int mt = tile % m_tiles;
+                mbar_expect_tx(smem_u32(&ctl->full[s]), C::A_BYTES);
+                bulk_g2s(st, g.img + ((size_t)mt * nks + ks) * C::A_BYTES, C::A_BYTES, smem_u32(&ctl->full[s]));
+            }
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const uint32_t nw = ~cur[q];
+                uint32_t wv[16];
+#pragma unroll
+                for (int t = 0; t < 16; ++t) wv[t] = ((nw << (15 - t)) & 0x80008000u) | 0x3F803F80u;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    sts128(st + C::A_BYTES + (c * UN + p + 256 * q) * 16, wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
+            if (++s == C::STAGES) { s = 0; ph ^= 1u; }
+            ++ks;
+            if ((ks & 3) == 0 || ks == nks) {   // group used up: take the prefetched one
+                grp[0] = nxt[0]; grp[1] = nxt[1];
+                fetch(nxt);
+            }
+            if (ks == nks) { ks = 0; tile += gridDim.x; }
+        }
+    } else if (warp == MMA_WARP) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc(kAccF32, kFmtBF16, kFmtBF16, BM, 256);
+            int it = 0, tl = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
+                ok = mbar_wait(smem_u32(&ctl->acc_empty), (uint32_t)((tl & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int ks = 0; ks < nks; ++ks, ++it) {
+                    const int s = it % C::STAGES;
+                    ok = mbar_wait(smem_u32(&ctl->full[s]), (uint32_t)((it / C::STAGES) & 1), abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t a0 = smem_u32(smem + s * C::STAGE_BYTES);
+                    const uint32_t b0 = a0 + C::A_BYTES;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+#pragma unroll
+                        for (int sub = 0; sub < 2; ++sub) {
+                            // rows [256 sub, 256 sub + 256) of the unit tile
+                            const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (UN * 16) + sub * 256 * 16, UN * 16, 128);
+#pragma unroll
+                            for (int q = 0; q < NT; ++q) {
+                                const uint64_t da = smem_desc_kmajor(a0 + q * A_PLANE + 2 * j * (BM * 16), BM * 16, 128);
+                                mma_f16(tmem + sub * 256, da, db, idesc, (ks | j | q) != 0);
+                            }
+                        }
+                    }
+                    mma_commit(smem_u32(&ctl->empty[s]));
+                }
+                if (ok) mma_commit(smem_u32(&ctl->acc_full));
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue: thread = one frame (TMEM lane), columns = units
+        const int row_in_tile = warp * 32 + lane;
+        const bool pack = g.act == BNN_ACT_SIGN_PACK;
+        const bool vy = g.Y && (g.ldy % 4 == 0) && ((reinterpret_cast<uintptr_t>(g.Y) & 15) == 0);
+        const int nw = words_for(N);
+        int tl = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
+            const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * UN;
+            const int m = m0 + row_in_tile;
+            epi_bar_sync();   // previous tile's readers of sc/sh are done
+#pragma unroll
+            for (int hh = 0; hh < UN / 128; ++hh) {
+                const int nl = row_in_tile + hh * 128, n = n0 + nl;
+                ctl->sc[nl] = (g.scale && n < N) ? g.scale[n] : 1.0f;
+                ctl->sh[nl] = (g.shift && n < N) ? g.shift[n] : 0.0f;
+            }
+            epi_bar_sync();
+            ok = epi_all(warp_wait(smem_u32(&ctl->acc_full), (uint32_t)(tl & 1), abort_flag, lane));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+            for (int q4 = 0; q4 < UN / 128; ++q4) {           // 4 groups of 32 columns = one 16-byte store of bits
+                if (n0 + q4 * 128 >= N) break;                // uniform over the CTA
+                uint32_t words[4];
+#pragma unroll
+                for (int gq = 0; gq < 4; ++gq) {
+                    const int gi = q4 * 4 + gq;
+                    uint32_t acc[32];
+                    tmem_ld32(taddr + gi * 32, acc);
+                    tmem_ld_wait();
+                    const int nb = n0 + gi * 32;
+                    float y[32];
+                    uint32_t wd = 0u;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float v = fmaf(ctl->sc[gi * 32 + j], __uint_as_float(acc[j]), ctl->sh[gi * 32 + j]);
+                        if (g.act == BNN_ACT_HARDTANH) v = fminf(fmaxf(v, -1.0f), 1.0f);
+                        y[j] = v;
+                        wd |= (uint32_t)(nb + j < N && sign_is_pos(v, g.sign_mode)) << j;
+                    }
+                    words[gq] = wd;
+                    if (g.Y && m < M && nb < N) {
+                        float* dst = g.Y + (size_t)m * g.ldy + nb;
+                        if (vy && nb + 31 < N) {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                reinterpret_cast<float4*>(dst)[q] = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (nb + j < N) dst[j] = y[j];
+                        }
+                    }
+                }
+                if (pack && m < M) {
+                    const int w0 = (n0 >> 5) + q4 * 4;
+                    uint32_t* dst = g.out_bits + (size_t)m * g.ldob + w0;
+                    if (w0 + 4 <= nw) {
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(words[0], words[1], words[2], words[3]);
+                    } else {
+#pragma unroll
+                        for (int gq = 0; gq < 4; ++gq)
+                            if (w0 + gq < nw) dst[gq] = words[gq];
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty));
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == MMA_WARP) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
+    if (threadIdx.x == 0 && ctl->abort) atomicExch(g.status, 1);
+}
+
+template <int NT>
+int launch_nt(const RealGemmArgs& r, void* workspace, cudaStream_t st) {
+    using C = Cfg<NT>;
+    constexpr int SMEM = C::STAGES * C::STAGE_BYTES + (int)sizeof(Control) + 128;
+    static bool configured = false;
+    static int sms = 0;
+    if (!configured) {
+        int dev = 0;
+        if (cudaFuncSetAttribute(signw_img_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess ||
+            cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return BNN_ERR_CUDA;
+        configured = true;
+    }
+    const int nks = ceil_div(r.K, BK), mt = ceil_div(r.M, BM);
+    uint8_t* img = static_cast<uint8_t*>(workspace);
+    x_split_kernel<NT><<<mt * nks, 256, 0, st>>>(r.Af, r.lda, r.M, r.K, nks, img);
+    Args a{img, r.Bb, r.ldb, r.M, r.N, r.K, r.scale, r.shift, r.act, r.sign_mode, r.Y, r.ldy, r.out_bits, r.ldob,
+           tc_status_ptr()};
+    if (!a.status) return BNN_ERR_CUDA;
+    const int tiles = mt * ceil_div(r.N, UN);
+    signw_img_kernel<NT><<<tiles < sms ? tiles : sms, THREADS, SMEM, st>>>(a);
+    return launch_status();
+}
+
+}  // namespace
+
+size_t signw_image_bytes(int M, int K, int terms) {
+    return (size_t)ceil_div(M, BM) * ceil_div(K, BK) * (terms == 3 ? 3 : 2) * A_PLANE;
+}
+
+int launch_signw_img(const RealGemmArgs& r, int terms, void* workspace, cudaStream_t st) {
+    return terms == 3 ? launch_nt<3>(r, workspace, st) : launch_nt<2>(r, workspace, st);
+}
+
+}  // namespace bnn

@@ -106,6 +106,27 @@ def test_forward_ami_config_full_batch_sampled_frames(env):
     run_binary_net(env, cfg, cfg.frames, sample=sample)
 
 
+def test_forward_minimal_workspace_gives_same_bits(env):
+    """With only the minimal scratch the first layer runs without the split-activation image:
+    both ways must agree with each other on every hidden bit that is not inside the float
+    tolerance band, and with the oracle (checked by run_binary_net for the full scratch)."""
+    torch, B, model = env
+    cfg = wl.CONFIGS["tiny"]
+    dn = model.DeviceNet(wl.make_model(cfg))
+    frames = 200
+    X = model.to_dev(wl.make_frames(cfg, frames))
+    full = dn.forward(X).clone()
+    small = torch.empty(dn.desc.min_workspace_bytes(frames), dtype=torch.uint8, device="cuda:0")
+    assert small.numel() < dn.desc.workspace_bytes(frames)
+    logp = torch.empty_like(full)
+    B.bnn_forward(dn.desc, X, logp, small)
+    # a first-layer bit inside the tolerance band may differ between the two float paths and
+    # change a frame's log-probs; require that nearly all frames agree closely
+    close = ((logp - full).abs().amax(dim=1) <= 1e-4).float().mean().item()
+    assert close > 0.9, close
+    assert B.bnn_device_status() == 0
+
+
 def test_forward_unwritten_workspace_path_equals_layer_out_path(env):
     """Without layer_out the activations go through the workspace: same log-probabilities."""
     torch, B, model = env

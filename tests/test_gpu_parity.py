@@ -38,13 +38,22 @@ def xnor_path(request, B):
     assert B.bnn_device_status() == 0, "a tensor-core kernel gave up on a bounded wait"
 
 
-@pytest.fixture(params=["fp32", "tensor"])
+@pytest.fixture(params=["fp32", "tensor", "tensor_ws"])
 def real_path(request, B):
-    """Runs a test once per real-valued GEMM kernel (FP32 pipe, tcgen05 with split operands)."""
+    """Runs a test once per real-valued GEMM kernel: FP32 pipe, tcgen05 with operands split on
+    the fly, tcgen05 with the activations split once into scratch (tensor_ws)."""
     prev = B.bnn_set_option(B.OPT_REAL_PATH, B.PATH_CUDA_CORE if request.param == "fp32" else B.PATH_TENSOR)
     yield request.param
     B.bnn_set_option(B.OPT_REAL_PATH, prev)
     assert B.bnn_device_status() == 0, "a tensor-core kernel gave up on a bounded wait"
+
+
+def signw_ws(B, path, m, k):
+    """Scratch for bnn_signw_gemm_ws when the test runs the split-once path, else None."""
+    if path != "tensor_ws":
+        return None
+    import torch
+    return torch.empty(B.bnn_signw_workspace_bytes(m, k) + 256, dtype=torch.uint8, device="cuda:0")
 
 
 def dev(a):
@@ -203,7 +212,7 @@ def test_xnor_gemm_fused_sign_pack_bit_exact(B, torch_, xnor_path, shape, mode, 
 
 # ------------------------------------------------------------------ +-1 weights x real input
 @pytest.mark.parametrize("shape", [(1, 1, 1), (3, 5, 33), (130, 129, 440), (257, 300, 600), (64, 256, 2048),
-                                   (20000, 260, 70)])
+                                   (20000, 260, 70), (300, 1300, 100)])
 def test_signw_gemm_within_tolerance(B, torch_, real_path, shape):
     m, n, k = shape
     rng = np.random.default_rng(m * n + k)
@@ -211,7 +220,7 @@ def test_signw_gemm_within_tolerance(B, torch_, real_path, shape):
     w = rng.standard_normal((n, k)).astype(np.float32)
     wp = o.sign_pack(w, 0, B.packed_pitch(k))
     y = torch_.full((m, n + 3), 123.0, dtype=torch_.float32, device="cuda:0")
-    B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y[:, :n])
+    B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y[:, :n], workspace=signw_ws(B, real_path, m, k))
     got = y.cpu().numpy()
     ref, sumabs = o.signw_gemm(x, wp, k)
     err = np.abs(got[:, :n] - ref)
@@ -231,7 +240,7 @@ def test_signw_gemm_sign_pack_epilogue(B, torch_, real_path, mode):
     out = packed_canary(torch_, m, n, B)
     y = torch_.empty((m, n), dtype=torch_.float32, device="cuda:0")
     B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y, act=B.ACT_SIGN_PACK, scale=dev(scale), shift=dev(shift),
-                     out_bits=out[:, :B.packed_pitch(n)], sign_mode=mode)
+                     out_bits=out[:, :B.packed_pitch(n)], sign_mode=mode, workspace=signw_ws(B, real_path, m, k))
     ref, sumabs = o.signw_gemm(x, wp, k)
     yh, _, bits = o.affine_act_f64(ref, scale, shift, o.ACT_SIGN, mode)
     tol = FLOAT_TOL * np.abs(scale)[None, :] * sumabs[:, None]
@@ -259,7 +268,8 @@ def test_signw_gemm_exact_zero_follows_sign_mode(B, torch_, real_path):
     assert (ref == 0).any()
     for mode in (0, 1):
         out = packed_canary(torch_, m, n, B)
-        B.bnn_signw_gemm(dev(x), dev(wp), k, act=B.ACT_SIGN_PACK, out_bits=out[:, :4], sign_mode=mode)
+        B.bnn_signw_gemm(dev(x), dev(wp), k, act=B.ACT_SIGN_PACK, out_bits=out[:, :4], sign_mode=mode,
+                         workspace=signw_ws(B, real_path, m, k))
         _, _, bits = o.affine_act_f64(ref, None, None, o.ACT_SIGN, mode)
         np.testing.assert_array_equal(out.cpu().numpy().view(np.uint32)[:, :2], bits)
 
@@ -271,7 +281,7 @@ def test_signw_gemm_hardtanh_epilogue(B, torch_, real_path):
     wp = wl.make_bit_planes(n, k, 0.5, 23, B.packed_pitch(k))
     scale = np.full(n, 0.05, np.float32)
     y = torch_.empty((m, n), dtype=torch_.float32, device="cuda:0")
-    B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y, act=B.ACT_HARDTANH, scale=dev(scale))
+    B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y, act=B.ACT_HARDTANH, scale=dev(scale), workspace=signw_ws(B, real_path, m, k))
     ref, sumabs = o.signw_gemm(x, wp, k)
     _, h, _ = o.affine_act_f64(ref, scale, None, o.ACT_HARDTANH)
     got = y.cpu().numpy()
@@ -288,7 +298,7 @@ def test_output_layer_bits_logp(B, torch_, real_path, c, m, h):
     wout = rng.normal(0, 1 / np.sqrt(h), (c, h)).astype(np.float32)
     b = rng.normal(0, 0.1, c).astype(np.float32)
     prep = None
-    if real_path == "tensor":
+    if real_path != "fp32":
         prep = torch_.empty(B.bnn_output_prepared_bytes(c, h), dtype=torch_.uint8, device="cuda:0")
         B.bnn_output_prepare(dev(wout), prep)
     z = torch_.full((m, c + 1), 9.0, dtype=torch_.float32, device="cuda:0")
@@ -334,8 +344,9 @@ def test_output_layer_wide_dynamic_range_weights(B, torch_):
     assert B.bnn_device_status() == 0
 
 
+@pytest.mark.parametrize("with_ws", [False, True])
 @pytest.mark.parametrize("terms", [2, 3])
-def test_signw_gemm_tensor_error_bound_by_terms(B, torch_, terms):
+def test_signw_gemm_tensor_error_bound_by_terms(B, torch_, terms, with_ws):
     """2 bf16 terms: |err| <= 2^-16 sum|x|; 3 terms: products exact, only fp32 accumulation."""
     m, n, k = 300, 256, 440
     rng = np.random.default_rng(13)
@@ -345,7 +356,7 @@ def test_signw_gemm_tensor_error_bound_by_terms(B, torch_, terms):
     prev_t = B.bnn_set_option(B.OPT_SIGNW_TERMS, terms)
     try:
         y = torch_.empty((m, n), dtype=torch_.float32, device="cuda:0")
-        B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y)
+        B.bnn_signw_gemm(dev(x), dev(wp), k, Y=y, workspace=signw_ws(B, "tensor_ws" if with_ws else "tensor", m, k))
         ref, sumabs = o.signw_gemm(x, wp, k)
         err = np.abs(y.cpu().numpy() - ref) / sumabs[:, None]
         assert err.max() <= (2.0 ** -16 if terms == 2 else 2.0 ** -21), err.max()

@@ -46,7 +46,7 @@ def test_static_forward_rejects_batches_beyond_its_array(env):
     cfg = wl.CONFIGS["tiny"]
     dn = model.DeviceNet(wl.make_model(cfg))
     frames = 40000   # 40000 x 128 B x 2 buffers > 8 MiB
-    assert dn.desc.workspace_bytes(frames) > B.STATIC_WORKSPACE_BYTES
+    assert dn.desc.min_workspace_bytes(frames) > B.STATIC_WORKSPACE_BYTES
     X = torch.zeros((frames, cfg.in_dim), dtype=torch.float32, device="cuda:0")
     out = torch.zeros((frames, cfg.classes), dtype=torch.float32, device="cuda:0")
     with pytest.raises(B.BnnError) as e:
