@@ -20,9 +20,15 @@
 // straight into tensor memory (tcgen05.st, lane = frame) and the MMA reads A from there.
 // TMEM budget (512 columns): two 192-column accumulators, so that the epilogue of tile i
 // overlaps the MMAs of tile i+1, plus 4 stages x 32 columns of A.
+// The packed rows themselves reach the SM by TMA: one 2-D tile load per operand brings the
+// next four stages (64 bytes per row) of all rows of the tile into a small staging ring
+// (64-byte swizzle, no multicast); each producer thread then reads its own row, 16 bytes per
+// stage, free of bank conflicts.  No thread waits on a global load.
 // The row popcounts the identity needs cost nothing extra: each producer thread sees every
 // word of its row anyway, sums their popcounts and hands the total to the epilogue through a
 // small ring in shared memory.
+#include <cuda.h>
+
 #include "bnn_common.cuh"
 #include "tcgen05.cuh"
 
@@ -40,10 +46,12 @@ constexpr int STAGES = 4;
 constexpr int B_BYTES = BN * BK, STAGE_BYTES = B_BYTES;  // only the unit operand lives in shared memory
 constexpr int EPI_WARPS = 4, MMA_WARP = 4, PROD_WARP0 = 5, A_WARPS = 4, B_WARPS = BN / 32;
 constexpr int PROD_WARPS = A_WARPS + B_WARPS;
-constexpr int THREADS = (PROD_WARP0 + PROD_WARPS) * 32;  // 480
+constexpr int TMA_WARP = PROD_WARP0 + PROD_WARPS;        // one more warp issues the tile loads
+constexpr int THREADS = (TMA_WARP + 1) * 32;             // 512
+constexpr int QUADS = 3;                                 // staging ring: 3 groups of 4 stages
+constexpr int QA_BYTES = BM * 64, QB_BYTES = BN * 64, QUAD_BYTES = QA_BYTES + QB_BYTES;
 constexpr uint32_t TMEM_A_COL = 2 * BN;                  // A stages start after the two accumulators
 constexpr uint32_t A_COLS = BK / 4;                      // 32-bit columns per A stage
-constexpr int PREFETCH = 3;                              // packed words in flight per producer
 constexpr uint32_t TMEM_COLS = 512;
 
 // Producers may run up to STAGES tiles ahead of the MMA warp (when a tile is a single stage)
@@ -55,10 +63,11 @@ struct Control {
     uint32_t flipw[BN / 32];
     int popc[RING][BM + BN];  // per tile: popcount of each frame row, then of each unit row
     uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], popc_ready[RING];
+    uint64_t quad_full[QUADS], quad_empty[QUADS];
     uint32_t tmem_base;
     int abort;
 };
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + (int)sizeof(Control) + 128;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + QUADS * QUAD_BYTES + (int)sizeof(Control) + 1024;
 
 
 
@@ -73,56 +82,54 @@ struct ProducerArgs {
     int lane;
 };
 
+__device__ __forceinline__ uint4 lds128u(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// 2-D tiled TMA load (no multicast): box at element coordinates (x = word, y = row).
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
 // Producer loop of one thread: row `r` of every tile of this CTA, stage by stage.  IS_A picks
-// the operand (frames / units): tile height, byte weights 2^t / 2^(7-t) and the slot in the
-// popcount ring are compile-time, so a stage is ~80 instructions.
+// the operand (frames / units): byte weights 2^t / 2^(7-t), destination (tensor memory /
+// shared memory) and the slot in the popcount ring are compile-time.
 template <bool IS_A>
-__device__ __forceinline__ void produce(const ProducerArgs& a, const uint32_t* __restrict__ base, int ld,
-                                        int rows, int r) {
+__device__ __forceinline__ void produce(const ProducerArgs& a, int r) {
     Control* ctl = a.ctl;
     const int my_tiles = (a.tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
     const int total = my_tiles * a.nks;
     const uint32_t dst0 = a.smem + r * 16;
     // TMEM lane of this thread's frame row: a warp may only touch lanes 32*(warp%4)..+31
     const uint32_t tdst0 = a.tmem + ((uint32_t)(r & ~31) << 16) + TMEM_A_COL;
-
-    // prefetch cursor: the divisions happen once per tile, not per stage
-    int pf_left = total, pf_ks = 0, pf_tile = blockIdx.x;
-    const uint4* pf_ptr = nullptr;
-    auto set_row = [&]() {
-        const int row = (IS_A ? (pf_tile % a.m_tiles) * BM : (pf_tile / a.m_tiles) * BN) + r;
-        pf_ptr = row < rows ? reinterpret_cast<const uint4*>(base + (size_t)row * ld) : nullptr;
-    };
-    set_row();
-    auto fetch = [&]() -> uint4 {
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (pf_left > 0) {
-            --pf_left;
-            if (pf_ptr) v = __ldg(pf_ptr + pf_ks);
-            if (++pf_ks == a.nks) {      // last stage of the row: clear the bits at positions >= K
-                const int last = a.kw - 1 - 4 * (a.nks - 1);
-                if (last == 0) { v.x &= a.tmask; v.y = 0u; v.z = 0u; v.w = 0u; }
-                else if (last == 1) { v.y &= a.tmask; v.z = 0u; v.w = 0u; }
-                else if (last == 2) { v.z &= a.tmask; v.w = 0u; }
-                else { v.w &= a.tmask; }
-                pf_ks = 0;
-                pf_tile += gridDim.x;
-                set_row();
-            }
-        }
-        return v;
-    };
-
-    uint4 ring[PREFETCH];
-#pragma unroll
-    for (int j = 0; j < PREFETCH; ++j) ring[j] = fetch();
+    // this row inside a staging slot: 64 bytes per row, 16-byte chunk c stored at c ^ ((r/2)%4)
+    const uint32_t stg0 = a.smem + STAGES * STAGE_BYTES + (IS_A ? 0 : QA_BYTES) + r * 64;
+    const uint32_t sw = (uint32_t)(r >> 1) & 3u;
+    const int last_word = a.kw - 1 - 4 * (a.nks - 1);   // index of the last valid word in the last stage
+    int qslot = 0;
+    uint32_t qph = 0;
     int pc = 0, ks = 0, slot = 0, s = 0;
     uint32_t ph = 1;  // parity to wait for on `empty`: a fresh barrier passes parity 1
     for (int it = 0; it < total; ++it) {
-        uint4 v = ring[0];
-#pragma unroll
-        for (int j = 0; j + 1 < PREFETCH; ++j) ring[j] = ring[j + 1];
-        ring[PREFETCH - 1] = fetch();
+        const int qi = ks & 3;   // stage inside its group of four
+        if (qi == 0 && !warp_wait(smem_u32(&ctl->quad_full[qslot]), qph, a.abort_flag, a.lane)) break;
+        uint4 v = lds128u(stg0 + qslot * QUAD_BYTES + (((uint32_t)qi ^ sw) << 4));
+        if (qi == 3 || ks == a.nks - 1) {   // group used up (values are in registers): release its slot
+            __syncwarp();
+            if (a.lane == 0) mbar_arrive(smem_u32(&ctl->quad_empty[qslot]));
+            if (++qslot == QUADS) { qslot = 0; qph ^= 1u; }
+        }
+        if (ks == a.nks - 1) {   // last stage of the row: clear the bits at positions >= K
+            if (last_word == 0) { v.x &= a.tmask; v.y = 0u; v.z = 0u; v.w = 0u; }
+            else if (last_word == 1) { v.y &= a.tmask; v.z = 0u; v.w = 0u; }
+            else if (last_word == 2) { v.z &= a.tmask; v.w = 0u; }
+            else { v.w &= a.tmask; }
+        }
         pc += __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w);
         if (!IS_A) {  // reverse the bits inside each byte, so that bit t carries weight 2^(7-t)
             v.x = __brev(__byte_perm(v.x, 0, 0x0123));
@@ -171,13 +178,13 @@ __device__ __forceinline__ void produce(const ProducerArgs& a, const uint32_t* _
 
 template <bool STORE_C, bool SIGN_PACK>
 __global__ void __launch_bounds__(THREADS, 1)
-xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __restrict__ Wp, int ldwp,
+xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                int M, int N, int K, int32_t* __restrict__ C, int ldc,
                const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
                uint32_t* __restrict__ out_bits, int ldob, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
-    Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES);
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES + QUADS * QUAD_BYTES);
     volatile int* abort_flag = &ctl->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -197,6 +204,10 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
             mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
         }
         for (int b = 0; b < RING; ++b) mbar_init(smem_u32(&ctl->popc_ready[b]), PROD_WARPS);
+        for (int b = 0; b < QUADS; ++b) {
+            mbar_init(smem_u32(&ctl->quad_full[b]), 1);            // the issuing thread (+ bytes)
+            mbar_init(smem_u32(&ctl->quad_empty[b]), PROD_WARPS);  // every producer warp has read it
+        }
         ctl->abort = 0;
         mbar_init_fence();
     }
@@ -212,8 +223,34 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
     if (warp >= PROD_WARP0) {
         // ---------------- producers: packed words -> widened byte tiles in shared memory
         ProducerArgs pa{smem_u32(smem), tmem, ctl, abort_flag, tiles, m_tiles, nks, kw, tmask, lane};
-        if (warp < PROD_WARP0 + A_WARPS) produce<true>(pa, Ap, ldap, M, (warp & 3) * 32 + lane);
-        else produce<false>(pa, Wp, ldwp, N, (warp - PROD_WARP0 - A_WARPS) * 32 + lane);
+        if (warp == TMA_WARP) {
+            // ---------------- one thread feeds the staging ring, a group of four stages at a time
+            if (lane == 0) {
+                const uint32_t stg = smem_u32(smem) + STAGES * STAGE_BYTES;
+                const int nq = ceil_div(nks, 4);
+                int qc = 0;
+                bool ok = true;
+                for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+                    const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+                    for (int gq = 0; gq < nq; ++gq, ++qc) {
+                        const int slot = qc % QUADS;
+                        if (qc >= QUADS) {
+                            ok = mbar_wait(smem_u32(&ctl->quad_empty[slot]), (uint32_t)(((qc / QUADS) - 1) & 1), abort_flag);
+                            if (!ok) break;
+                        }
+                        const uint32_t bar = smem_u32(&ctl->quad_full[slot]);
+                        mbar_arrive_expect_tx(bar, QUAD_BYTES);
+                        tma_load_2d(stg + slot * QUAD_BYTES, &mapA, gq * 16, m0, bar);
+                        tma_load_2d(stg + slot * QUAD_BYTES + QA_BYTES, &mapB, gq * 16, n0, bar);
+                    }
+                }
+            }
+            __syncwarp();
+        } else if (warp < PROD_WARP0 + A_WARPS) {
+            produce<true>(pa, (warp & 3) * 32 + lane);
+        } else {
+            produce<false>(pa, (warp - PROD_WARP0 - A_WARPS) * 32 + lane);
+        }
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issue: one thread
         if (lane == 0) {
@@ -365,6 +402,16 @@ xnor_tc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __rest
 
 int g_sm_count = 0;
 
+bool encode_packed_map(CUtensorMap* map, const uint32_t* base, int ld, int rows, int K, int box_rows) {
+    const cuuint64_t dims[2] = {(cuuint64_t)words_for(K), (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(uint32_t)};   // bytes between rows (multiple of 16)
+    const cuuint32_t box[2] = {16u, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return cuTensorMapEncodeTiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(base), dims, strides,
+                                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <bool STORE_C, bool SIGN_PACK>
 int launch_variant(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N, int K,
                    int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
@@ -386,7 +433,12 @@ int launch_variant(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, i
     const int grid = tiles < g_sm_count ? tiles : g_sm_count;
     int* status = tc_status_ptr();
     if (!status) return BNN_ERR_CUDA;
-    kern<<<grid, THREADS, SMEM_BYTES, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, status);
+    // tensor maps of the two packed operands: [rows][ceil(K/32) words] with the caller's pitch;
+    // boxes of 16 words x (128 | 192) rows; whatever lies outside the tensor reads as zero
+    CUtensorMap mapA, mapB;
+    if (!encode_packed_map(&mapA, Ap, ldap, M, K, BM) || !encode_packed_map(&mapB, Wp, ldwp, N, K, BN))
+        return BNN_ERR_CUDA;
+    kern<<<grid, THREADS, SMEM_BYTES, st>>>(mapA, mapB, M, N, K, C, ldc, thr, flip, out_bits, ldob, status);
     return launch_status();
 }
 
