@@ -13,6 +13,8 @@
 //     accumulator is exactly 128 * popc(a AND w) (u8 x u8 -> s32).
 //
 // One persistent CTA per SM, tile 128 frames x 192 units, 128 bits of K per pipeline stage.
+// Tiles are numbered with the unit index fastest, so that the CTAs running at the same time
+// share frame rows (L2 hits) and, with int32 output, fill whole output rows together.
 // Warp roles: warps 0-3 epilogue (TMEM -> thresholds -> packed bits / int32), warp 4 issues
 // the MMAs, warps 5-8 widen the frame rows and warps 9-14 the unit rows (one packed row per
 // thread and stage).  The kernel is bound by the shared-memory pipe, not by the tensor pipe,
@@ -64,6 +66,8 @@ struct Control {
     int popc[RING][BM + BN];  // per tile: popcount of each frame row, then of each unit row
     uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], popc_ready[RING];
     uint64_t quad_full[QUADS], quad_empty[QUADS];
+    // int32 output: per warp two staging blocks of 32 rows x 128 bytes (pitch 144: conflict-free 16-byte accesses)
+    __align__(16) int cstage[EPI_WARPS][2][32][36];
     uint32_t tmem_base;
     int abort;
 };
@@ -231,7 +235,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                 int qc = 0;
                 bool ok = true;
                 for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-                    const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+                    const int n0 = (tile % n_tiles) * BN, m0 = (tile / n_tiles) * BM;   // unit tiles vary fastest
                     for (int gq = 0; gq < nq; ++gq, ++qc) {
                         const int slot = qc % QUADS;
                         if (qc >= QUADS) {
@@ -288,7 +292,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         int tl = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
-            const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+            const int n0 = (tile % n_tiles) * BN, m0 = (tile / n_tiles) * BM;   // unit tiles vary fastest
             const int m = m0 + row_in_tile;
             // row popcounts of this tile, published by the producers
             ok = epi_all(warp_wait(smem_u32(&ctl->popc_ready[tl % RING]), (uint32_t)((tl / RING) & 1), abort_flag, lane));
@@ -331,18 +335,34 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                     int d[32];
 #pragma unroll
                     for (int j = 0; j < 32; ++j) d[j] = (int)(acc[j] >> 5) - 2 * pa - ctl->T[g * 32 + j];
-                    if (m < M) {
-                        int32_t* dst = C + (size_t)m * ldc + nb;
-                        const bool vec = (ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && nb + 31 < N;
-                        if (vec) {
+                    // Each thread parks its 32 integers (128 bytes of one output row) in shared
+                    // memory; the warp then writes the 32 x 128-byte block with 16-byte stores in
+                    // which 8 consecutive lanes cover one row: every store instruction writes four
+                    // whole 128-byte lines.
+                    const bool vec_ok = (ldc % 4 == 0) && ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && nb + 31 < N;
+                    if (vec_ok) {
+                        int (*blk)[36] = ctl->cstage[warp][g & 1];
+                        const uint32_t row_smem = smem_u32(&blk[lane][0]);
 #pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                reinterpret_cast<int4*>(dst)[q] = make_int4(d[4 * q], d[4 * q + 1], d[4 * q + 2], d[4 * q + 3]);
-                        } else {
+                        for (int q = 0; q < 8; ++q)
+                            sts128(row_smem + 16 * q, (uint32_t)d[4 * q], (uint32_t)d[4 * q + 1], (uint32_t)d[4 * q + 2], (uint32_t)d[4 * q + 3]);
+                        __syncwarp();
+                        const int rr = lane >> 3, qq = lane & 7;
+                        const int mrow0 = m0 + warp * 32;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (nb + j < N) dst[j] = d[j];
+                        for (int i = 0; i < 8; ++i) {
+                            const int row = 4 * i + rr;
+                            const int4 v = *reinterpret_cast<const int4*>(&blk[row][4 * qq]);
+                            if (mrow0 + row < M)
+                                *reinterpret_cast<int4*>(C + (size_t)(mrow0 + row) * ldc + nb + 4 * qq) = v;
                         }
+                        // the buffer is written again two blocks later: by then every lane has passed
+                        // the __syncwarp of the next block, i.e. has finished reading this one
+                    } else if (m < M) {
+                        int32_t* dst = C + (size_t)m * ldc + nb;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < N) dst[j] = d[j];
                     }
                     if (SIGN_PACK) {
                         uint32_t wd = 0u;
