@@ -1,6 +1,7 @@
 // Shared device/host helpers of the sm_100a binarised-DNN forward library.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -54,6 +55,9 @@ constexpr int kMaxKTensor = 1 << 22;
 int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
                    int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
                    uint32_t* out_bits, int ldob, cudaStream_t st);
+// Tensor map of a packed operand [rows][ceil(K/32) words] of pitch `ld` words: boxes of 16 words x
+// box_rows rows, 64-byte swizzle, zero fill outside the tensor.  False when the encoder fails.
+bool encode_packed_map(CUtensorMap* map, const uint32_t* base, int ld, int rows, int K, int box_rows);
 // Reads (synchronously) the word that a tensor-core kernel sets when a bounded wait ran out.
 int read_tc_status(int* out);
 // Device address of that word, passed to every tensor-core kernel (nullptr on failure).

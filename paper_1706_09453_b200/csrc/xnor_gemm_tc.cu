@@ -422,16 +422,6 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 
 int g_sm_count = 0;
 
-bool encode_packed_map(CUtensorMap* map, const uint32_t* base, int ld, int rows, int K, int box_rows) {
-    const cuuint64_t dims[2] = {(cuuint64_t)words_for(K), (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(uint32_t)};   // bytes between rows (multiple of 16)
-    const cuuint32_t box[2] = {16u, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1u, 1u};
-    return cuTensorMapEncodeTiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(base), dims, strides,
-                                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
-                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <bool STORE_C, bool SIGN_PACK>
 int launch_variant(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N, int K,
                    int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
@@ -463,6 +453,30 @@ int launch_variant(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, i
 }
 
 }  // namespace
+
+// The driver's tensor-map encoder is looked up through the runtime, so that the library does not
+// link against the driver library (which only exists on machines with a GPU).
+bool encode_packed_map(CUtensorMap* map, const uint32_t* base, int ld, int rows, int K, int box_rows) {
+    using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess || !fn)
+            return false;
+        encode = reinterpret_cast<EncodeFn>(fn);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)words_for(K), (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(uint32_t)};   // bytes between rows (multiple of 16)
+    const cuuint32_t box[2] = {16u, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint32_t*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
                    int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
