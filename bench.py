@@ -175,10 +175,16 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
         xnor = cfg.act == 1 and l > 0
         work = 2.0 * frames * cfg.hidden * k
         if xnor and xnor_path == "tensor":
-            # u8 x u8 tensor-core MACs: 2 x the measured bf16 rate (nominal ratio), sustained
-            # figure because the kernel is timed inside a long step; 1 bit-MAC = 2 bop
+            # 4-bit (e2m1, kind::mxf4) tensor-core MACs: 4 x the measured bf16 rate (nominal ratio
+            # 9 : 2.25 PFLOP/s), sustained figure because the kernel is timed inside a long step;
+            # 1 bit-MAC = 2 bop.  smem_bytes: what the kernel moves through the SM's shared
+            # memory per launch (4 bits stored + 4 bits read by the tensor core per operand bit
+            # and tile visit, plus the packed bits staged by TMA and read back once).
+            tiles_m, tiles_n = -(-frames // 128), -(-cfg.hidden // 192)
+            kpad = -(-k // 256) * 256
+            smem_bytes = tiles_m * tiles_n * (128 + 192) * kpad * (0.5 + 0.5 + 0.125 + 0.125)
             rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_tc_kernel", work=work, unit="Tbop/s",
-                             bound="tensor", peak=2.0 * peaks["bf16_tflops_sustained"]))
+                             bound="tensor", peak=4.0 * peaks["bf16_tflops_sustained"], smem_bytes=smem_bytes))
         elif xnor:
             rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_popc_kernel", work=work, unit="Tbop/s",
                              bound="alu", peak=popc_peak))
@@ -332,6 +338,9 @@ def run_ours(args):
         r["achieved"] = r["work"] / (t * 1e-3) / r.get("scale", 1e12)
         r["frac"] = r["achieved"] / r["peak"]
         r["pipe_util"] = r["frac"] * r.get("passes", 1)
+        if "smem_bytes" in r:
+            # fraction of the SMs' shared-memory bandwidth (128 B per clock and SM at the maximum clock)
+            r["smem_pipe_util"] = r["smem_bytes"] / (r["ms"] * 1e-3) / (SMS * 128 * peaks["sm_max_mhz"] * 1e6)
     # dominant KERNEL: group the layers by the kernel that runs them (the five binary hidden
     # layers are five launches of one kernel) and take the largest share of the step
     groups = {}
@@ -344,7 +353,7 @@ def run_ours(args):
     roofline = {"kernel": dk, "launches_per_step": dg["n"], "bound": dom["bound"],
                 "achieved": achieved, "peak": dom["peak"], "unit": dom["unit"],
                 "frac": achieved / dom["peak"], "traffic": ncu_traffic(dk),
-                "peak_source": ("2 x bf16_tflops_sustained of MEASURED_PEAKS.json (%s): u8 MMA = 2 x bf16 (nominal ratio), "
+                "peak_source": ("4 x bf16_tflops_sustained of MEASURED_PEAKS.json (%s): e2m1 (mxf4) MMA = 4 x bf16 (nominal ratio), "
                                 "sustained figure because the kernel is timed inside a long step; of measured"
                                 % peaks["source"]) if dk == "xnor_tc_kernel" else
                                ("bf16_tflops_sustained of MEASURED_PEAKS.json (%s); of measured" % peaks["source"])
@@ -371,7 +380,7 @@ def run_ours(args):
         "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "%s (hidden layers) + %s (first and top layer)"
-                 % ("u8 tensor-core MMA, s32 accumulate" if args.xnor_path == "tensor" else "int32 popcount",
+                 % ("e2m1 (mxf4) tensor-core MMA, f32 accumulate, exact" if args.xnor_path == "tensor" else "int32 popcount",
                     "split bf16/fp16 tensor-core MMA, f32 accumulate" if args.real_path == "tensor" else "f32"),
         "device_status": B.bnn_device_status(), "data": "synthetic",
         "config": {"workload": workload_name(cfg, frames), "frames_per_gpu": frames,
@@ -387,7 +396,7 @@ def run_ours(args):
         "paths": {"xnor": args.xnor_path, "real": args.real_path},
         "roofline": roofline,
         "forward_roofline": forward_roofline,
-        "layers": [{k: r[k] for k in ("name", "kernel", "bound", "ms", "achieved", "peak", "unit", "frac", "pipe_util")}
+        "layers": [{k: r[k] for k in ("name", "kernel", "bound", "ms", "achieved", "peak", "unit", "frac", "pipe_util", "smem_pipe_util") if k in r}
                    for r in rows],
         "xnor_tbops": (xnor_work / (xnor_ms * 1e-3) / 1e12) if xnor_ms else None,
         "hbm": {"algorithmic_bytes_per_step": hbm, "achieved_gbs": hbm / (total_ms / K * 1e-3) / 1e9,
@@ -469,8 +478,8 @@ def run_sweep(args):
                             reps = 2
                         ms = timeit(call, reps)
                         rec[name] = {"ms": ms, "tbops": bops / ms / 1e9, "gbs": nbytes / ms / 1e6}
-                    t_roof = max(nbytes / (peaks["hbm_gbs"] * 1e9), bops / (2 * peaks["bf16_tflops"] * 1e12))
-                    rec["bound"] = "hbm" if nbytes / (peaks["hbm_gbs"] * 1e9) > bops / (2 * peaks["bf16_tflops"] * 1e12) else "tensor"
+                    t_roof = max(nbytes / (peaks["hbm_gbs"] * 1e9), bops / (4 * peaks["bf16_tflops"] * 1e12))
+                    rec["bound"] = "hbm" if nbytes / (peaks["hbm_gbs"] * 1e9) > bops / (4 * peaks["bf16_tflops"] * 1e12) else "tensor"
                     rec["roofline_frac_tensor_kernel"] = t_roof / (rec["tensor"]["ms"] * 1e-3)
                     # parity on sampled rows (first, last, two in between)
                     B.bnn_set_xnor_path(B.XNOR_TENSOR)

@@ -210,6 +210,44 @@ def test_xnor_gemm_fused_sign_pack_bit_exact(B, torch_, xnor_path, shape, mode, 
         assert (d[:, 2::5].astype(np.float32) + shift[2::5] == 0).any(), "no exact zero was exercised"
 
 
+@pytest.mark.parametrize("shape", [(8192, 2048, 2048), (16384, 2048, 2048)])
+def test_xnor_gemm_full_size_every_output_on_repeated_launches(B, torch_, shape):
+    """A hidden layer at full size, every output bit compared with the oracle, on many launches in
+    a row: a hand-off between the kernel's roles that is wrong once in ten thousand tiles only
+    shows on a run of this length (sampled outputs would miss it)."""
+    m, n, k = shape
+    prev = B.bnn_set_xnor_path(B.XNOR_TENSOR)
+    try:
+        rng = np.random.default_rng(m)
+        ap = wl.make_bit_planes(m, k, 0.5, [5, m, n, k], B.packed_pitch(k))
+        wp = wl.make_bit_planes(n, k, 0.5, [6, m, n, k], B.packed_pitch(k))
+        scale = np.ones(n, dtype=np.float32)
+        shift = np.round(rng.normal(0, 20, n)).astype(np.float32)   # thresholds where the dot products are dense
+        thr = torch_.empty(n, dtype=torch_.int32, device="cuda:0")
+        flip = torch_.empty((n + 31) // 32, dtype=torch_.int32, device="cuda:0")
+        B.bnn_fold_thresholds(dev(scale), dev(shift), n, k, thr, flip, 0)
+        d = o.xnor_gemm(ap, wp, k)
+        want_bits = torch_.from_numpy(o.affine_sign_pack_i32(d, scale, shift, 0).view(np.int32)).to("cuda:0")
+        want_c = torch_.from_numpy(d).to("cuda:0")
+        a_dev, w_dev = dev(ap), dev(wp)
+        out = torch_.zeros((m, B.packed_pitch(n)), dtype=torch_.int32, device="cuda:0")
+        c = torch_.zeros((m, n), dtype=torch_.int32, device="cuda:0")
+        nw = (n + 31) // 32
+        for launch in range(40):
+            out.zero_()
+            B.bnn_xnor_gemm(a_dev, w_dev, k, thr=thr, flip=flip, out_bits=out)
+            bad = int((out[:, :nw] != want_bits).sum().item())
+            assert bad == 0, "launch %d (fused Sign): %d packed words differ" % (launch, bad)
+        for launch in range(20):
+            c.zero_()
+            B.bnn_xnor_gemm(a_dev, w_dev, k, C_out=c)
+            bad = int((c != want_c).sum().item())
+            assert bad == 0, "launch %d (int32 output): %d outputs differ" % (launch, bad)
+    finally:
+        B.bnn_set_xnor_path(prev)
+    assert B.bnn_device_status() == 0, "a tensor-core kernel gave up on a bounded wait"
+
+
 # ------------------------------------------------------------------ +-1 weights x real input
 @pytest.mark.parametrize("shape", [(1, 1, 1), (3, 5, 33), (130, 129, 440), (257, 300, 600), (64, 256, 2048),
                                    (20000, 260, 70), (300, 1300, 100)])
