@@ -178,11 +178,12 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
             # 4-bit (e2m1, kind::mxf4) tensor-core MACs: 4 x the measured bf16 rate (nominal ratio
             # 9 : 2.25 PFLOP/s), sustained figure because the kernel is timed inside a long step;
             # 1 bit-MAC = 2 bop.  smem_bytes: what the kernel moves through the SM's shared
-            # memory per launch (4 bits stored + 4 bits read by the tensor core per operand bit
-            # and tile visit, plus the packed bits staged by TMA and read back once).
+            # memory per launch (per bit of the unit operand and tile visit 4 bits stored + 4 bits
+            # read by the tensor core; the packed bits of both operands staged by TMA and read
+            # back once; the widened frame operand goes to tensor memory instead).
             tiles_m, tiles_n = -(-frames // 128), -(-cfg.hidden // 192)
             kpad = -(-k // 256) * 256
-            smem_bytes = tiles_m * tiles_n * (128 + 192) * kpad * (0.5 + 0.5 + 0.125 + 0.125)
+            smem_bytes = tiles_m * tiles_n * kpad * (192 * (0.5 + 0.5 + 0.125 + 0.125) + 128 * (0.125 + 0.125))
             rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_tc_kernel", work=work, unit="Tbop/s",
                              bound="tensor", peak=4.0 * peaks["bf16_tflops_sustained"], smem_bytes=smem_bytes))
         elif xnor:

@@ -41,36 +41,35 @@ using namespace tc;
 constexpr int BM = 128, BN = 192;
 constexpr int BK = 256;                                   // bits of K per stage = nibbles per widened row
 constexpr int ROW_BYTES = BK / 2;                         // widened bytes per row and stage (128)
-constexpr int A_BYTES = BM * ROW_BYTES, B_BYTES = BN * ROW_BYTES, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int B_BYTES = BN * ROW_BYTES, STAGE_BYTES = B_BYTES;   // only the unit operand lives in shared memory
+constexpr int STAGES = 3;
 constexpr int EPI_WARPS = 4, MMA_WARP = 4, PROD_WARP0 = 5, A_WARPS = BM / 32, B_WARPS = BN / 32;
 constexpr int PROD_WARPS = A_WARPS + B_WARPS;
 constexpr int TMA_WARP = PROD_WARP0 + PROD_WARPS;
 constexpr int THREADS = (TMA_WARP + 1) * 32;              // 512
-constexpr int GROUPS = 3;                                 // staging ring: groups of two stages
+constexpr int GROUPS = 4;                                 // staging ring: groups of two stages
 constexpr int GA_BYTES = BM * 64, GB_BYTES = BN * 64, GROUP_BYTES = GA_BYTES + GB_BYTES;
-constexpr uint32_t TMEM_SF_COL = 2 * BN;                  // scale factors sit after the two accumulators
-constexpr uint32_t SF_COLS = 64;
+constexpr uint32_t TMEM_A_COL = 2 * BN;                   // A stages start after the two accumulators
+constexpr uint32_t A_COLS = ROW_BYTES / 4;                // 32-bit columns per A stage
+constexpr uint32_t TMEM_SF_COL = TMEM_A_COL + STAGES * A_COLS, SF_COLS = 32;   // block scales: 16 columns per operand
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int kMagicBits = 0x4B400000;                    // bits of 1.5 * 2^23: x + magic has the integer x in its low bits
 
-// With int32 output each epilogue warp needs two staging blocks of 32 rows x 128 bytes; that
-// variant runs with one pipeline stage less to make room for them.
+// With int32 output each epilogue warp needs two staging blocks of 32 rows x 128 bytes.
 template <bool STORE_C> struct Cfg {
-    static constexpr int STAGES = STORE_C ? 3 : 4;
     static constexpr int CSTAGE_BYTES = STORE_C ? EPI_WARPS * 2 * 32 * 36 * 4 : 0;
 };
-constexpr int MAX_STAGES = 4;
 
 struct Control {
     int T[BN];               // per unit: threshold + kMagicBits (Sign epilogue only)
     uint32_t flipw[BN / 32];
-    uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
+    uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
     uint64_t group_full[GROUPS], group_empty[GROUPS];
     uint32_t tmem_base;
     int abort;
 };
 template <bool STORE_C> constexpr int smem_bytes() {
-    return Cfg<STORE_C>::STAGES * STAGE_BYTES + GROUPS * GROUP_BYTES + (int)sizeof(Control) + Cfg<STORE_C>::CSTAGE_BYTES + 1024;
+    return STAGES * STAGE_BYTES + GROUPS * GROUP_BYTES + (int)sizeof(Control) + Cfg<STORE_C>::CSTAGE_BYTES + 1024;
 }
 static_assert(smem_bytes<false>() <= 232448 && smem_bytes<true>() <= 232448, "shared memory of one CTA");
 static_assert(TMEM_SF_COL + SF_COLS <= TMEM_COLS, "tensor memory columns");
@@ -78,6 +77,7 @@ static_assert(sizeof(Control) % 16 == 0, "the int32 staging blocks follow the co
 
 struct ProducerArgs {
     uint32_t smem;        // shared-space address of stage 0
+    uint32_t tmem;        // base of the tensor-memory allocation
     Control* ctl;
     volatile int* abort_flag;
     int tiles, nks, kw;
@@ -102,13 +102,14 @@ __device__ __forceinline__ uint4 widen_masked(uint32_t w, uint32_t valid) {
 
 // Producer loop of one thread: row `r` of every tile of this CTA, stage by stage.  IS_A picks
 // the operand (frames / units), i.e. where the row sits in a stage and in a staging group.
-template <bool IS_A, int STAGES>
+template <bool IS_A>
 __device__ __forceinline__ void produce(const ProducerArgs& a, int r) {
     Control* ctl = a.ctl;
-    constexpr int R = IS_A ? BM : BN;   // rows of the operand tile; 16-byte chunk c of row r sits at (c R + r) 16
     const int my_tiles = (a.tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
     const int total = my_tiles * a.nks;
-    const uint32_t dst0 = a.smem + (IS_A ? 0 : A_BYTES) + r * 16;
+    const uint32_t dst0 = a.smem + r * 16;
+    // TMEM lane of this thread's frame row: a warp may only touch lanes 32*(warp%4)..+31
+    const uint32_t tdst0 = a.tmem + ((uint32_t)(r & ~31) << 16) + TMEM_A_COL;
     // this row inside a staging group: 64 bytes per row, 16-byte chunk c stored at c ^ ((r/2)%4)
     const uint32_t stg0 = a.smem + STAGES * STAGE_BYTES + (IS_A ? 0 : GA_BYTES) + r * 64;
     const uint32_t sw = (uint32_t)(r >> 1) & 3u;
@@ -124,24 +125,34 @@ __device__ __forceinline__ void produce(const ProducerArgs& a, int r) {
         const uint4 v0 = lds128u(src + (((2u * gi) ^ sw) << 4));
         const uint4 v1 = lds128u(src + (((2u * gi + 1u) ^ sw) << 4));
         if (!warp_wait(smem_u32(&ctl->empty[s]), ph, a.abort_flag, a.lane)) break;
-        const uint32_t dst = dst0 + s * STAGE_BYTES;
         const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+        uint4 o[8];   // 16-byte chunk c of the widened row
         if (ragged && ks == a.nks - 1) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const int g = 8 * ks + c;   // index of the word in the row
                 const uint32_t valid = g < a.kw - 1 ? 0xFFFFFFFFu : (g == a.kw - 1 ? a.tmask : 0u);
-                const uint4 o = widen_masked(w[c], valid);
-                sts128(dst + c * (R * 16), o.x, o.y, o.z, o.w);
+                o[c] = widen_masked(w[c], valid);
             }
         } else {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint4 o = widen(w[c]);
-                sts128(dst + c * (R * 16), o.x, o.y, o.z, o.w);
-            }
+            for (int c = 0; c < 8; ++c) o[c] = widen(w[c]);
         }
-        fence_proxy_async_smem();
+        if (IS_A) {
+            // 32-bit column 4c + t of the stage = word t of chunk c: the byte order of the
+            // K-major shared-memory layout of the other operand
+            uint32_t wr[32];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) { wr[4 * c] = o[c].x; wr[4 * c + 1] = o[c].y; wr[4 * c + 2] = o[c].z; wr[4 * c + 3] = o[c].w; }
+            tmem_st32(tdst0 + s * A_COLS, wr);
+            tmem_st_wait();
+            tc_fence_before_sync();
+        } else {
+            const uint32_t dst = dst0 + s * STAGE_BYTES;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) sts128(dst + c * (BN * 16), o[c].x, o[c].y, o[c].z, o[c].w);
+            fence_proxy_async_smem();
+        }
         __syncwarp();
         if (a.lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
         // The staging slot is handed back only here, after the stores that consumed the loaded
@@ -163,7 +174,6 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                 int M, int N, int K, int32_t* __restrict__ C, int ldc,
                 const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
                 uint32_t* __restrict__ out_bits, int ldob, int* __restrict__ status) {
-    constexpr int STAGES = Cfg<STORE_C>::STAGES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES + GROUPS * GROUP_BYTES);
@@ -206,9 +216,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         uint32_t ones[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) ones[j] = 0x7F7F7F7Fu;
-        const uint32_t t0 = tmem + ((uint32_t)(warp * 32) << 16) + TMEM_SF_COL;
-        tmem_st32(t0, ones);
-        tmem_st32(t0 + 32, ones);
+        tmem_st32(tmem + ((uint32_t)(warp * 32) << 16) + TMEM_SF_COL, ones);
         tmem_st_wait();
     }
     tc_fence_before_sync();
@@ -216,7 +224,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     tc_fence_after_sync();
 
     if (warp >= PROD_WARP0) {
-        ProducerArgs pa{smem_u32(smem), ctl, abort_flag, tiles, nks, kw, tail_mask(K), lane};
+        ProducerArgs pa{smem_u32(smem), tmem, ctl, abort_flag, tiles, nks, kw, tail_mask(K), lane};
         if (warp == TMA_WARP) {
             // ---------------- one thread feeds the staging ring, a group of two stages at a time
             if (lane == 0) {
@@ -229,7 +237,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                     for (int g = 0; g < ng; ++g, ++gc) {
                         const int slot = gc % GROUPS;
                         if (gc >= GROUPS) {
-                            ok = mbar_wait(smem_u32(&ctl->group_empty[slot]), (uint32_t)(((gc / GROUPS) - 1) & 1), abort_flag);
+                            ok = mbar_wait_relaxed(smem_u32(&ctl->group_empty[slot]), (uint32_t)(((gc / GROUPS) - 1) & 1), abort_flag);
                             if (!ok) break;
                         }
                         const uint32_t bar = smem_u32(&ctl->group_full[slot]);
@@ -241,15 +249,15 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             }
             __syncwarp();
         } else if (warp < PROD_WARP0 + A_WARPS) {
-            produce<true, STAGES>(pa, (warp - PROD_WARP0) * 32 + lane);
+            produce<true>(pa, (warp & 3) * 32 + lane);
         } else {
-            produce<false, STAGES>(pa, (warp - PROD_WARP0 - A_WARPS) * 32 + lane);
+            produce<false>(pa, (warp - PROD_WARP0 - A_WARPS) * 32 + lane);
         }
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issue: one thread
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc_mxf4(BM, BN);
-            const uint32_t sfa = tmem + TMEM_SF_COL, sfb = tmem + TMEM_SF_COL + 32;
+            const uint32_t sfa = tmem + TMEM_SF_COL, sfb = tmem + TMEM_SF_COL + SF_COLS / 2;
             int it = 0;
             int tl = 0;
             bool ok = true;
@@ -264,12 +272,12 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                     ok = mbar_wait(smem_u32(&ctl->full[s]), (uint32_t)((it / STAGES) & 1), abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t a0 = smem_u32(smem + s * STAGE_BYTES), b0 = a0 + A_BYTES;
+                    const uint32_t b0 = smem_u32(smem + s * STAGE_BYTES);
+                    const uint32_t ta = tmem + TMEM_A_COL + s * A_COLS;
 #pragma unroll
-                    for (int j = 0; j < BK / 64; ++j) {   // 64 positions of K = 32 bytes = two 16-byte chunks per MMA
-                        const uint64_t da = smem_desc_kmajor(a0 + 2 * j * (BM * 16), BM * 16, 128);
+                    for (int j = 0; j < BK / 64; ++j) {   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
                         const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (BN * 16), BN * 16, 128);
-                        mma_mxf4(d, da, db, idesc, sfa, sfb, (ks | j) != 0);
+                        mma_mxf4_ts(d, ta + 8 * j, db, idesc, sfa, sfb, (ks | j) != 0);
                     }
                     mma_commit(smem_u32(&ctl->empty[s]));
                 }
@@ -301,7 +309,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             }
             const int b = tl & 1;
             // all four epilogue warps take the same decision, so none is left at a barrier
-            ok = epi_all(warp_wait(smem_u32(&ctl->acc_full[b]), (uint32_t)((tl >> 1) & 1), abort_flag, lane));
+            ok = epi_all(warp_wait_relaxed(smem_u32(&ctl->acc_full[b]), (uint32_t)((tl >> 1) & 1), abort_flag, lane));
             if (!ok) break;
             tc_fence_after_sync();
             const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * BN);
