@@ -238,14 +238,26 @@ log_softmax_rows_kernel(float* __restrict__ Z, int ldz, int M, int C) {
     }
 }
 
+// 2^x on the special-function unit (relative error ~2^-22; the arguments here are <= 0).
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 // Same result with the whole row held in registers (C <= 256*4*V, 16-byte aligned rows):
-// every logit is read from memory once and written once.
+// every logit is read from memory once and written once.  The maximum is reduced first (warp
+// shuffles, then 8 values through shared memory), so each element costs a subtract, a
+// multiply, one ex2 and one add; the sum is reduced the same way.
 template <int V>
 __global__ void __launch_bounds__(256)
 log_softmax_rows_reg_kernel(float* __restrict__ Z, int ldz, int M, int C) {
-    __shared__ float sm[8], ss[8];
+    __shared__ float sm[2][8], ss[2][8];
     const int c4 = C >> 2;  // C % 4 == 0
-    for (int row = blockIdx.x; row < M; row += gridDim.x) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+    int par = 0;   // the two halves of the scratch alternate, which saves a barrier per row
+    for (int row = blockIdx.x; row < M; row += gridDim.x, par ^= 1) {
         float4* z = reinterpret_cast<float4*>(Z + (size_t)row * ldz);
         float4 v[V];
         float mx = -FLT_MAX;
@@ -255,12 +267,29 @@ log_softmax_rows_reg_kernel(float* __restrict__ Z, int ldz, int M, int C) {
             v[i] = c < c4 ? z[c] : make_float4(-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX);
             mx = fmaxf(fmaxf(mx, fmaxf(v[i].x, v[i].y)), fmaxf(v[i].z, v[i].w));
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        if (lane == 0) sm[par][w] = mx;
+        __syncthreads();
+        mx = sm[par][0];
+#pragma unroll
+        for (int i = 1; i < 8; ++i) mx = fmaxf(mx, sm[par][i]);
+        // sum of exp(z - max) = sum of 2^((z - max) log2 e); the difference is taken first, so the
+        // rounding error scales with the distance from the maximum, not with the logit itself;
+        // padding (-FLT_MAX) contributes 0
         float s = 0.f;
 #pragma unroll
         for (int i = 0; i < V; ++i)
-            if (threadIdx.x + i * 256 < c4)
-                s += expf(v[i].x - mx) + expf(v[i].y - mx) + expf(v[i].z - mx) + expf(v[i].w - mx);
-        const float lse = block_logsumexp(mx, s, sm, ss);
+            s += (ex2_approx((v[i].x - mx) * kLog2e) + ex2_approx((v[i].y - mx) * kLog2e)) +
+                 (ex2_approx((v[i].z - mx) * kLog2e) + ex2_approx((v[i].w - mx) * kLog2e));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        if (lane == 0) ss[par][w] = s;
+        __syncthreads();
+        s = ss[par][0];
+#pragma unroll
+        for (int i = 1; i < 8; ++i) s += ss[par][i];
+        const float lse = mx + kLn2 * log2f(s);
 #pragma unroll
         for (int i = 0; i < V; ++i) {
             const int c = threadIdx.x + i * 256;
