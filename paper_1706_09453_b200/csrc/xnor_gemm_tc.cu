@@ -22,8 +22,9 @@
 // Roles in a CTA of 16 warps (persistent, one CTA per SM, tiles of 128 frames x 192 units):
 //   warp 15      one thread issues 2-D TMA tile loads of the packed rows (64 bytes per row =
 //                two stages) into a staging ring (64-byte swizzle, no multicast)
-//   warps 5-8    widen the frame rows: thread = one row, 32 bytes -> 128 bytes per stage
-//   warps 9-14   widen the unit rows the same way
+//   warps 5-8    widen the frame rows, thread = one row, 32 bytes -> 128 bytes per stage,
+//                written to tensor memory (the MMA reads its A operand from there)
+//   warps 9-14   widen the unit rows the same way into shared memory, two stages per iteration
 //   warp 4       one thread issues the MMAs (4 per stage, K = 64 each) and the commits
 //   warps 0-3    epilogue: accumulator -> Sign/threshold -> repacked bits (or int32 output);
 //                two accumulators in tensor memory, so it overlaps the next tile's MMAs
@@ -42,7 +43,7 @@ constexpr int BM = 128, BN = 192;
 constexpr int BK = 256;                                   // bits of K per stage = nibbles per widened row
 constexpr int ROW_BYTES = BK / 2;                         // widened bytes per row and stage (128)
 constexpr int B_BYTES = BN * ROW_BYTES, STAGE_BYTES = B_BYTES;   // only the unit operand lives in shared memory
-constexpr int STAGES = 3;
+constexpr int A_STAGES = 3, B_STAGES = 4;               // rings of the frame operand (tensor memory) and the unit operand
 constexpr int EPI_WARPS = 4, MMA_WARP = 4, PROD_WARP0 = 5, A_WARPS = BM / 32, B_WARPS = BN / 32;
 constexpr int PROD_WARPS = A_WARPS + B_WARPS;
 constexpr int TMA_WARP = PROD_WARP0 + PROD_WARPS;
@@ -51,7 +52,7 @@ constexpr int GROUPS = 4;                                 // staging ring: group
 constexpr int GA_BYTES = BM * 64, GB_BYTES = BN * 64, GROUP_BYTES = GA_BYTES + GB_BYTES;
 constexpr uint32_t TMEM_A_COL = 2 * BN;                   // A stages start after the two accumulators
 constexpr uint32_t A_COLS = ROW_BYTES / 4;                // 32-bit columns per A stage
-constexpr uint32_t TMEM_SF_COL = TMEM_A_COL + STAGES * A_COLS, SF_COLS = 32;   // block scales: 16 columns per operand
+constexpr uint32_t TMEM_SF_COL = TMEM_A_COL + A_STAGES * A_COLS, SF_COLS = 32;   // block scales: 16 columns per operand
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int kMagicBits = 0x4B400000;                    // bits of 1.5 * 2^23: x + magic has the integer x in its low bits
 
@@ -63,13 +64,13 @@ template <bool STORE_C> struct Cfg {
 struct Control {
     int T[BN];               // per unit: threshold + kMagicBits (Sign epilogue only)
     uint32_t flipw[BN / 32];
-    uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
+    uint64_t full_a[A_STAGES], empty_a[A_STAGES], full_b[B_STAGES], empty_b[B_STAGES], acc_full[2], acc_empty[2];
     uint64_t group_full[GROUPS], group_empty[GROUPS];
     uint32_t tmem_base;
     int abort;
 };
 template <bool STORE_C> constexpr int smem_bytes() {
-    return STAGES * STAGE_BYTES + GROUPS * GROUP_BYTES + (int)sizeof(Control) + Cfg<STORE_C>::CSTAGE_BYTES + 1024;
+    return B_STAGES * STAGE_BYTES + GROUPS * GROUP_BYTES + (int)sizeof(Control) + Cfg<STORE_C>::CSTAGE_BYTES + 1024;
 }
 static_assert(smem_bytes<false>() <= 232448 && smem_bytes<true>() <= 232448, "shared memory of one CTA");
 static_assert(TMEM_SF_COL + SF_COLS <= TMEM_COLS, "tensor memory columns");
@@ -100,18 +101,32 @@ __device__ __forceinline__ uint4 widen_masked(uint32_t w, uint32_t valid) {
     return o;
 }
 
-// Producer loop of one thread: row `r` of every tile of this CTA, stage by stage.  IS_A picks
-// the operand (frames / units), i.e. where the row sits in a stage and in a staging group.
-template <bool IS_A>
-__device__ __forceinline__ void produce(const ProducerArgs& a, int r) {
+// The eight 16-byte chunks of one widened row and stage; `ks` is the stage's index in the row.
+__device__ __forceinline__ void widen_stage(const ProducerArgs& a, bool ragged, int ks, const uint4& v0, const uint4& v1, uint4 (&o)[8]) {
+    const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+    if (ragged && ks == a.nks - 1) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int g = 8 * ks + c;   // index of the word in the row
+            const uint32_t valid = g < a.kw - 1 ? 0xFFFFFFFFu : (g == a.kw - 1 ? a.tmask : 0u);
+            o[c] = widen_masked(w[c], valid);
+        }
+    } else {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) o[c] = widen(w[c]);
+    }
+}
+
+// Producer of the frame operand: thread = row `r` of every tile of this CTA, one stage per
+// iteration, widened rows written to tensor memory (ring of A_STAGES stages).
+__device__ __forceinline__ void produce_a(const ProducerArgs& a, int r) {
     Control* ctl = a.ctl;
     const int my_tiles = (a.tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
     const int total = my_tiles * a.nks;
-    const uint32_t dst0 = a.smem + r * 16;
     // TMEM lane of this thread's frame row: a warp may only touch lanes 32*(warp%4)..+31
     const uint32_t tdst0 = a.tmem + ((uint32_t)(r & ~31) << 16) + TMEM_A_COL;
     // this row inside a staging group: 64 bytes per row, 16-byte chunk c stored at c ^ ((r/2)%4)
-    const uint32_t stg0 = a.smem + STAGES * STAGE_BYTES + (IS_A ? 0 : GA_BYTES) + r * 64;
+    const uint32_t stg0 = a.smem + B_STAGES * STAGE_BYTES + r * 64;
     const uint32_t sw = (uint32_t)(r >> 1) & 3u;
     const bool ragged = (a.kw % 8 != 0) || a.tmask != 0xFFFFFFFFu;   // last stage has positions >= K
     int gslot = 0;
@@ -124,37 +139,19 @@ __device__ __forceinline__ void produce(const ProducerArgs& a, int r) {
         const uint32_t src = stg0 + gslot * GROUP_BYTES;
         const uint4 v0 = lds128u(src + (((2u * gi) ^ sw) << 4));
         const uint4 v1 = lds128u(src + (((2u * gi + 1u) ^ sw) << 4));
-        if (!warp_wait(smem_u32(&ctl->empty[s]), ph, a.abort_flag, a.lane)) break;
-        const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-        uint4 o[8];   // 16-byte chunk c of the widened row
-        if (ragged && ks == a.nks - 1) {
+        if (!warp_wait(smem_u32(&ctl->empty_a[s]), ph, a.abort_flag, a.lane)) break;
+        uint4 o[8];
+        widen_stage(a, ragged, ks, v0, v1, o);
+        // 32-bit column 4c + t of the stage = word t of chunk c: the byte order of the
+        // K-major shared-memory layout of the other operand
+        uint32_t wr[32];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const int g = 8 * ks + c;   // index of the word in the row
-                const uint32_t valid = g < a.kw - 1 ? 0xFFFFFFFFu : (g == a.kw - 1 ? a.tmask : 0u);
-                o[c] = widen_masked(w[c], valid);
-            }
-        } else {
-#pragma unroll
-            for (int c = 0; c < 8; ++c) o[c] = widen(w[c]);
-        }
-        if (IS_A) {
-            // 32-bit column 4c + t of the stage = word t of chunk c: the byte order of the
-            // K-major shared-memory layout of the other operand
-            uint32_t wr[32];
-#pragma unroll
-            for (int c = 0; c < 8; ++c) { wr[4 * c] = o[c].x; wr[4 * c + 1] = o[c].y; wr[4 * c + 2] = o[c].z; wr[4 * c + 3] = o[c].w; }
-            tmem_st32(tdst0 + s * A_COLS, wr);
-            tmem_st_wait();
-            tc_fence_before_sync();
-        } else {
-            const uint32_t dst = dst0 + s * STAGE_BYTES;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) sts128(dst + c * (BN * 16), o[c].x, o[c].y, o[c].z, o[c].w);
-            fence_proxy_async_smem();
-        }
+        for (int c = 0; c < 8; ++c) { wr[4 * c] = o[c].x; wr[4 * c + 1] = o[c].y; wr[4 * c + 2] = o[c].z; wr[4 * c + 3] = o[c].w; }
+        tmem_st32(tdst0 + s * A_COLS, wr);
+        tmem_st_wait();
+        tc_fence_before_sync();
         __syncwarp();
-        if (a.lane == 0) mbar_arrive(smem_u32(&ctl->full[s]));
+        if (a.lane == 0) mbar_arrive(smem_u32(&ctl->full_a[s]));
         // The staging slot is handed back only here, after the stores that consumed the loaded
         // words: a shared-memory load that has merely been issued does not hold back the TMA
         // write that refills the slot (that write belongs to the async proxy; only the data
@@ -163,8 +160,57 @@ __device__ __forceinline__ void produce(const ProducerArgs& a, int r) {
             if (a.lane == 0) mbar_arrive(smem_u32(&ctl->group_empty[gslot]));
             if (++gslot == GROUPS) { gslot = 0; gph ^= 1u; }
         }
-        if (++s == STAGES) { s = 0; ph ^= 1u; }
+        if (++s == A_STAGES) { s = 0; ph ^= 1u; }
         if (++ks == a.nks) ks = 0;
+    }
+}
+
+// Producer of the unit operand: thread = row `r`, one staging group (two stages) per
+// iteration, so the fixed costs of an iteration (group wait, proxy fence, warp barrier,
+// release) are paid once per two stages; widened rows go to shared memory (ring of B_STAGES).
+__device__ __forceinline__ void produce_b(const ProducerArgs& a, int r) {
+    Control* ctl = a.ctl;
+    const int my_tiles = (a.tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
+    const int ng = ceil_div(a.nks, 2);
+    const int total = my_tiles * ng;
+    const uint32_t dst0 = a.smem + r * 16;
+    const uint32_t stg0 = a.smem + B_STAGES * STAGE_BYTES + GA_BYTES + r * 64;
+    const uint32_t sw = (uint32_t)(r >> 1) & 3u;
+    const bool ragged = (a.kw % 8 != 0) || a.tmask != 0xFFFFFFFFu;
+    int gslot = 0;
+    uint32_t gph = 0;
+    int kg = 0, s = 0;
+    uint32_t ph = 1;
+    for (int g = 0; g < total; ++g) {
+        const bool two = 2 * kg + 1 < a.nks;   // the last group of a row may hold a single stage
+        if (!warp_wait(smem_u32(&ctl->group_full[gslot]), gph, a.abort_flag, a.lane)) break;
+        const uint32_t src = stg0 + gslot * GROUP_BYTES;
+        const uint4 v0 = lds128u(src + ((0u ^ sw) << 4)), v1 = lds128u(src + ((1u ^ sw) << 4));
+        const uint4 v2 = lds128u(src + ((2u ^ sw) << 4)), v3 = lds128u(src + ((3u ^ sw) << 4));
+        const int s2 = s + 1 == B_STAGES ? 0 : s + 1;
+        const uint32_t ph2 = s + 1 == B_STAGES ? ph ^ 1u : ph;
+        if (!warp_wait(smem_u32(&ctl->empty_b[s]), ph, a.abort_flag, a.lane)) break;
+        uint4 o[8];
+        widen_stage(a, ragged, 2 * kg, v0, v1, o);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) sts128(dst0 + s * STAGE_BYTES + c * (BN * 16), o[c].x, o[c].y, o[c].z, o[c].w);
+        if (two) {
+            if (!warp_wait(smem_u32(&ctl->empty_b[s2]), ph2, a.abort_flag, a.lane)) break;
+            widen_stage(a, ragged, 2 * kg + 1, v2, v3, o);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) sts128(dst0 + s2 * STAGE_BYTES + c * (BN * 16), o[c].x, o[c].y, o[c].z, o[c].w);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (a.lane == 0) {
+            mbar_arrive(smem_u32(&ctl->full_b[s]));
+            if (two) mbar_arrive(smem_u32(&ctl->full_b[s2]));
+            mbar_arrive(smem_u32(&ctl->group_empty[gslot]));   // after the stores that consumed the loaded words (see produce_a)
+        }
+        if (++gslot == GROUPS) { gslot = 0; gph ^= 1u; }
+        if (two) { s = s2; ph = ph2; }
+        if (++s == B_STAGES) { s = 0; ph ^= 1u; }
+        if (++kg == ng) kg = 0;
     }
 }
 
@@ -176,7 +222,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                 uint32_t* __restrict__ out_bits, int ldob, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES + GROUPS * GROUP_BYTES);
+    Control* ctl = reinterpret_cast<Control*>(smem + B_STAGES * STAGE_BYTES + GROUPS * GROUP_BYTES);
     int (*cstage)[2][32][36] = reinterpret_cast<int (*)[2][32][36]>(reinterpret_cast<uint8_t*>(ctl) + sizeof(Control));
     volatile int* abort_flag = &ctl->abort;
 
@@ -187,9 +233,13 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     const int tiles = m_tiles * n_tiles;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), PROD_WARPS);
-            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        for (int s = 0; s < A_STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full_a[s]), A_WARPS);
+            mbar_init(smem_u32(&ctl->empty_a[s]), 1);
+        }
+        for (int s = 0; s < B_STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full_b[s]), B_WARPS);
+            mbar_init(smem_u32(&ctl->empty_b[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
@@ -228,7 +278,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         if (warp == TMA_WARP) {
             // ---------------- one thread feeds the staging ring, a group of two stages at a time
             if (lane == 0) {
-                const uint32_t stg = smem_u32(smem) + STAGES * STAGE_BYTES;
+                const uint32_t stg = smem_u32(smem) + B_STAGES * STAGE_BYTES;
                 const int ng = ceil_div(nks, 2);
                 int gc = 0;
                 bool ok = true;
@@ -249,9 +299,9 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             }
             __syncwarp();
         } else if (warp < PROD_WARP0 + A_WARPS) {
-            produce<true>(pa, (warp & 3) * 32 + lane);
+            produce_a(pa, (warp & 3) * 32 + lane);
         } else {
-            produce<false>(pa, (warp - PROD_WARP0 - A_WARPS) * 32 + lane);
+            produce_b(pa, (warp - PROD_WARP0 - A_WARPS) * 32 + lane);
         }
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issue: one thread
@@ -268,18 +318,20 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                 tc_fence_after_sync();
                 const uint32_t d = tmem + (uint32_t)(b * BN);
                 for (int ks = 0; ks < nks; ++ks, ++it) {
-                    const int s = it % STAGES;
-                    ok = mbar_wait(smem_u32(&ctl->full[s]), (uint32_t)((it / STAGES) & 1), abort_flag);
+                    const int sa = it % A_STAGES, sb = it % B_STAGES;
+                    ok = mbar_wait(smem_u32(&ctl->full_b[sb]), (uint32_t)((it / B_STAGES) & 1), abort_flag) &&
+                         mbar_wait(smem_u32(&ctl->full_a[sa]), (uint32_t)((it / A_STAGES) & 1), abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t b0 = smem_u32(smem + s * STAGE_BYTES);
-                    const uint32_t ta = tmem + TMEM_A_COL + s * A_COLS;
+                    const uint32_t b0 = smem_u32(smem + sb * STAGE_BYTES);
+                    const uint32_t ta = tmem + TMEM_A_COL + sa * A_COLS;
 #pragma unroll
                     for (int j = 0; j < BK / 64; ++j) {   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
                         const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (BN * 16), BN * 16, 128);
                         mma_mxf4_ts(d, ta + 8 * j, db, idesc, sfa, sfb, (ks | j) != 0);
                     }
-                    mma_commit(smem_u32(&ctl->empty[s]));
+                    mma_commit(smem_u32(&ctl->empty_a[sa]));
+                    mma_commit(smem_u32(&ctl->empty_b[sb]));
                 }
                 if (ok) mma_commit(smem_u32(&ctl->acc_full[b]));
             }
