@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--sweep", action="store_true",
                     help="isolated XNOR GEMM sweep (M x K x N x bit density), one JSON line per point")
     ap.add_argument("--sweep-quick", action="store_true", help="only the corner points of the sweep")
+    ap.add_argument("--pipe-rates", action="store_true",
+                    help="measure the rates of the pipes that bound the kernels (popc, lop3, iadd, fadd, ffma, "
+                         "4-bit and fp16 tensor-core MMA, L2 reads); one JSON line per pipe")
     ap.add_argument("--real-path", default="tensor", choices=["tensor", "fp32"],
                     help="kernel of the real-valued layers: tcgen05 with split operands or the FP32 pipe")
     ap.add_argument("--xnor-path", default="tensor", choices=["tensor", "popc"],
@@ -527,9 +530,53 @@ def run_sweep(args):
                 del A
 
 
+def run_pipe_rates(args):
+    """Rates of the execution pipes the kernels are bound by, measured with the library's own
+    micro-benchmark launches (bnn_pipe_rate), each timed with CUDA events after a warm-up launch;
+    SM clock and throttle reasons sampled meanwhile."""
+    import torch
+    from paper_1706_09453_b200 import build
+    build.build()
+    from paper_1706_09453_b200 import binding as B
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    scratch = torch.zeros(max(B.bnn_pipe_rate_scratch_bytes(k) for k in B.RATE_KINDS.values()), dtype=torch.uint8, device=dev)
+    plan = [("popc", 256, "Tbop/s", 1e12), ("lop3", 256, "Tinst/s", 1e12), ("iadd", 256, "Tinst/s", 1e12),
+            ("fadd", 256, "Tinst/s", 1e12), ("ffma", 256, "TFLOP/s", 1e12),
+            ("mma_mxf4_n256", 512, "Tbop/s", 1e12), ("mma_mxf4_n192", 512, "Tbop/s", 1e12),
+            ("mma_mxf4_n192_atmem", 512, "Tbop/s", 1e12), ("mma_f16_n256", 512, "TFLOP/s", 1e12),
+            ("l2_read", 4, "GB/s", 1e9)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for name, repeat, unit, scale in plan:
+        kind = B.RATE_KINDS[name]
+        B.bnn_pipe_rate(kind, repeat, scratch)          # warm-up
+        torch.cuda.synchronize()
+        sampler = ClockSampler(torch, 0)
+        sampler.start()
+        reps = 10
+        e0.record()
+        for _ in range(reps):
+            work = B.bnn_pipe_rate(kind, repeat, scratch)
+        e1.record()
+        torch.cuda.synchronize()
+        sampler.stop()
+        ms = e0.elapsed_time(e1) / reps
+        rec = {"pipe_rate": name, "rate": work / (ms * 1e-3) / scale, "unit": unit, "ms_per_launch": ms,
+               "work_per_launch": work, "launches": reps, "clocks": sampler.summary(),
+               "device_status": B.bnn_device_status()}
+        if name.startswith("mma_mxf4"):
+            rec["vs_4x_bf16_burst"] = rec["rate"] / (4 * peaks["bf16_tflops"])
+        if name == "mma_f16_n256":
+            rec["vs_bf16_burst"] = rec["rate"] / peaks["bf16_tflops"]
+        print(json.dumps(rec), flush=True)
+
+
 if __name__ == "__main__":
     a = parse_args()
-    if a.sweep:
+    if a.pipe_rates:
+        run_pipe_rates(a)
+    elif a.sweep:
         run_sweep(a)
     elif a.impl == "reference":
         run_reference(a)

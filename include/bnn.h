@@ -277,6 +277,33 @@ BNN_API int bnn_set_option(int option, int value);
  * affected launch are invalid).  The paper has no counterpart. */
 BNN_API int bnn_device_status(int* status);
 
+/* Micro-benchmarks of the pipes that bound the kernels above (measurement support; the paper
+ * has no counterpart: its Section 3 reports accuracy only).  bnn_pipe_rate enqueues ONE launch
+ * on `stream` that executes a fixed number of operations of the chosen kind on every SM and
+ * stores that number in *work (host pointer, written before the call returns): bit
+ * operations for POPC (32 x 2 per instruction, the convention of the XNOR layer: 1 bit-MAC =
+ * 2 bop), thread-level instructions for LOP3 / IADD / FADD, flops for FFMA (2 per
+ * instruction), bop for the 4-bit MMAs and flop for the fp16 MMA (2 per MAC), bytes for
+ * L2_READ.  The caller times the launch with CUDA events on `stream`; rate = *work / time.
+ *   POPC, LOP3, IADD, FADD, FFMA : 8 independent dependency chains per thread, 2048 threads/SM
+ *   MMA_MXF4_N256 / _N192        : tcgen05.mma kind::mxf4, 128 x N x 64, operands in shared memory
+ *   MMA_MXF4_N192_ATMEM          : the same with the A operand in tensor memory
+ *   MMA_F16_N256                 : tcgen05.mma kind::f16, 128 x 256 x 16
+ *   L2_READ                      : every SM reads the same 32 MB of `scratch`
+ * repeat (1 .. 2^20) scales the work linearly (loop trips; groups of 64 MMAs; passes over
+ * the 32 MB).  scratch: DEVICE buffer owned by the caller, 16-byte aligned, at least
+ * bnn_pipe_rate_scratch_bytes(which) bytes; its contents are overwritten (L2_READ only reads
+ * the first 32 MB).  Errors: BNN_ERR_NULL, BNN_ERR_SHAPE (repeat), BNN_ERR_WORKSPACE,
+ * BNN_ERR_ALIGN, BNN_ERR_UNSUPPORTED (unknown kind), BNN_ERR_CUDA.  The MMA kinds use bounded
+ * waits like every tensor kernel here; a wait that runs out shows in bnn_device_status. */
+typedef enum {
+    BNN_RATE_POPC = 0, BNN_RATE_LOP3 = 1, BNN_RATE_IADD = 2, BNN_RATE_FADD = 3, BNN_RATE_FFMA = 4,
+    BNN_RATE_MMA_MXF4_N256 = 5, BNN_RATE_MMA_MXF4_N192 = 6, BNN_RATE_MMA_MXF4_N192_ATMEM = 7,
+    BNN_RATE_MMA_F16_N256 = 8, BNN_RATE_L2_READ = 9
+} bnn_rate_kind;
+BNN_API size_t bnn_pipe_rate_scratch_bytes(int which);
+BNN_API int bnn_pipe_rate(int which, int repeat, void* scratch, size_t scratch_bytes, double* work, void* stream);
+
 /* Smallest legal packed pitch (in words) for rows of K bits: ceil(K/32) rounded up to 4. */
 BNN_API int bnn_packed_pitch(int K);
 

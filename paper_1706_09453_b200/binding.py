@@ -70,6 +70,10 @@ def lib():
         L.bnn_output_prepared_bytes.restype = C.c_size_t
         L.bnn_output_prepare.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
         L.bnn_output_prepare.restype = C.c_int
+        L.bnn_pipe_rate_scratch_bytes.argtypes = [C.c_int]
+        L.bnn_pipe_rate_scratch_bytes.restype = C.c_size_t
+        L.bnn_pipe_rate.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.POINTER(C.c_double), C.c_void_p]
+        L.bnn_pipe_rate.restype = C.c_int
         L.bnn_device_status.argtypes = [C.POINTER(C.c_int)]
         L.bnn_device_status.restype = C.c_int
         L.bnn_forward_workspace_bytes.restype = C.c_size_t
@@ -122,6 +126,22 @@ def bnn_set_option(option: int, value: int) -> int:
 
 def bnn_set_xnor_path(path: int) -> int:
     return bnn_set_option(OPT_XNOR_PATH, path)
+
+
+RATE_KINDS = {"popc": 0, "lop3": 1, "iadd": 2, "fadd": 3, "ffma": 4, "mma_mxf4_n256": 5, "mma_mxf4_n192": 6,
+              "mma_mxf4_n192_atmem": 7, "mma_f16_n256": 8, "l2_read": 9}
+
+
+def bnn_pipe_rate_scratch_bytes(which: int) -> int:
+    return lib().bnn_pipe_rate_scratch_bytes(which)
+
+
+def bnn_pipe_rate(which: int, repeat: int, scratch) -> float:
+    """Enqueues one micro-benchmark launch on the current stream; returns the work it performs."""
+    work = C.c_double(0.0)
+    _check(lib().bnn_pipe_rate(which, repeat, _ptr(scratch), scratch.numel() * scratch.element_size(),
+                               C.byref(work), _stream()), "bnn_pipe_rate")
+    return work.value
 
 
 def bnn_device_status() -> int:

@@ -88,6 +88,12 @@ extern "C" {
 
 int bnn_packed_pitch(int K) { return (words_for(K) + 3) & ~3; }
 
+size_t bnn_pipe_rate_scratch_bytes(int which) { return pipe_rate_scratch_bytes(which); }
+
+int bnn_pipe_rate(int which, int repeat, void* scratch, size_t scratch_bytes, double* work, void* stream) {
+    return launch_pipe_rate(which, repeat, scratch, scratch_bytes, work, static_cast<cudaStream_t>(stream));
+}
+
 int bnn_set_option(int option, int value) {
     int* slot = nullptr;
     switch (option) {

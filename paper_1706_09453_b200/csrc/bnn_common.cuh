@@ -55,6 +55,9 @@ constexpr int kMaxKTensor = 1 << 22;
 int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
                    int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
                    uint32_t* out_bits, int ldob, cudaStream_t st);
+// Pipe micro-benchmarks (pipe_rates.cu).
+size_t pipe_rate_scratch_bytes(int which);
+int launch_pipe_rate(int which, int repeat, void* scratch, size_t scratch_bytes, double* work, cudaStream_t st);
 // Tensor map of a packed operand [rows][ceil(K/32) words] of pitch `ld` words: boxes of 16 words x
 // box_rows rows, 64-byte swizzle, zero fill outside the tensor.  False when the encoder fails.
 bool encode_packed_map(CUtensorMap* map, const uint32_t* base, int ld, int rows, int K, int box_rows);

@@ -402,3 +402,19 @@ def test_signw_gemm_tensor_error_bound_by_terms(B, torch_, terms, with_ws):
         B.bnn_set_option(B.OPT_SIGNW_TERMS, prev_t)
         B.bnn_set_option(B.OPT_REAL_PATH, prev_p)
     assert B.bnn_device_status() == 0
+
+
+# ------------------------------------------------------------------ pipe micro-benchmarks
+def test_pipe_rate_launches_run_and_report_their_work(B, torch_):
+    scratch = torch_.zeros(max(B.bnn_pipe_rate_scratch_bytes(k) for k in B.RATE_KINDS.values()), dtype=torch_.uint8,
+                           device="cuda:0")
+    for name, kind in B.RATE_KINDS.items():
+        w1 = B.bnn_pipe_rate(kind, 1, scratch)
+        w2 = B.bnn_pipe_rate(kind, 2, scratch)
+        assert w1 > 0 and w2 == 2 * w1, name          # the work scales linearly with `repeat`
+    torch_.cuda.synchronize()
+    assert B.bnn_device_status() == 0
+    with pytest.raises(B.BnnError):
+        B.bnn_pipe_rate(99, 1, scratch)               # unknown kind
+    with pytest.raises(B.BnnError):
+        B.bnn_pipe_rate(0, 1, scratch[:1024])         # scratch too small
