@@ -47,7 +47,7 @@ def parse_args():
                          "4-bit and fp16 tensor-core MMA, L2 reads); one JSON line per pipe")
     ap.add_argument("--real-path", default="tensor", choices=["tensor", "fp32"],
                     help="kernel of the real-valued layers: tcgen05 with split operands or the FP32 pipe")
-    ap.add_argument("--xnor-path", default="tensor", choices=["tensor", "popc"],
+    ap.add_argument("--xnor-path", default="tensor", choices=["tensor", "tensor-unprepared", "popc"],
                     help="kernel of the binary hidden layers: tcgen05 tensor core or integer-pipe popcount")
     return ap.parse_args()
 
@@ -177,7 +177,7 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
     for l in range(cfg.n_hidden):
         xnor = cfg.act == 1 and l > 0
         work = 2.0 * frames * cfg.hidden * k
-        if xnor and xnor_path == "tensor":
+        if xnor and xnor_path in ("tensor", "tensor-unprepared"):
             # 4-bit (e2m1, kind::mxf4) tensor-core MACs: 4 x the measured bf16 rate (nominal ratio
             # 9 : 2.25 PFLOP/s), sustained figure because the kernel is timed inside a long step;
             # 1 bit-MAC = 2 bop.  smem_bytes: what the kernel moves through the SM's shared
@@ -187,7 +187,12 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
             tiles_m, tiles_n = -(-frames // 128), -(-cfg.hidden // 192)
             kpad = -(-k // 256) * 256
             smem_bytes = tiles_m * tiles_n * kpad * (192 * (0.5 + 0.5 + 0.125 + 0.125) + 128 * (0.125 + 0.125))
-            rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_tc_kernel", work=work, unit="Tbop/s",
+            if xnor_path == "tensor":
+                # weights prepared once: their widened image arrives by bulk copies (4 bits written,
+                # 4 bits read by the tensor core per weight bit and tile visit); nothing else
+                smem_bytes = tiles_m * tiles_n * kpad * (192 * (0.5 + 0.5) + 128 * (0.125 + 0.125))
+            rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_img_kernel" if xnor_path == "tensor" else "xnor_tc_kernel",
+                             work=work, unit="Tbop/s",
                              bound="tensor", peak=4.0 * peaks["bf16_tflops_sustained"], smem_bytes=smem_bytes))
         elif xnor:
             rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_popc_kernel", work=work, unit="Tbop/s",
@@ -261,9 +266,9 @@ def run_ours(args):
     cfg = wl.CONFIGS[args.config]
     frames = args.frames or cfg.frames
     net = wl.make_model(cfg)
-    B.bnn_set_xnor_path(B.XNOR_TENSOR if args.xnor_path == "tensor" else B.XNOR_POPC)
+    B.bnn_set_xnor_path(B.XNOR_POPC if args.xnor_path == "popc" else B.XNOR_TENSOR)
     B.bnn_set_option(B.OPT_REAL_PATH, B.PATH_TENSOR if args.real_path == "tensor" else B.PATH_CUDA_CORE)
-    dn = model.DeviceNet(net, device=dev)
+    dn = model.DeviceNet(net, device=dev, prepare_xnor=args.xnor_path == "tensor")
     # Frames are independent, so ranks shard them with no exchange: each rank owns its own batch.
     Xh = wl.make_frames(cfg, frames, seed=D.frames_seed(cfg.seed, rank))
     set_bytes = frames * (cfg.in_dim + cfg.classes) * 4
@@ -389,7 +394,7 @@ def run_ours(args):
                 "frac": achieved / dom["peak"], "traffic": ncu_traffic(dk),
                 "peak_source": ("4 x bf16_tflops_sustained of MEASURED_PEAKS.json (%s): e2m1 (mxf4) MMA = 4 x bf16 (nominal ratio), "
                                 "sustained figure because the kernel is timed inside a long step; of measured"
-                                % peaks["source"]) if dk == "xnor_tc_kernel" else
+                                % peaks["source"]) if dk in ("xnor_tc_kernel", "xnor_img_kernel") else
                                ("bf16_tflops_sustained of MEASURED_PEAKS.json (%s); of measured" % peaks["source"])
                                if dom["bound"] == "tensor" else
                                ("hbm_gbs of MEASURED_PEAKS.json (%s); of measured" % peaks["source"])
@@ -414,7 +419,7 @@ def run_ours(args):
         "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "%s (hidden layers) + %s (first and top layer)"
-                 % ("e2m1 (mxf4) tensor-core MMA, f32 accumulate, exact" if args.xnor_path == "tensor" else "int32 popcount",
+                 % ("e2m1 (mxf4) tensor-core MMA, f32 accumulate, exact" if args.xnor_path != "popc" else "int32 popcount",
                     "split bf16/fp16 tensor-core MMA, f32 accumulate" if args.real_path == "tensor" else "f32"),
         "device_status": B.bnn_device_status(), "data": "synthetic",
         "config": {"workload": workload_name(cfg, frames), "frames_per_gpu": frames,

@@ -123,6 +123,27 @@ BNN_API int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int 
                   int M, int N, int K, int32_t* C, int ldc,
                   const bnn_epilogue* epi, void* stream);
 
+/* One-time preparation of a binary layer's weights for the tensor cores, and the product of
+ * bnn_xnor_gemm on the prepared form.  The tensor cores multiply nothing narrower than 4-bit
+ * numbers, so every +-1 has to be widened to 4 bits on its way to them; a layer's weights are
+ * the same for every batch, so bnn_xnor_prepare widens them once, into an image laid out in
+ * the order the tensor core reads shared memory (4 bits per weight, rounded up to tiles of
+ * 192 units x 256 inputs), and bnn_xnor_gemm_prepared streams that image with bulk copies
+ * instead of widening the weights again for every tile of frames.  Same integers, same bits.
+ * The packed matrix Wp stays the model's stored form (1 bit per weight, the paper's memory
+ * argument); the image is a cache that can be rebuilt from it at any time.
+ *   prepared : device buffer, 256-byte aligned, at least bnn_xnor_prepared_bytes(N, K) bytes;
+ *              written by bnn_xnor_prepare, read by bnn_xnor_gemm_prepared with the SAME N, K.
+ *   K <= 2^22 (larger K: BNN_ERR_UNSUPPORTED; use bnn_xnor_gemm).  Other arguments and errors
+ *   as bnn_xnor_gemm; a short buffer -> BNN_ERR_WORKSPACE.
+ * The paper has no counterpart (it leaves efficient binary products to hardware; Section 3). */
+BNN_API size_t bnn_xnor_prepared_bytes(int N, int K);
+BNN_API int bnn_xnor_prepare(const uint32_t* Wp, int ldwp, int N, int K,
+                             void* prepared, size_t prepared_bytes, void* stream);
+BNN_API int bnn_xnor_gemm_prepared(const uint32_t* Ap, int ldap, const void* prepared,
+                                   int M, int N, int K, int32_t* C, int ldc,
+                                   const bnn_epilogue* epi, void* stream);
+
 /* ------------------------------------------------------------------------------------
  * Binary weights against real-valued activations (Section 2.1; Algorithm 1 forward):
  * y[m][n] = sum_k w^b[n][k]*x[m][k] -- additions and subtractions only -- followed by the
@@ -189,7 +210,8 @@ typedef struct bnn_layer {
     int ldwp;
     const float* W;        /* REAL_OUT: fp32 weights [N][ldw] */
     int ldw;
-    const void* W_prepared;/* REAL_OUT: bnn_output_prepare image of W, or NULL */
+    const void* W_prepared;/* REAL_OUT: bnn_output_prepare image of W, or NULL;
+                              XNOR: bnn_xnor_prepare image of Wp, or NULL */
     const float* scale;    /* SIGNW: per-unit scale or NULL */
     const float* shift;    /* SIGNW: per-unit shift or NULL; REAL_OUT: bias or NULL */
     const int32_t* thr;    /* XNOR: folded thresholds [N] */

@@ -70,6 +70,13 @@ def lib():
         L.bnn_output_prepared_bytes.restype = C.c_size_t
         L.bnn_output_prepare.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
         L.bnn_output_prepare.restype = C.c_int
+        L.bnn_xnor_prepared_bytes.argtypes = [C.c_int, C.c_int]
+        L.bnn_xnor_prepared_bytes.restype = C.c_size_t
+        L.bnn_xnor_prepare.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.bnn_xnor_prepare.restype = C.c_int
+        L.bnn_xnor_gemm_prepared.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                             C.c_int, C.POINTER(Epilogue), C.c_void_p]
+        L.bnn_xnor_gemm_prepared.restype = C.c_int
         L.bnn_pipe_rate_scratch_bytes.argtypes = [C.c_int]
         L.bnn_pipe_rate_scratch_bytes.restype = C.c_size_t
         L.bnn_pipe_rate.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.POINTER(C.c_double), C.c_void_p]
@@ -222,6 +229,27 @@ def bnn_xnor_gemm(Ap, Wp, K, C_out=None, thr=None, flip=None, out_bits=None):
     _check(lib().bnn_xnor_gemm(_ptr(Ap, torch.int32), _ld(Ap), _ptr(Wp, torch.int32), _ld(Wp), m, n, K,
                                _ptr(C_out, torch.int32), _ld(C_out) if C_out is not None else 0,
                                e, _stream()), "bnn_xnor_gemm")
+
+
+def bnn_xnor_prepared_bytes(N, K) -> int:
+    return int(lib().bnn_xnor_prepared_bytes(int(N), int(K)))
+
+
+def bnn_xnor_prepare(Wp, K, prepared):
+    """Packed weights [N][pitch] -> their widened image in ``prepared`` (uint8 CUDA tensor)."""
+    _check(lib().bnn_xnor_prepare(_ptr(Wp, torch.int32), _ld(Wp), Wp.shape[0], K, _ptr(prepared),
+                                  prepared.numel() * prepared.element_size(), _stream()), "bnn_xnor_prepare")
+    return prepared
+
+
+def bnn_xnor_gemm_prepared(Ap, prepared, N, K, C_out=None, thr=None, flip=None, out_bits=None):
+    """bnn_xnor_gemm with the weights given as the image bnn_xnor_prepare made of them."""
+    e = None
+    if out_bits is not None:
+        e = C.byref(_epilogue(ACT_SIGN_PACK, thr=thr, flip=flip, out_bits=out_bits))
+    _check(lib().bnn_xnor_gemm_prepared(_ptr(Ap, torch.int32), _ld(Ap), _ptr(prepared), Ap.shape[0], N, K,
+                                        _ptr(C_out, torch.int32), _ld(C_out) if C_out is not None else 0,
+                                        e, _stream()), "bnn_xnor_gemm_prepared")
 
 
 def bnn_signw_workspace_bytes(M, K) -> int:

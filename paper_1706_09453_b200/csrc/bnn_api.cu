@@ -148,13 +148,19 @@ int bnn_fold_thresholds(const float* scale, const float* shift, int N, int K, in
     return launch_fold_thresholds(scale, shift, N, K, sign_mode, thr, flip, (cudaStream_t)stream);
 }
 
-int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
-                  int M, int N, int K, int32_t* C, int ldc,
-                  const bnn_epilogue* epi, void* stream) {
+// Shared by bnn_xnor_gemm (image == nullptr) and bnn_xnor_gemm_prepared (Wp == nullptr).
+static int xnor_gemm_impl(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, const void* image,
+                          int M, int N, int K, int32_t* C, int ldc,
+                          const bnn_epilogue* epi, void* stream) {
     if (int rc = check_dims(M, N, K)) return rc;
     if (K > kMaxK) return BNN_ERR_SHAPE;
     if (int rc = check_packed(Ap, ldap, K)) return rc;
-    if (int rc = check_packed(Wp, ldwp, K)) return rc;
+    if (image) {
+        if (K > kMaxKTensor) return BNN_ERR_UNSUPPORTED;
+        if (reinterpret_cast<uintptr_t>(image) & 255u) return BNN_ERR_ALIGN;
+    } else if (int rc = check_packed(Wp, ldwp, K)) {
+        return rc;
+    }
     if (C && ldc < N) return BNN_ERR_SHAPE;
     const int32_t* thr = nullptr;
     const uint32_t* flip = nullptr;
@@ -167,9 +173,46 @@ int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
         thr = epi->thr; flip = epi->flip; ob = epi->out_bits; ldob = epi->ldob;
     }
     if (!C && !ob) return BNN_ERR_NULL;
+    if (image) {
+        // fused Sign layer: the kernel that keeps a unit tile's weights in shared memory, when
+        // they fit; int32 output and the remaining shapes: the kernel that streams the image
+        if (!C && xnor_res_applicable(N, K))
+            return launch_xnor_res(Ap, ldap, image, M, N, K, thr, flip, ob, ldob, (cudaStream_t)stream);
+        return launch_xnor_img(Ap, ldap, image, M, N, K, C, ldc, thr, flip, ob, ldob, (cudaStream_t)stream);
+    }
     const bool tensor = g_xnor_path != BNN_PATH_CUDA_CORE && K <= kMaxKTensor;
     return (tensor ? launch_xnor_tc : launch_xnor_popc)(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip,
                                                         ob, ldob, (cudaStream_t)stream);
+}
+
+int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
+                  int M, int N, int K, int32_t* C, int ldc,
+                  const bnn_epilogue* epi, void* stream) {
+    if (!Wp) return BNN_ERR_NULL;
+    return xnor_gemm_impl(Ap, ldap, Wp, ldwp, nullptr, M, N, K, C, ldc, epi, stream);
+}
+
+size_t bnn_xnor_prepared_bytes(int N, int K) {
+    if (N < 1 || K < 1 || K > kMaxKTensor) return 0;
+    return xnor_image_bytes(N, K);
+}
+
+int bnn_xnor_prepare(const uint32_t* Wp, int ldwp, int N, int K,
+                     void* prepared, size_t prepared_bytes, void* stream) {
+    if (!prepared) return BNN_ERR_NULL;
+    if (N < 1 || K < 1) return BNN_ERR_SHAPE;
+    if (K > kMaxKTensor) return BNN_ERR_UNSUPPORTED;
+    if (int rc = check_packed(Wp, ldwp, K)) return rc;
+    if (prepared_bytes < xnor_image_bytes(N, K)) return BNN_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(prepared) & 255u) return BNN_ERR_ALIGN;
+    return launch_xnor_prepare(Wp, ldwp, N, K, prepared, (cudaStream_t)stream);
+}
+
+int bnn_xnor_gemm_prepared(const uint32_t* Ap, int ldap, const void* prepared,
+                           int M, int N, int K, int32_t* C, int ldc,
+                           const bnn_epilogue* epi, void* stream) {
+    if (!prepared) return BNN_ERR_NULL;
+    return xnor_gemm_impl(Ap, ldap, nullptr, 0, prepared, M, N, K, C, ldc, epi, stream);
 }
 
 size_t bnn_signw_workspace_bytes(int M, int K) {
@@ -363,8 +406,9 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
         } else {
             e.thr = y.thr; e.flip = y.flip;
             e.out_bits = static_cast<uint32_t*>(out); e.ldob = bnn_packed_pitch(y.N);
-            rc = bnn_xnor_gemm(static_cast<const uint32_t*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
-                               nullptr, 0, &e, stream);
+            const bool image = y.W_prepared && g_xnor_path != BNN_PATH_CUDA_CORE && y.K <= kMaxKTensor;
+            rc = xnor_gemm_impl(static_cast<const uint32_t*>(in), in_ld, y.Wp, y.ldwp,
+                                image ? y.W_prepared : nullptr, M, y.N, y.K, nullptr, 0, &e, stream);
             in_ld = e.ldob;
         }
         if (rc) return rc;

@@ -55,6 +55,20 @@ constexpr int kMaxKTensor = 1 << 22;
 int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
                    int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
                    uint32_t* out_bits, int ldob, cudaStream_t st);
+// The same product with the unit operand given as the image launch_xnor_prepare built from the
+// packed weights (xnor_gemm_img.cu): xnor_image_bytes(N, K) bytes, 256-byte aligned.
+size_t xnor_image_bytes(int N, int K);
+// Units per chunk of the image: N rounded up to a multiple of 384 (tiles of 192 or 128 units).
+__host__ __device__ __forceinline__ int xnor_image_npad(int N) { return ceil_div(N, 384) * 384; }
+// Fused Sign layer with the weights of a unit tile resident in shared memory (xnor_gemm_res.cu);
+// xnor_res_applicable says whether a layer of this shape fits that kernel.
+bool xnor_res_applicable(int N, int K);
+int launch_xnor_res(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
+                    const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, cudaStream_t st);
+int launch_xnor_prepare(const uint32_t* Wp, int ldwp, int N, int K, void* image, cudaStream_t st);
+int launch_xnor_img(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
+                    int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
+                    uint32_t* out_bits, int ldob, cudaStream_t st);
 // Pipe micro-benchmarks (pipe_rates.cu).
 size_t pipe_rate_scratch_bytes(int which);
 int launch_pipe_rate(int which, int repeat, void* scratch, size_t scratch_bytes, double* work, cudaStream_t st);

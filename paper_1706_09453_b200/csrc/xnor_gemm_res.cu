@@ -1,0 +1,416 @@
+// Fused binary hidden layer on the tensor cores with the layer's weights RESIDENT in shared
+// memory:  bits[m][n] = Sign(scale[n] * sum_k a[m][k] * w[n][k] + shift[n]),  a, w in {-1, +1}.
+//
+// Same contraction as xnor_gemm_tc.cu / xnor_gemm_img.cu (every +-1 widened to a 4-bit e2m1
+// nibble, kind::mxf4, unit block scales, exact fp32 sums).  Measured on B200, streaming the
+// widened weights from L2 for every tile of frames holds the tensor pipe at about a third of
+// its rate (24 KB per 384 MMA clocks and SM is more than L2 delivers to 148 SMs at once).  So
+// here a CTA owns ONE tile of units for the whole launch: it loads that tile's slice of the
+// prepared weight image (all of K, up to 192 KB) into shared memory once and then walks over
+// frame tiles, for which only the packed frame bits (4 KB per stage) cross L2.  CTA c works on
+// unit tile c mod n_tiles and shares that tile's frame tiles with the other CTAs of the same
+// residue.
+//
+// The image is the one xnor_gemm_img.cu describes: a tile of BN units is, per stage of 256
+// positions of K, eight contiguous runs of BN x 16 bytes, copied to offsets c * BN * 16 of the
+// stage's block (K-major core matrices).  BN = 192 while K <= 2048 and BN = 128 while
+// K <= 3072 keep the slice within 192 KB; other shapes are left to the streaming kernel.
+//
+// Roles in a CTA of 14 warps (one CTA per SM):
+//   warp 13      one thread issues the bulk copies of the weight slice (once) and the 2-D TMA
+//                tile loads of the packed frame rows (64 bytes per row = two stages) into a
+//                staging ring (64-byte swizzle, no multicast)
+//   warps 5-12   two teams of four warps widen the frame rows, thread = one row, 32 bytes ->
+//                128 bytes per stage, into tensor memory (the MMA reads its A operand from
+//                there); the teams take alternate stages
+//   warp 4       one thread issues the MMAs (4 per stage, K = 64 each) and the commits
+//   warps 0-3    epilogue: accumulator -> threshold -> repacked bits; two accumulators in
+//                tensor memory, so it overlaps the next tile's MMAs
+// Every wait is bounded; a wait that runs out sets the CTA's abort flag, all roles fall
+// through to the common teardown and the device status word is set.
+#include "bnn_common.cuh"
+#include "tcgen05.cuh"
+#include "xnor_widen.cuh"
+
+namespace bnn {
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128;
+constexpr int BK = 256;                                   // positions of K per stage
+constexpr int ROW_BYTES = BK / 2;                         // widened bytes per row and stage (128)
+constexpr int B_REGION = 192 * 1024;                      // shared memory that holds the weight slice
+constexpr int EPI_WARPS = 4, MMA_WARP = 4, PROD_WARP0 = 5, A_WARPS = BM / 32, TEAMS = 2;
+constexpr int TMA_WARP = PROD_WARP0 + TEAMS * A_WARPS;
+constexpr int THREADS = (TMA_WARP + 1) * 32;              // 448
+constexpr int GROUPS = 4;                                 // staging ring of the packed frame rows: groups of two stages
+constexpr int GROUP_BYTES = BM * 64;
+constexpr uint32_t A_COLS = ROW_BYTES / 4;                // 32-bit columns per A stage
+constexpr uint32_t SF_COLS = 32, TMEM_COLS = 512;
+constexpr int MAX_NKS = 16;
+
+template <int BN> struct Cfg {
+    static constexpr int B_BYTES = BN * ROW_BYTES;                 // one stage of the unit operand
+    static constexpr int NKS = B_REGION / B_BYTES;                 // stages that fit: 8 (BN 192), 12 (BN 128)
+    static constexpr int A_STAGES = (int)((TMEM_COLS - SF_COLS - 2 * BN) / A_COLS) > 6 ? 6 : (int)((TMEM_COLS - SF_COLS - 2 * BN) / A_COLS);
+    static constexpr uint32_t TMEM_A_COL = 2 * BN;                 // A stages start after the two accumulators
+    static constexpr uint32_t TMEM_SF_COL = TMEM_A_COL + A_STAGES * A_COLS;
+    static_assert(NKS <= MAX_NKS && A_STAGES >= 3 && TMEM_SF_COL + SF_COLS <= TMEM_COLS, "tile configuration");
+};
+
+struct Control {
+    int T[192];              // per unit: threshold + kMagicBits
+    uint32_t flipw[8];
+    uint64_t full_a[6], empty_a[6], full_b[MAX_NKS], acc_full[2], acc_empty[2];
+    uint64_t group_full[GROUPS], group_empty[GROUPS];
+    uint32_t tmem_base;
+    int abort;
+};
+constexpr int SMEM_BYTES = B_REGION + GROUPS * GROUP_BYTES + (int)sizeof(Control) + 1024;
+static_assert(SMEM_BYTES <= 232448, "shared memory of one CTA");
+
+// 1-D bulk asynchronous copy global -> shared; completion is counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Frame tiles of this CTA: mt = first, first + step, ... < m_tiles.
+struct Share {
+    int first, step, count;
+};
+__device__ __forceinline__ Share my_share(int m_tiles, int n_tiles) {
+    const int nt = (int)blockIdx.x % n_tiles, r = (int)blockIdx.x / n_tiles;
+    const int peers = ((int)gridDim.x - 1 - nt) / n_tiles + 1;    // CTAs that work on unit tile nt
+    Share s;
+    s.first = r; s.step = peers;
+    s.count = r < m_tiles ? (m_tiles - 1 - r) / peers + 1 : 0;
+    return s;
+}
+
+struct ProducerArgs {
+    uint32_t smem_stage;  // shared-space address of the staging ring
+    uint32_t tmem_a;      // tensor-memory address of A stage 0 (lane 0)
+    Control* ctl;
+    volatile int* abort_flag;
+    int my_tiles, nks, kw;
+    uint32_t tmask;
+    int lane;
+};
+
+// Producer of the frame operand: thread = row `r` of every tile of this CTA; team `team`
+// takes the stages it = team, team + TEAMS, ... of the CTA's sequence of (tile, stage) pairs.
+template <int A_STAGES>
+__device__ __forceinline__ void produce_a(const ProducerArgs& a, int r, int team) {
+    Control* ctl = a.ctl;
+    const int total = a.my_tiles * a.nks;
+    const int ng = ceil_div(a.nks, 2);
+    // TMEM lane of this thread's frame row: a warp may only touch lanes 32*(warp%4)..+31
+    const uint32_t tdst0 = a.tmem_a + ((uint32_t)(r & ~31) << 16);
+    // this row inside a staging group: 64 bytes per row, 16-byte chunk c stored at c ^ ((r/2)%4)
+    const uint32_t stg0 = a.smem_stage + r * 64;
+    const uint32_t sw = (uint32_t)(r >> 1) & 3u;
+    const bool ragged = (a.kw % 8 != 0) || a.tmask != 0xFFFFFFFFu;   // last stage has positions >= K
+    int ks = team, tl = 0;
+    while (ks >= a.nks) { ks -= a.nks; ++tl; }
+    for (int it = team; it < total; it += TEAMS) {
+        const int gidx = tl * ng + (ks >> 1);          // staging group that holds this stage
+        const int gslot = gidx % GROUPS;
+        const uint32_t gi = (uint32_t)ks & 1u;         // stage inside its group of two
+        if (!warp_wait(smem_u32(&ctl->group_full[gslot]), (uint32_t)((gidx / GROUPS) & 1), a.abort_flag, a.lane)) break;
+        const uint32_t src = stg0 + gslot * GROUP_BYTES;
+        const uint4 v0 = lds128u(src + (((2u * gi) ^ sw) << 4));
+        const uint4 v1 = lds128u(src + (((2u * gi + 1u) ^ sw) << 4));
+        const int s = it % A_STAGES;
+        if (!warp_wait(smem_u32(&ctl->empty_a[s]), (uint32_t)(((it / A_STAGES) & 1) ^ 1), a.abort_flag, a.lane)) break;
+        const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+        // 32-bit column 4c + t of the stage = word t of chunk c: the byte order of the
+        // K-major shared-memory layout of the other operand
+        uint32_t wr[32];
+        if (ragged && ks == a.nks - 1) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const int g = 8 * ks + c;   // index of the word in the row
+                const uint32_t valid = g < a.kw - 1 ? 0xFFFFFFFFu : (g == a.kw - 1 ? a.tmask : 0u);
+                const uint4 o = widen_masked(w[c], valid);
+                wr[4 * c] = o.x; wr[4 * c + 1] = o.y; wr[4 * c + 2] = o.z; wr[4 * c + 3] = o.w;
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint4 o = widen(w[c]);
+                wr[4 * c] = o.x; wr[4 * c + 1] = o.y; wr[4 * c + 2] = o.z; wr[4 * c + 3] = o.w;
+            }
+        }
+        tmem_st32(tdst0 + s * A_COLS, wr);
+        tmem_st_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (a.lane == 0) {
+            mbar_arrive(smem_u32(&ctl->full_a[s]));
+            // The staging slot is handed back only after the stores that consumed the loaded
+            // words: a shared-memory load that has merely been issued does not hold back the
+            // TMA write that refills the slot.  A group counts one arrival per warp and stage;
+            // the last group of a row with an odd number of stages holds a single stage, whose
+            // consumers arrive twice.
+            mbar_arrive(smem_u32(&ctl->group_empty[gslot]));
+            if (gi == 0 && ks == a.nks - 1) mbar_arrive(smem_u32(&ctl->group_empty[gslot]));
+        }
+        ks += TEAMS;
+        while (ks >= a.nks) { ks -= a.nks; ++tl; }
+    }
+}
+
+template <int BN>
+__global__ void __launch_bounds__(THREADS, 1)
+xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restrict__ img,
+                int M, int N, int K, const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
+                uint32_t* __restrict__ out_bits, int ldob, int* __restrict__ status) {
+    using C = Cfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Control* ctl = reinterpret_cast<Control*>(smem + B_REGION + GROUPS * GROUP_BYTES);
+    volatile int* abort_flag = &ctl->abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int kw = words_for(K);
+    const int nks = ceil_div(K, BK);
+    const int m_tiles = ceil_div(M, BM), n_tiles = ceil_div(N, BN);
+    const Share share = my_share(m_tiles, n_tiles);
+    const int nt = (int)blockIdx.x % n_tiles, n0 = nt * BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::A_STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full_a[s]), A_WARPS);
+            mbar_init(smem_u32(&ctl->empty_a[s]), 1);
+        }
+        for (int s = 0; s < MAX_NKS; ++s) mbar_init(smem_u32(&ctl->full_b[s]), 1);   // the copying thread (+ bytes)
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
+        }
+        for (int b = 0; b < GROUPS; ++b) {
+            mbar_init(smem_u32(&ctl->group_full[b]), 1);              // the issuing thread (+ bytes)
+            mbar_init(smem_u32(&ctl->group_empty[b]), 2 * A_WARPS);   // per stage of the group, every warp of its team
+        }
+        ctl->abort = 0;
+        mbar_init_fence();
+    }
+    if (warp == MMA_WARP) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ctl->tmem_base;
+    if (warp < EPI_WARPS) {
+        // Block scales of both operands: every byte 127, the ue8m0 code of 2^0.  The whole
+        // region is filled, so the values do not depend on how the scales are laid out in it.
+        uint32_t ones[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) ones[j] = 0x7F7F7F7Fu;
+        tmem_st32(tmem + ((uint32_t)(warp * 32) << 16) + C::TMEM_SF_COL, ones);
+        tmem_st_wait();
+        // thresholds of this CTA's units: the unit tile never changes
+        const int t = warp * 32 + lane;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int nl = t + h * 128, n = n0 + nl;
+            if (nl < BN) ctl->T[nl] = kMagicBits + (n < N ? thr[n] : 0);
+        }
+        if (t < BN / 32) {
+            const int wi = (n0 >> 5) + t;
+            ctl->flipw[t] = wi < words_for(N) ? flip[wi] : 0u;
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+
+    if (warp == TMA_WARP) {
+        // ---------------- one thread: the weight slice once, then the staging ring of frame rows
+        if (lane == 0 && share.count > 0) {
+            const uint32_t stg = smem_u32(smem) + B_REGION;
+            const int ng = ceil_div(nks, 2);
+            const int total_groups = share.count * ng;
+            int gc = 0;
+            auto load_group = [&](int g) {   // g: index in this CTA's sequence of groups, < GROUPS ahead of its consumers
+                const int slot = g % GROUPS;
+                const int m0 = (share.first + (g / ng) * share.step) * BM;
+                const uint32_t bar = smem_u32(&ctl->group_full[slot]);
+                mbar_arrive_expect_tx(bar, GROUP_BYTES);
+                tma_load_2d(stg + slot * GROUP_BYTES, &mapA, (g % ng) * 16, m0, bar);
+            };
+            for (; gc < GROUPS && gc < total_groups; ++gc) load_group(gc);   // frames first: they are small
+            const uint8_t* src = img + (size_t)n0 * 16;
+            const size_t run = (size_t)xnor_image_npad(N) * 16;   // bytes between chunks of the image
+            for (int ks = 0; ks < nks; ++ks) {
+                const uint32_t bar = smem_u32(&ctl->full_b[ks]);
+                mbar_arrive_expect_tx(bar, C::B_BYTES);
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    bulk_g2s(smem_u32(smem + ks * C::B_BYTES + c * (BN * 16)), src + (size_t)(ks * 8 + c) * run, BN * 16, bar);
+            }
+            for (; gc < total_groups; ++gc) {
+                if (!mbar_wait_relaxed(smem_u32(&ctl->group_empty[gc % GROUPS]), (uint32_t)(((gc / GROUPS) - 1) & 1), abort_flag)) break;
+                load_group(gc);
+            }
+        }
+        __syncwarp();
+    } else if (warp >= PROD_WARP0) {
+        ProducerArgs pa{smem_u32(smem) + B_REGION, tmem + C::TMEM_A_COL, ctl, abort_flag, share.count, nks, kw, tail_mask(K), lane};
+        produce_a<C::A_STAGES>(pa, (warp & 3) * 32 + lane, (warp - PROD_WARP0) / A_WARPS);
+    } else if (warp == MMA_WARP) {
+        // ---------------- MMA issue: one thread
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_mxf4(BM, BN);
+            const uint32_t sfa = tmem + C::TMEM_SF_COL, sfb = tmem + C::TMEM_SF_COL + SF_COLS / 2;
+            int it = 0;
+            bool ok = true;
+            for (int tl = 0; tl < share.count && ok; ++tl) {
+                const int b = tl & 1;
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), (uint32_t)(((tl >> 1) & 1) ^ 1), abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t d = tmem + (uint32_t)(b * BN);
+                for (int ks = 0; ks < nks; ++ks, ++it) {
+                    const int sa = it % C::A_STAGES;
+                    // the weight stage arrives once (phase 0) and then stays
+                    ok = (tl > 0 || mbar_wait(smem_u32(&ctl->full_b[ks]), 0u, abort_flag)) &&
+                         mbar_wait(smem_u32(&ctl->full_a[sa]), (uint32_t)((it / C::A_STAGES) & 1), abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t b0 = smem_u32(smem + ks * C::B_BYTES);
+                    const uint32_t ta = tmem + C::TMEM_A_COL + sa * A_COLS;
+#pragma unroll
+                    for (int j = 0; j < BK / 64; ++j) {   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
+                        const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (BN * 16), BN * 16, 128);
+                        mma_mxf4_ts(d, ta + 8 * j, db, idesc, sfa, sfb, (ks | j) != 0);
+                    }
+                    mma_commit(smem_u32(&ctl->empty_a[sa]));
+                }
+                if (ok) mma_commit(smem_u32(&ctl->acc_full[b]));
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue: 128 threads, thread = one frame (TMEM lane)
+        const int row_in_tile = warp * 32 + lane;
+        const float magic = __int_as_float(kMagicBits);
+        bool ok = true;
+        for (int tl = 0; tl < share.count && ok; ++tl) {
+            const int m0 = (share.first + tl * share.step) * BM;
+            const int m = m0 + row_in_tile;
+            const int b = tl & 1;
+            // all four epilogue warps take the same decision, so none is left at a barrier
+            ok = epi_all(warp_wait_relaxed(smem_u32(&ctl->acc_full[b]), (uint32_t)((tl >> 1) & 1), abort_flag, lane));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * BN);
+            uint32_t words[BN / 32];
+#pragma unroll
+            for (int g = 0; g < BN / 32; ++g) {
+                uint32_t acc[32];
+                tmem_ld32(taddr + g * 32, acc);
+                tmem_ld_wait();
+                // The accumulator holds the integer dot product as a float; adding 1.5 * 2^23
+                // leaves that integer, offset by kMagicBits, in the bit pattern of the sum.
+                // bit = (dot - thr >= 0); the sign bits are shifted in from the top, element 31
+                // first, so element j ends up in bit j, inverted.
+                uint32_t wd = 0u;
+#pragma unroll
+                for (int j = 31; j >= 0; --j)
+                    wd = __funnelshift_l((uint32_t)(__float_as_int(__uint_as_float(acc[j]) + magic) - ctl->T[g * 32 + j]), wd, 1);
+                words[g] = ~wd ^ ctl->flipw[g];
+                const int valid = N - (n0 + g * 32);  // columns of this word that exist
+                if (valid < 32) words[g] = valid > 0 ? (words[g] & ((1u << valid) - 1u)) : 0u;
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+            if (m < M) {
+                const int nw = words_for(N), w0 = n0 >> 5;
+                uint32_t* dst = out_bits + (size_t)m * ldob + w0;
+                if (w0 + BN / 32 <= nw) {   // rows are 16-byte aligned and BN/32 is even: 8-byte stores
+#pragma unroll
+                    for (int i = 0; i < BN / 64; ++i)
+                        reinterpret_cast<uint2*>(dst)[i] = make_uint2(words[2 * i], words[2 * i + 1]);
+                } else {
+#pragma unroll
+                    for (int g = 0; g < BN / 32; ++g)
+                        if (w0 + g < nw) dst[g] = words[g];
+                }
+            }
+        }
+    }
+
+    // ---------------- teardown: every thread arrives here, also after an aborted wait
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == MMA_WARP) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
+    if (threadIdx.x == 0 && ctl->abort) atomicExch(status, 1);
+}
+
+template <int BN>
+int launch_bn(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
+              const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int sm_count, cudaStream_t st) {
+    auto kern = xnor_res_kernel<BN>;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return BNN_ERR_CUDA;
+        configured = true;
+    }
+    const long long tiles = (long long)ceil_div(M, BM) * ceil_div(N, BN);
+    const int grid = tiles < sm_count ? (int)tiles : sm_count;
+    int* status = tc_status_ptr();
+    if (!status) return BNN_ERR_CUDA;
+    CUtensorMap mapA;
+    if (!encode_packed_map(&mapA, Ap, ldap, M, K, BM)) return BNN_ERR_CUDA;
+    kern<<<grid, THREADS, SMEM_BYTES, st>>>(mapA, static_cast<const uint8_t*>(image), M, N, K, thr, flip, out_bits, ldob, status);
+    return launch_status();
+}
+
+}  // namespace
+
+// Units per tile for a layer of this shape, or 0 when the kernel does not apply: the slice of
+// a tile must fit the shared-memory region, and every unit tile needs a CTA of its own.
+static int tile_units(int N, int K, int sm_count) {
+    const int nks = ceil_div(K, BK);
+    const int bn = nks <= Cfg<192>::NKS ? 192 : (nks <= Cfg<128>::NKS ? 128 : 0);
+    if (bn == 0 || ceil_div(N, bn) > sm_count) return 0;
+    return bn;
+}
+
+static int sm_count_of_device() {
+    static int sm_count = 0;
+    if (!sm_count) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            sm_count = 0;
+    }
+    return sm_count;
+}
+
+bool xnor_res_applicable(int N, int K) {
+    const int sms = sm_count_of_device();
+    return sms > 0 && tile_units(N, K, sms) != 0;
+}
+
+int launch_xnor_res(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
+                    const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, cudaStream_t st) {
+    const int sms = sm_count_of_device();
+    if (sms <= 0) return BNN_ERR_CUDA;
+    const int bn = tile_units(N, K, sms);
+    if (bn == 192) return launch_bn<192>(Ap, ldap, image, M, N, K, thr, flip, out_bits, ldob, sms, st);
+    if (bn == 128) return launch_bn<128>(Ap, ldap, image, M, N, K, thr, flip, out_bits, ldob, sms, st);
+    return BNN_ERR_UNSUPPORTED;
+}
+
+}  // namespace bnn

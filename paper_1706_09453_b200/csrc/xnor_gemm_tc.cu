@@ -32,6 +32,7 @@
 // through to the common teardown and the device status word is set.
 #include "bnn_common.cuh"
 #include "tcgen05.cuh"
+#include "xnor_widen.cuh"
 
 namespace bnn {
 
@@ -54,7 +55,6 @@ constexpr uint32_t TMEM_A_COL = 2 * BN;                   // A stages start afte
 constexpr uint32_t A_COLS = ROW_BYTES / 4;                // 32-bit columns per A stage
 constexpr uint32_t TMEM_SF_COL = TMEM_A_COL + A_STAGES * A_COLS, SF_COLS = 32;   // block scales: 16 columns per operand
 constexpr uint32_t TMEM_COLS = 512;
-constexpr int kMagicBits = 0x4B400000;                    // bits of 1.5 * 2^23: x + magic has the integer x in its low bits
 
 // With int32 output each epilogue warp needs two staging blocks of 32 rows x 128 bytes.
 template <bool STORE_C> struct Cfg {
@@ -85,21 +85,6 @@ struct ProducerArgs {
     uint32_t tmask;
     int lane;
 };
-
-// Four output words of one input word: nibble i of word t <- bit 4i + t.
-__device__ __forceinline__ uint4 widen(uint32_t w) {
-    return make_uint4(((w << 3) & 0x88888888u) ^ 0xAAAAAAAAu, ((w << 2) & 0x88888888u) ^ 0xAAAAAAAAu,
-                      ((w << 1) & 0x88888888u) ^ 0xAAAAAAAAu, (w & 0x88888888u) ^ 0xAAAAAAAAu);
-}
-// The same with the nibbles of invalid positions (bit of `valid` clear) set to +0.
-__device__ __forceinline__ uint4 widen_masked(uint32_t w, uint32_t valid) {
-    uint4 o = widen(w);
-    o.x &= (valid & 0x11111111u) * 15u;
-    o.y &= ((valid >> 1) & 0x11111111u) * 15u;
-    o.z &= ((valid >> 2) & 0x11111111u) * 15u;
-    o.w &= ((valid >> 3) & 0x11111111u) * 15u;
-    return o;
-}
 
 // The eight 16-byte chunks of one widened row and stage; `ks` is the stage's index in the row.
 __device__ __forceinline__ void widen_stage(const ProducerArgs& a, bool ragged, int ks, const uint4& v0, const uint4& v1, uint4 (&o)[8]) {

@@ -26,10 +26,10 @@ def words_to_numpy(t: torch.Tensor, k: int) -> np.ndarray:
 
 
 class DeviceNet:
-    def __init__(self, net: wl.Model, sign_mode=B.SIGN_ZERO_POS, device="cuda:0"):
+    def __init__(self, net: wl.Model, sign_mode=B.SIGN_ZERO_POS, device="cuda:0", prepare_xnor=True):
         cfg = net.cfg
         self.cfg, self.sign_mode, self.device = cfg, sign_mode, device
-        self.Wp, self.scale, self.shift, self.thr, self.flip = [], [], [], [], []
+        self.Wp, self.scale, self.shift, self.thr, self.flip, self.Wimg = [], [], [], [], [], []
         layers = []
         binary_act = cfg.act == wl.ACT_SIGN
         for l, w in enumerate(net.W):
@@ -49,7 +49,12 @@ class DeviceNet:
                 flip = torch.empty((n + 31) // 32, dtype=torch.int32, device=device)
                 B.bnn_fold_thresholds(sc, sh, n, k, thr, flip, sign_mode)
                 self.thr.append(thr); self.flip.append(flip)
-                layers.append(dict(kind=B.LAYER_XNOR, K=k, N=n, Wp=wp, thr=thr, flip=flip,
+                img = None
+                if prepare_xnor:   # widened image of the weights for the tensor cores (built once)
+                    img = torch.empty(B.bnn_xnor_prepared_bytes(n, k), dtype=torch.uint8, device=device)
+                    B.bnn_xnor_prepare(wp, k, img)
+                self.Wimg.append(img)
+                layers.append(dict(kind=B.LAYER_XNOR, K=k, N=n, Wp=wp, thr=thr, flip=flip, W_prepared=img,
                                    act=B.ACT_SIGN_PACK))
         self.Wout, self.bout = to_dev(net.Wout, device), to_dev(net.bout, device)
         self.Wout_prepared = torch.empty(B.bnn_output_prepared_bytes(cfg.classes, cfg.hidden),

@@ -74,6 +74,20 @@ def test_bad_arguments_are_rejected_without_a_launch(lib):
     assert rc("bnn_output_prepare", fake, 4, 1, 4, None, 1 << 20, None) == 1
     assert rc("bnn_output_prepare", fake, 4, 1, 4, fake, 16, None) == 5
     assert B.bnn_output_prepared_bytes(3400, 2048) == 27 * 64 * 16384 + 27 * 128 * 4
+    # prepared weights of a binary layer
+    assert B.bnn_xnor_prepared_bytes(2048, 2048) == 8 * 2304 * 128
+    assert B.bnn_xnor_prepared_bytes(1, 1) == 384 * 128
+    assert B.bnn_xnor_prepared_bytes(4, (1 << 22) + 1) == 0
+    assert rc("bnn_xnor_prepare", fake, 4, 4, 32, None, 1 << 20, None) == 1
+    assert rc("bnn_xnor_prepare", None, 4, 4, 32, fake, 1 << 20, None) == 1
+    assert rc("bnn_xnor_prepare", fake, 4, 0, 32, fake, 1 << 20, None) == 2
+    assert rc("bnn_xnor_prepare", fake, 4, 4, 32, fake, 100, None) == 5
+    assert rc("bnn_xnor_prepare", fake, 4, 4, 32, fake + 16, 1 << 20, None) == 3
+    assert rc("bnn_xnor_prepare", fake, 1 << 18, 4, (1 << 22) + 1, fake, 1 << 30, None) == 4
+    assert rc("bnn_xnor_gemm_prepared", fake, 4, None, 1, 1, 32, fake, 1, None, None) == 1
+    assert rc("bnn_xnor_gemm_prepared", fake, 4, fake + 16, 1, 1, 32, fake, 1, None, None) == 3
+    assert rc("bnn_xnor_gemm_prepared", fake, 4, fake, 1, 1, 32, None, 0, None, None) == 1
+    assert rc("bnn_xnor_gemm_prepared", fake, 4, fake, 1, 40, 32, fake, 8, None, None) == 2
     # options
     assert B.bnn_set_option(B.OPT_XNOR_PATH, B.PATH_CUDA_CORE) == 0
     assert B.bnn_set_option(B.OPT_XNOR_PATH, B.PATH_AUTO) == 1

@@ -27,12 +27,12 @@ def env():
     return torch, binding, model
 
 
-def run_binary_net(env, cfg, frames, mode=0, sample=None):
+def run_binary_net(env, cfg, frames, mode=0, sample=None, prepare_xnor=True):
     """Runs bnn_forward on `frames` frames; compares the frames in `sample` (all if None)."""
     torch, B, model = env
     net = wl.make_model(cfg)
     X = wl.make_frames(cfg, frames)
-    dn = model.DeviceNet(net, mode)
+    dn = model.DeviceNet(net, mode, prepare_xnor=prepare_xnor)
     outs = dn.layer_out_buffers(frames)
     logp = dn.forward(model.to_dev(X), layer_out=outs)
     torch.cuda.synchronize()
@@ -65,6 +65,11 @@ def test_forward_tiny_config_all_frames(env):
     r = run_binary_net(env, wl.CONFIGS["tiny"], 256)
     assert r["flipped"] <= r["ambiguous"]
     assert env[1].bnn_device_status() == 0
+
+
+def test_forward_tiny_config_weights_widened_on_the_fly(env):
+    """The model without prepared images of the hidden layers' weights (bnn_xnor_gemm's kernel)."""
+    run_binary_net(env, wl.CONFIGS["tiny"], 256, prepare_xnor=False)
 
 
 def test_forward_tiny_config_popcount_path(env):

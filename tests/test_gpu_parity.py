@@ -29,13 +29,27 @@ def torch_():
     return torch
 
 
-@pytest.fixture(params=["popc", "tensor"])
+@pytest.fixture(params=["popc", "tensor", "prepared"])
 def xnor_path(request, B):
-    """Runs a test once per XNOR kernel (integer-pipe popcount, tcgen05 tensor core)."""
+    """Runs a test once per XNOR kernel: integer-pipe popcount, tcgen05 tensor core widening both
+    operands on the fly, tcgen05 with the weights widened once (bnn_xnor_prepare)."""
     prev = B.bnn_set_xnor_path(B.XNOR_POPC if request.param == "popc" else B.XNOR_TENSOR)
     yield request.param
     B.bnn_set_xnor_path(prev)
     assert B.bnn_device_status() == 0, "a tensor-core kernel gave up on a bounded wait"
+
+
+def run_xnor(B, path, a_dev, w_dev, k, image=None, **kw):
+    """bnn_xnor_gemm, or (path "prepared") bnn_xnor_prepare + bnn_xnor_gemm_prepared."""
+    if path != "prepared":
+        return B.bnn_xnor_gemm(a_dev, w_dev, k, **kw)
+    import torch
+    n = w_dev.shape[0]
+    if image is None:
+        image = torch.full((B.bnn_xnor_prepared_bytes(n, k),), 0x5A, dtype=torch.uint8, device="cuda:0")
+        B.bnn_xnor_prepare(w_dev, k, image)
+    B.bnn_xnor_gemm_prepared(a_dev, image, n, k, **kw)
+    return image
 
 
 @pytest.fixture(params=["fp32", "tensor", "tensor_ws"])
@@ -153,7 +167,7 @@ def test_xnor_gemm_int32_bit_exact(B, torch_, xnor_path, shape, p):
     ap = wl.make_bit_planes(m, k, p, [1, m, n, k], B.packed_pitch(k))
     wp = wl.make_bit_planes(n, k, p, [2, m, n, k], B.packed_pitch(k))
     c = torch_.full((m, n + 5), -77, dtype=torch_.int32, device="cuda:0")
-    B.bnn_xnor_gemm(dev(ap), dev(wp), k, C_out=c[:, :n])
+    run_xnor(B, xnor_path, dev(ap), dev(wp), k, C_out=c[:, :n])
     got = c.cpu().numpy()
     np.testing.assert_array_equal(got[:, :n], o.xnor_gemm(ap, wp, k))
     np.testing.assert_array_equal(got[:, n:], -77)
@@ -173,12 +187,12 @@ def test_xnor_gemm_ignores_garbage_in_pad_bits(B, torch_, xnor_path):
     ap2[:, kw - 1] |= np.uint32(0xFFFFFFFF << (k % 32) & 0xFFFFFFFF)
     wp2[:, kw - 1] |= rng.integers(0, 2**32, n, dtype=np.uint32) & np.uint32(0xFFFFFFFF << (k % 32) & 0xFFFFFFFF)
     c = torch_.empty((m, n), dtype=torch_.int32, device="cuda:0")
-    B.bnn_xnor_gemm(dev(ap2), dev(wp2), k, C_out=c)
+    run_xnor(B, xnor_path, dev(ap2), dev(wp2), k, C_out=c)
     np.testing.assert_array_equal(c.cpu().numpy(), want)
 
 
 @pytest.mark.parametrize("shape", [(5, 7, 33), (129, 130, 127), (300, 257, 1000), (256, 1024, 1024), (131, 96, 440),
-                                   (19100, 300, 160)])
+                                   (19100, 300, 160), (300, 260, 3000), (150, 200, 5000), (2000, 3072, 2100)])
 @pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("with_c", [False, True])
 def test_xnor_gemm_fused_sign_pack_bit_exact(B, torch_, xnor_path, shape, mode, with_c):
@@ -197,7 +211,7 @@ def test_xnor_gemm_fused_sign_pack_bit_exact(B, torch_, xnor_path, shape, mode, 
     B.bnn_fold_thresholds(dev(scale), dev(shift), n, k, thr, flip, mode)
     out = packed_canary(torch_, m, n, B)
     c = torch_.empty((m, n), dtype=torch_.int32, device="cuda:0") if with_c else None
-    B.bnn_xnor_gemm(dev(ap), dev(wp), k, C_out=c, thr=thr, flip=flip, out_bits=out[:, :B.packed_pitch(n)])
+    run_xnor(B, xnor_path, dev(ap), dev(wp), k, C_out=c, thr=thr, flip=flip, out_bits=out[:, :B.packed_pitch(n)])
     d = o.xnor_gemm(ap, wp, k)
     want = o.affine_sign_pack_i32(d, scale, shift, mode)
     got = out.cpu().numpy().view(np.uint32)
@@ -210,8 +224,9 @@ def test_xnor_gemm_fused_sign_pack_bit_exact(B, torch_, xnor_path, shape, mode, 
         assert (d[:, 2::5].astype(np.float32) + shift[2::5] == 0).any(), "no exact zero was exercised"
 
 
+@pytest.mark.parametrize("path", ["tensor", "prepared"])
 @pytest.mark.parametrize("shape", [(8192, 2048, 2048), (16384, 2048, 2048)])
-def test_xnor_gemm_full_size_every_output_on_repeated_launches(B, torch_, shape):
+def test_xnor_gemm_full_size_every_output_on_repeated_launches(B, torch_, shape, path):
     """A hidden layer at full size, every output bit compared with the oracle, on many launches in
     a row: a hand-off between the kernel's roles that is wrong once in ten thousand tiles only
     shows on a run of this length (sampled outputs would miss it)."""
@@ -233,14 +248,15 @@ def test_xnor_gemm_full_size_every_output_on_repeated_launches(B, torch_, shape)
         out = torch_.zeros((m, B.packed_pitch(n)), dtype=torch_.int32, device="cuda:0")
         c = torch_.zeros((m, n), dtype=torch_.int32, device="cuda:0")
         nw = (n + 31) // 32
+        image = None
         for launch in range(40):
             out.zero_()
-            B.bnn_xnor_gemm(a_dev, w_dev, k, thr=thr, flip=flip, out_bits=out)
+            image = run_xnor(B, path, a_dev, w_dev, k, image=image, thr=thr, flip=flip, out_bits=out)
             bad = int((out[:, :nw] != want_bits).sum().item())
             assert bad == 0, "launch %d (fused Sign): %d packed words differ" % (launch, bad)
         for launch in range(20):
             c.zero_()
-            B.bnn_xnor_gemm(a_dev, w_dev, k, C_out=c)
+            run_xnor(B, path, a_dev, w_dev, k, image=image, C_out=c)
             bad = int((c != want_c).sum().item())
             assert bad == 0, "launch %d (int32 output): %d outputs differ" % (launch, bad)
     finally:
