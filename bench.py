@@ -39,6 +39,10 @@ def parse_args():
     ap.add_argument("--frames", type=int, default=None, help="override the batch size (frames per step)")
     ap.add_argument("--cpu-frames", type=int, default=16384, help="frames of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--xnor-prepared", default="auto", choices=["auto", "stream", "resident"],
+                    help="kernel for hidden layers with prepared weights (see BNN_OPT_XNOR_PREPARED)")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="launch every step's kernels from the host instead of replaying a captured CUDA graph")
     ap.add_argument("--sweep", action="store_true",
                     help="isolated XNOR GEMM sweep (M x K x N x bit density), one JSON line per point")
     ap.add_argument("--sweep-quick", action="store_true", help="only the corner points of the sweep")
@@ -161,7 +165,20 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ roofline bookkeeping
-def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tensor"):
+def xnor_kernel_name(k, xnor_path, prepared):
+    """The kernel bnn_forward runs for a binary hidden layer of fan-in k (see bnn_api.cu)."""
+    if xnor_path == "popc":
+        return "xnor_popc_kernel"
+    if xnor_path == "tensor-unprepared":
+        return "xnor_tc_kernel"
+    if prepared == "stream":
+        return "xnor_img_kernel"
+    if k <= 2048 or (prepared == "resident" and k <= 3072):
+        return "xnor_res_kernel"
+    return "xnor_tc_kernel"
+
+
+def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tensor", prepared="auto"):
     """Per layer: algorithmic work, the pipe that bounds the kernel and its peak.
 
     Algorithmic work: 2 binary ops per bit-MAC for XNOR layers, 2 flop per add/sub or MAC for
@@ -187,12 +204,17 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
             tiles_m, tiles_n = -(-frames // 128), -(-cfg.hidden // 192)
             kpad = -(-k // 256) * 256
             smem_bytes = tiles_m * tiles_n * kpad * (192 * (0.5 + 0.5 + 0.125 + 0.125) + 128 * (0.125 + 0.125))
-            if xnor_path == "tensor":
+            kern = xnor_kernel_name(k, xnor_path, prepared)
+            if kern == "xnor_img_kernel":
                 # weights prepared once: their widened image arrives by bulk copies (4 bits written,
                 # 4 bits read by the tensor core per weight bit and tile visit); nothing else
                 smem_bytes = tiles_m * tiles_n * kpad * (192 * (0.5 + 0.5) + 128 * (0.125 + 0.125))
-            rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_img_kernel" if xnor_path == "tensor" else "xnor_tc_kernel",
-                             work=work, unit="Tbop/s",
+            elif kern == "xnor_res_kernel":
+                # weights resident: written once per CTA, read by the tensor core on every tile visit
+                bn = 192 if k <= 2048 else 128
+                tiles_n = -(-cfg.hidden // bn)
+                smem_bytes = tiles_m * tiles_n * kpad * (bn * 0.5 + 128 * (0.125 + 0.125)) + SMS * kpad * bn * 0.5
+            rows.append(dict(name="xnor_%d" % (l + 1), kernel=kern, work=work, unit="Tbop/s",
                              bound="tensor", peak=4.0 * peaks["bf16_tflops_sustained"], smem_bytes=smem_bytes))
         elif xnor:
             rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_popc_kernel", work=work, unit="Tbop/s",
@@ -268,6 +290,7 @@ def run_ours(args):
     net = wl.make_model(cfg)
     B.bnn_set_xnor_path(B.XNOR_POPC if args.xnor_path == "popc" else B.XNOR_TENSOR)
     B.bnn_set_option(B.OPT_REAL_PATH, B.PATH_TENSOR if args.real_path == "tensor" else B.PATH_CUDA_CORE)
+    B.bnn_set_option(B.OPT_XNOR_PREPARED, {"auto": 0, "stream": 1, "resident": 2}[args.xnor_prepared])
     dn = model.DeviceNet(net, device=dev, prepare_xnor=args.xnor_path == "tensor")
     # Frames are independent, so ranks shard them with no exchange: each rank owns its own batch.
     Xh = wl.make_frames(cfg, frames, seed=D.frames_seed(cfg.seed, rank))
@@ -289,13 +312,38 @@ def run_ours(args):
 
     for i in range(W):
         step(i)
+    # bnn_forward only enqueues kernels on the caller's stream, so a caller can capture it: one
+    # CUDA graph per buffer set (one bnn_forward each), replayed in turn.  The device then starts
+    # each kernel of a step without a host launch in between.
+    graphs = None
+    if not args.no_graph:
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream(dev)
+        side.wait_stream(torch.cuda.current_stream())
+        graphs = []
+        with torch.cuda.stream(side):
+            for b in range(nsets):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    step(b)
+                graphs.append(g)
+        torch.cuda.current_stream().wait_stream(side)
+        for b in range(min(nsets, W)):
+            graphs[b].replay()
+
+    def timed_step(i):
+        if graphs:
+            graphs[i % nsets].replay()
+        else:
+            step(i)
+
     clocks = ClockSampler(torch, local)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     clocks.start()
     e0.record()
     for i in range(K):
-        step(i)
+        timed_step(i)
     e1.record()
     barrier()
     clocks.stop()
@@ -370,7 +418,7 @@ def run_ours(args):
 
     peaks = load_peaks()
     ck = clocks.summary()
-    rows = layer_table(cfg, frames, peaks, ck.get("sm_mhz"), args.xnor_path, args.real_path)
+    rows = layer_table(cfg, frames, peaks, ck.get("sm_mhz"), args.xnor_path, args.real_path, args.xnor_prepared)
     assert len(rows) == len(layer_ms)
     for r, t in zip(rows, layer_ms):
         r["ms"] = t
@@ -394,7 +442,7 @@ def run_ours(args):
                 "frac": achieved / dom["peak"], "traffic": ncu_traffic(dk),
                 "peak_source": ("4 x bf16_tflops_sustained of MEASURED_PEAKS.json (%s): e2m1 (mxf4) MMA = 4 x bf16 (nominal ratio), "
                                 "sustained figure because the kernel is timed inside a long step; of measured"
-                                % peaks["source"]) if dk in ("xnor_tc_kernel", "xnor_img_kernel") else
+                                % peaks["source"]) if dk in ("xnor_tc_kernel", "xnor_img_kernel", "xnor_res_kernel") else
                                ("bf16_tflops_sustained of MEASURED_PEAKS.json (%s); of measured" % peaks["source"])
                                if dom["bound"] == "tensor" else
                                ("hbm_gbs of MEASURED_PEAKS.json (%s); of measured" % peaks["source"])
@@ -423,7 +471,7 @@ def run_ours(args):
                     "split bf16/fp16 tensor-core MMA, f32 accumulate" if args.real_path == "tensor" else "f32"),
         "device_status": B.bnn_device_status(), "data": "synthetic",
         "config": {"workload": workload_name(cfg, frames), "frames_per_gpu": frames,
-                   "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 2 x L2); weights stay hot"
+                   "launch": "host launches" if args.no_graph else "one captured CUDA graph per step (a single bnn_forward call each)", "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 2 x L2); weights stay hot"
                          % (nsets, nsets * set_bytes / 1e6),
                    "sign_zero": "+1", "seed": cfg.seed},
         "clocks": ck,

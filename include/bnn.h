@@ -288,9 +288,16 @@ BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, 
  *                        tcgen05 with split bf16/fp16 operands.  AUTO = TENSOR.
  *   BNN_OPT_SIGNW_TERMS: 2 (default) or 3 bf16 terms for the real operand of bnn_signw_gemm
  *                        on the tensor path: |error| <= 2^-17 sum|x_i| with 2, fp32-exact
- *                        products with 3. */
-typedef enum { BNN_OPT_XNOR_PATH = 0, BNN_OPT_REAL_PATH = 1, BNN_OPT_SIGNW_TERMS = 2 } bnn_option;
+ *                        products with 3.
+ *   BNN_OPT_XNOR_PREPARED: which kernel bnn_xnor_gemm_prepared (and bnn_forward on prepared
+ *                        layers) runs for a fused Sign layer: BNN_PREPARED_STREAM reads the
+ *                        weight image from L2 for every tile of frames; BNN_PREPARED_RESIDENT
+ *                        keeps a tile of units' weights in shared memory for the whole launch
+ *                        (needs K <= 3072; other shapes stream); AUTO picks by shape. */
+typedef enum { BNN_OPT_XNOR_PATH = 0, BNN_OPT_REAL_PATH = 1, BNN_OPT_SIGNW_TERMS = 2,
+               BNN_OPT_XNOR_PREPARED = 3 } bnn_option;
 typedef enum { BNN_PATH_AUTO = 0, BNN_PATH_CUDA_CORE = 1, BNN_PATH_TENSOR = 2 } bnn_path;
+typedef enum { BNN_PREPARED_AUTO = 0, BNN_PREPARED_STREAM = 1, BNN_PREPARED_RESIDENT = 2 } bnn_prepared_kernel;
 BNN_API int bnn_set_option(int option, int value);
 
 /* Tensor-core kernels bound every wait they perform; a CTA whose wait runs out stops, frees

@@ -10,6 +10,7 @@ namespace {
 constexpr int kMaxK = 1 << 24;
 int g_xnor_path = BNN_PATH_AUTO;
 int g_real_path = BNN_PATH_AUTO;
+int g_xnor_prepared = BNN_PREPARED_AUTO;
 int g_signw_terms = 2;  // |dot| <= K stays exact in every accumulator type used
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
@@ -100,10 +101,13 @@ int bnn_set_option(int option, int value) {
         case BNN_OPT_XNOR_PATH: slot = &g_xnor_path; break;
         case BNN_OPT_REAL_PATH: slot = &g_real_path; break;
         case BNN_OPT_SIGNW_TERMS: slot = &g_signw_terms; break;
+        case BNN_OPT_XNOR_PREPARED: slot = &g_xnor_prepared; break;
         default: return -1;
     }
     if (option == BNN_OPT_SIGNW_TERMS) {
         if (value != 2 && value != 3) return -1;
+    } else if (option == BNN_OPT_XNOR_PREPARED) {
+        if (value != BNN_PREPARED_AUTO && value != BNN_PREPARED_STREAM && value != BNN_PREPARED_RESIDENT) return -1;
     } else if (value != BNN_PATH_AUTO && value != BNN_PATH_CUDA_CORE && value != BNN_PATH_TENSOR) {
         return -1;
     }
@@ -148,7 +152,8 @@ int bnn_fold_thresholds(const float* scale, const float* shift, int N, int K, in
     return launch_fold_thresholds(scale, shift, N, K, sign_mode, thr, flip, (cudaStream_t)stream);
 }
 
-// Shared by bnn_xnor_gemm (image == nullptr) and bnn_xnor_gemm_prepared (Wp == nullptr).
+// Shared by bnn_xnor_gemm (image == nullptr), bnn_xnor_gemm_prepared (Wp == nullptr) and
+// bnn_forward (both, when the layer has an image).
 static int xnor_gemm_impl(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, const void* image,
                           int M, int N, int K, int32_t* C, int ldc,
                           const bnn_epilogue* epi, void* stream) {
@@ -158,9 +163,9 @@ static int xnor_gemm_impl(const uint32_t* Ap, int ldap, const uint32_t* Wp, int 
     if (image) {
         if (K > kMaxKTensor) return BNN_ERR_UNSUPPORTED;
         if (reinterpret_cast<uintptr_t>(image) & 255u) return BNN_ERR_ALIGN;
-    } else if (int rc = check_packed(Wp, ldwp, K)) {
-        return rc;
     }
+    if (Wp || !image)
+        if (int rc = check_packed(Wp, ldwp, K)) return rc;
     if (C && ldc < N) return BNN_ERR_SHAPE;
     const int32_t* thr = nullptr;
     const uint32_t* flip = nullptr;
@@ -174,11 +179,17 @@ static int xnor_gemm_impl(const uint32_t* Ap, int ldap, const uint32_t* Wp, int 
     }
     if (!C && !ob) return BNN_ERR_NULL;
     if (image) {
-        // fused Sign layer: the kernel that keeps a unit tile's weights in shared memory, when
-        // they fit; int32 output and the remaining shapes: the kernel that streams the image
-        if (!C && xnor_res_applicable(N, K))
+        // Fused Sign layer: the kernel that keeps a unit tile's weights in shared memory where
+        // measurement favours it (K <= 2048, tiles of 192 units; with K <= 3072 its tiles shrink
+        // to 128 units and the kernel that widens packed weights on the fly is faster, so that
+        // one runs when the packed weights are at hand).  int32 output and the remaining shapes:
+        // the kernel that streams the image.
+        const bool fused = !C && g_xnor_prepared != BNN_PREPARED_STREAM && xnor_res_applicable(N, K);
+        const bool wide_tiles = K <= 2048;
+        if (fused && (wide_tiles || !Wp || g_xnor_prepared == BNN_PREPARED_RESIDENT))
             return launch_xnor_res(Ap, ldap, image, M, N, K, thr, flip, ob, ldob, (cudaStream_t)stream);
-        return launch_xnor_img(Ap, ldap, image, M, N, K, C, ldc, thr, flip, ob, ldob, (cudaStream_t)stream);
+        if (!Wp || g_xnor_prepared == BNN_PREPARED_STREAM)
+            return launch_xnor_img(Ap, ldap, image, M, N, K, C, ldc, thr, flip, ob, ldob, (cudaStream_t)stream);
     }
     const bool tensor = g_xnor_path != BNN_PATH_CUDA_CORE && K <= kMaxKTensor;
     return (tensor ? launch_xnor_tc : launch_xnor_popc)(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip,
