@@ -9,7 +9,8 @@
  * never be called from the product path.  All pointers are HOST pointers.
  *
  * Conventions (the paper fixes none for storage; these are this project's):
- *   bit = 1 <=> +1, bit = 0 <=> -1; element k of a row is bit k%32 of 32-bit word k/32;
+ *   bit = 1 <=> +1, bit = 0 <=> -1 (activations of a (0,1) network: bit = the value itself);
+ *   element k of a row is bit k%32 of 32-bit word k/32;
  *   bits at positions >= K are zero.  Row pitches (ld*) are in elements of the array type.
  *
  * Build: gcc -O2 -fopenmp -ffp-contract=off -fPIC -shared bnn_oracle.c -o libbnn_oracle.so -lm
@@ -64,6 +65,36 @@ void oracle_unpack_pm1(const uint32_t* P, long ldp, long M, long K, int8_t* S) {
     for (long m = 0; m < M; ++m)
         for (long k = 0; k < K; ++k)
             S[m * K + k] = ((P[m * ldp + k / 32] >> (k % 32)) & 1u) ? 1 : -1;
+}
+
+/* Decode a packed plane to (0,1) values: the binary pair the paper compares with (-1,+1)
+ * for activations (Section 3.2, Table 3; Section 3.3, Table 4). */
+void oracle_unpack_01(const uint32_t* P, long ldp, long M, long K, int8_t* S) {
+    for (long m = 0; m < M; ++m)
+        for (long k = 0; k < K; ++k)
+            S[m * K + k] = (int8_t)((P[m * ldp + k / 32] >> (k % 32)) & 1u);
+}
+
+/*
+ * Binary weights in {-1,+1} against binary activations in {0,1} (Section 3.2: "(0,1) for
+ * binary activations"): d[m][n] = sum_k h[m][k] * w[n][k].  Exact integer arithmetic.
+ */
+void oracle_gemm01(const uint32_t* Hp, long ldhp, const uint32_t* Wp, long ldwp,
+                   long M, long N, long K, int32_t* D, long ldd) {
+    int8_t* h = (int8_t*)malloc((size_t)M * K);
+    int8_t* w = (int8_t*)malloc((size_t)N * K);
+    oracle_unpack_01(Hp, ldhp, M, K, h);
+    oracle_unpack_pm1(Wp, ldwp, N, K, w);
+#pragma omp parallel for schedule(static)
+    for (long m = 0; m < M; ++m) {
+        for (long n = 0; n < N; ++n) {
+            int32_t s = 0;
+            for (long k = 0; k < K; ++k) s += (int32_t)h[m * K + k] * (int32_t)w[n * K + k];
+            D[m * ldd + n] = s;
+        }
+    }
+    free(h);
+    free(w);
 }
 
 /*
@@ -172,6 +203,22 @@ void oracle_real_gemm_bits(const uint32_t* Hp, long ldhp, const float* Wout, lon
                            const float* b, long M, long C, long H, double* Z, long ldz) {
     int8_t* h = (int8_t*)malloc((size_t)M * H);
     oracle_unpack_pm1(Hp, ldhp, M, H, h);
+#pragma omp parallel for schedule(static)
+    for (long m = 0; m < M; ++m) {
+        for (long c = 0; c < C; ++c) {
+            double s = 0.0;
+            for (long n = 0; n < H; ++n) s += (double)Wout[c * ldw + n] * (double)h[m * H + n];
+            Z[m * ldz + c] = s + (b ? (double)b[c] : 0.0);
+        }
+    }
+    free(h);
+}
+
+/* The same top layer on (0,1) activations given as bits (Section 3.2). */
+void oracle_real_gemm_bits01(const uint32_t* Hp, long ldhp, const float* Wout, long ldw,
+                             const float* b, long M, long C, long H, double* Z, long ldz) {
+    int8_t* h = (int8_t*)malloc((size_t)M * H);
+    oracle_unpack_01(Hp, ldhp, M, H, h);
 #pragma omp parallel for schedule(static)
     for (long m = 0; m < M; ++m) {
         for (long c = 0; c < C; ++c) {

@@ -87,6 +87,28 @@ def unpack_pm1(P, K):
     return S
 
 
+VALUES_PM1, VALUES_01 = 0, 1   # what the bits of a binary ACTIVATION stand for
+
+
+def unpack_01(P, K):
+    P = np.ascontiguousarray(P, dtype=np.uint32)
+    M, ldp = P.shape
+    S = np.empty((M, K), dtype=np.int8)
+    lib().oracle_unpack_01(_p(P), _L(ldp), _L(M), _L(K), _p(S))
+    return S
+
+
+def gemm01(Hp, Wp, K):
+    """d = sum_k h*w with h in {0,1} (bits of Hp) and w in {-1,+1} (bits of Wp)."""
+    Hp = np.ascontiguousarray(Hp, dtype=np.uint32)
+    Wp = np.ascontiguousarray(Wp, dtype=np.uint32)
+    M, N = Hp.shape[0], Wp.shape[0]
+    D = np.empty((M, N), dtype=np.int32)
+    lib().oracle_gemm01(_p(Hp), _L(Hp.shape[1]), _p(Wp), _L(Wp.shape[1]),
+                        _L(M), _L(N), _L(K), _p(D), _L(N))
+    return D
+
+
 def xnor_gemm(Ap, Wp, K):
     Ap = np.ascontiguousarray(Ap, dtype=np.uint32)
     Wp = np.ascontiguousarray(Wp, dtype=np.uint32)
@@ -150,6 +172,16 @@ def real_gemm_bits(Hp, Wout, b, H):
     return Z
 
 
+def real_gemm_bits01(Hp, Wout, b, H):
+    Hp = np.ascontiguousarray(Hp, dtype=np.uint32)
+    Wout, b = _f32(Wout), _f32(b)
+    M, Cn = Hp.shape[0], Wout.shape[0]
+    Z = np.empty((M, Cn), dtype=np.float64)
+    lib().oracle_real_gemm_bits01(_p(Hp), _L(Hp.shape[1]), _p(Wout), _L(Wout.shape[1]), _p(b),
+                                  _L(M), _L(Cn), _L(H), _p(Z), _L(Cn))
+    return Z
+
+
 def real_gemm_f32(Hf, Wout, b):
     Hf, Wout, b = _f32(Hf), _f32(Wout), _f32(b)
     M, H = Hf.shape
@@ -169,7 +201,7 @@ def log_softmax(Z):
 
 
 def forward(X, W, scale, shift, Wout, bout, act=ACT_SIGN, mode=SIGN_ZERO_POS,
-            layer1_bits=None):
+            layer1_bits=None, values=VALUES_PM1):
     """Whole forward pass, layer by layer in the order of Algorithms 1 and 2.
 
     W: list of real-valued weight matrices [N_l][K_l]; they are binarised with Eq. 3 first.
@@ -177,7 +209,9 @@ def forward(X, W, scale, shift, Wout, bout, act=ACT_SIGN, mode=SIGN_ZERO_POS,
     act == ACT_HARDTANH: every hidden layer is +-1 weights on real activations.
     ``layer1_bits`` (optional) replaces the oracle's own first-layer bits, so that a caller
     can continue from another implementation's decision on values inside the float
-    tolerance band.  Returns a dict of per-layer taps and ``logp``.
+    tolerance band.  ``values`` = VALUES_01 makes the binary activations (0,1) instead of
+    (-1,+1) (Section 3.2): the stored bit is the same decision (pre-activation above / at zero),
+    it stands for 1 / 0 in the layer that consumes it.  Returns a dict of per-layer taps and ``logp``.
     """
     X = _f32(X)
     taps = {"Wp": [], "pre": [], "bits": [], "h": []}
@@ -194,11 +228,11 @@ def forward(X, W, scale, shift, Wout, bout, act=ACT_SIGN, mode=SIGN_ZERO_POS,
             P = np.ascontiguousarray(layer1_bits, dtype=np.uint32)[:, :words(W[0].shape[0])]
         taps["bits"].append(P)
         for l in range(1, len(W)):
-            D = xnor_gemm(P, Wp[l], W[l].shape[1])
+            D = (gemm01 if values == VALUES_01 else xnor_gemm)(P, Wp[l], W[l].shape[1])
             P = affine_sign_pack_i32(D, scale[l], shift[l], mode)
             taps["pre"].append(D)
             taps["bits"].append(P)
-        Z = real_gemm_bits(P, Wout, bout, Wout.shape[1])
+        Z = (real_gemm_bits01 if values == VALUES_01 else real_gemm_bits)(P, Wout, bout, Wout.shape[1])
     else:
         Hf = X
         for l in range(len(W)):

@@ -290,3 +290,72 @@ def test_forward_binary_weight_variant_against_numpy():
     z = h @ Wout.astype(np.float64).T + bout
     z = z - z.max(1, keepdims=True)
     np.testing.assert_allclose(t["logp"], z - np.log(np.exp(z).sum(1, keepdims=True)), atol=1e-12)
+
+
+# ---------------------------------------------------------------- (0,1) activations (Section 3.2)
+@pytest.mark.parametrize("k", [1, 31, 32, 33, 127, 440, 600])
+def test_gemm01_brute_force_float_matmul(k):
+    h = wl.make_bit_matrix(5, k, 0.4, [12, k])
+    w = wl.make_bit_matrix(9, k, 0.5, [13, k])
+    d = o.gemm01(np_pack(h), np_pack(w), k)
+    ref = h.astype(np.float64) @ pm1(w).T   # h in {0,1}, w in {-1,+1}; exact in float64
+    assert d.dtype == np.int32 and d.shape == (5, 9)
+    np.testing.assert_array_equal(d, ref.astype(np.int64))
+
+
+def test_gemm01_invariants_and_relation_to_the_pm1_product():
+    k = 203
+    h = wl.make_bit_matrix(6, k, 0.5, 21)
+    w = wl.make_bit_matrix(4, k, 0.3, 22)
+    hp, wp = np_pack(h), np_pack(w)
+    d = o.gemm01(hp, wp, k)
+    ones = h.sum(1, dtype=np.int64)
+    # |d| <= number of ones in the row, and d has that number's parity
+    assert np.all(np.abs(d) <= ones[:, None]) and np.all((d - ones[:, None]) % 2 == 0)
+    # AND-popcount identity  d = 2 popc(h and w) - popc(h)
+    an = (h[:, None, :] & w[None, :, :]).sum(-1).astype(np.int64)
+    np.testing.assert_array_equal(d, 2 * an - ones[:, None])
+    # h = (a + 1) / 2  =>  2 d = dot_pm1(a, w) + sum_k w[n][k]
+    wsum = pm1(w).sum(1).astype(np.int64)
+    np.testing.assert_array_equal(2 * d, o.xnor_gemm(hp, wp, k) + wsum[None, :])
+    # an all-zero row gives 0, an all-one row the sum of the unit's weights
+    np.testing.assert_array_equal(o.gemm01(np_pack(np.zeros((1, k), np.uint8)), wp, k), 0)
+    np.testing.assert_array_equal(o.gemm01(np_pack(np.ones((1, k), np.uint8)), wp, k)[0], wsum)
+    # pad bits and pitch words are ignored
+    hp2 = np.concatenate([hp, np.full((6, 2), 0xFFFFFFFF, np.uint32)], 1)
+    hp2[:, (k - 1) // 32] |= np.uint32((0xFFFFFFFF << (k % 32)) & 0xFFFFFFFF)
+    np.testing.assert_array_equal(o.gemm01(hp2, wp, k), d)
+
+
+def test_real_gemm_bits01_against_matmul():
+    rng = np.random.default_rng(8)
+    h = wl.make_bit_matrix(7, 70, 0.5, 31)
+    Wout = rng.standard_normal((11, 70)).astype(np.float32)
+    b = rng.standard_normal(11).astype(np.float32)
+    z = o.real_gemm_bits01(np_pack(h), Wout, b, 70)
+    np.testing.assert_allclose(z, h.astype(np.float64) @ Wout.astype(np.float64).T + b, atol=1e-12)
+
+
+def test_forward_with_01_activations_against_numpy():
+    """Algorithm 2's forward loop with the hidden activations in (0,1): h = 1 where the
+    pre-activation is positive, 0 elsewhere; exactly representable values, so the numpy
+    restatement must agree to rounding."""
+    rng = np.random.default_rng(14)
+    dims = [37, 50, 41, 33]
+    X = rng.integers(-4, 5, (6, dims[0])).astype(np.float32)
+    W = [rng.choice([-0.7, 0.0, 0.3, 1.0], (dims[i + 1], dims[i])).astype(np.float32) for i in range(3)]
+    r = [(rng.integers(-3, 4, dims[i + 1]) + 0.5).astype(np.float32) for i in range(3)]
+    r[1][:5] = [0.0, 1.0, -1.0, 2.0, -2.0]
+    Wout = rng.standard_normal((19, dims[-1])).astype(np.float32)
+    bout = rng.standard_normal(19).astype(np.float32)
+    t = o.forward(X, W, [None] * 3, r, Wout, bout, o.ACT_SIGN, o.SIGN_ZERO_NEG, values=o.VALUES_01)
+    h = X.astype(np.float64)
+    for w, b in zip(W, r):
+        wb = np.where(w > 0, 1.0, -1.0)                  # Eq. 3 as printed
+        h = ((h @ wb.T + b.astype(np.float64)) > 0).astype(np.float64)
+    z = h @ Wout.astype(np.float64).T + bout
+    z = z - z.max(1, keepdims=True)
+    np.testing.assert_allclose(t["logp"], z - np.log(np.exp(z).sum(1, keepdims=True)), atol=1e-12)
+    # and it is a different function from the (-1,+1) network on this input
+    t2 = o.forward(X, W, [None] * 3, r, Wout, bout, o.ACT_SIGN, o.SIGN_ZERO_NEG)
+    assert np.abs(t["logp"] - t2["logp"]).max() > 1e-3
