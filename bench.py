@@ -41,6 +41,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--xnor-prepared", default="auto", choices=["auto", "stream", "resident"],
                     help="kernel for hidden layers with prepared weights (see BNN_OPT_XNOR_PREPARED)")
+    ap.add_argument("--act-values", default="pm1", choices=["pm1", "01"],
+                    help="what the binary activations stand for: (-1,+1) or (0,1)")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every step's kernels from the host instead of replaying a captured CUDA graph")
     ap.add_argument("--sweep", action="store_true",
@@ -291,7 +293,8 @@ def run_ours(args):
     B.bnn_set_xnor_path(B.XNOR_POPC if args.xnor_path == "popc" else B.XNOR_TENSOR)
     B.bnn_set_option(B.OPT_REAL_PATH, B.PATH_TENSOR if args.real_path == "tensor" else B.PATH_CUDA_CORE)
     B.bnn_set_option(B.OPT_XNOR_PREPARED, {"auto": 0, "stream": 1, "resident": 2}[args.xnor_prepared])
-    dn = model.DeviceNet(net, device=dev, prepare_xnor=args.xnor_path == "tensor")
+    dn = model.DeviceNet(net, device=dev, prepare_xnor=args.xnor_path == "tensor",
+                         act_values=B.VALUES_01 if args.act_values == "01" else B.VALUES_PM1)
     # Frames are independent, so ranks shard them with no exchange: each rank owns its own batch.
     Xh = wl.make_frames(cfg, frames, seed=D.frames_seed(cfg.seed, rank))
     set_bytes = frames * (cfg.in_dim + cfg.classes) * 4
@@ -473,7 +476,7 @@ def run_ours(args):
         "config": {"workload": workload_name(cfg, frames), "frames_per_gpu": frames,
                    "launch": "host launches" if args.no_graph else "one captured CUDA graph per step (a single bnn_forward call each)", "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 2 x L2); weights stay hot"
                          % (nsets, nsets * set_bytes / 1e6),
-                   "sign_zero": "+1", "seed": cfg.seed},
+                   "sign_zero": "+1", "act_values": "(0,1)" if args.act_values == "01" else "(-1,+1)", "seed": cfg.seed},
         "clocks": ck,
         "e2e": {"value": e2e_fps, "unit": UNIT, "h2d_bytes_per_step": int(Xp.numel() * 4),
                 "d2h_bytes_per_step": int(Lp.numel() * 4), "steps": Ke,

@@ -52,6 +52,14 @@ typedef enum {
  * NaN maps to -1 in both modes (every comparison with NaN is false). */
 typedef enum { BNN_SIGN_ZERO_POS = 0, BNN_SIGN_ZERO_NEG = 1 } bnn_sign_mode;
 
+/* What a stored bit of a binarised ACTIVATION matrix stands for in the layer that reads it.
+ * The paper works with the pair (-1,+1) and also reports binary activations in (0,1), "the
+ * hard version of Sigmoid" (Section 3.2, Table 3; Section 3.3, Table 4).  The decision that
+ * sets the bit is the same in both (pre-activation positive, or zero under
+ * BNN_SIGN_ZERO_POS); only the value the next layer multiplies differs.  Weights are always
+ * (-1,+1): the paper's (0,1) weights did not train (Table 3). */
+typedef enum { BNN_VALUES_PM1 = 0, BNN_VALUES_01 = 1 } bnn_act_values;
+
 /* What happens to a pre-activation after the per-unit affine (Eq. 2, h = f(h_hat)). */
 typedef enum {
     BNN_ACT_NONE = 0,      /* write the value itself */
@@ -144,6 +152,17 @@ BNN_API int bnn_xnor_gemm_prepared(const uint32_t* Ap, int ldap, const void* pre
                                    int M, int N, int K, int32_t* C, int ldc,
                                    const bnn_epilogue* epi, void* stream);
 
+/* The product of bnn_xnor_gemm for activations in (0,1) (Section 3.2):
+ * d[m][n] = sum_k h[m][k]*w[n][k] with h in {0,1}, w in {-1,+1}
+ *         = 2*popcount(h_bits AND w_bits) - popcount(h_bits).
+ * Hp : [M][ldhp] packed activations (bit = value).  Wp : [N][ldwp] packed weights, or NULL when
+ * `prepared` (the bnn_xnor_prepare image of the same weights) is given; with both, the library
+ * picks the faster kernel.  C, epi, errors: as bnn_xnor_gemm (the thresholds of
+ * bnn_fold_thresholds apply unchanged: d still lies in [-K, K]). */
+BNN_API int bnn_gemm01(const uint32_t* Hp, int ldhp, const uint32_t* Wp, int ldwp, const void* prepared,
+                       int M, int N, int K, int32_t* C, int ldc,
+                       const bnn_epilogue* epi, void* stream);
+
 /* ------------------------------------------------------------------------------------
  * Binary weights against real-valued activations (Section 2.1; Algorithm 1 forward):
  * y[m][n] = sum_k w^b[n][k]*x[m][k] -- additions and subtractions only -- followed by the
@@ -184,6 +203,12 @@ BNN_API int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int 
                      int M, int C, int H, float* logp, int ldo, int log_softmax,
                      void* stream);
 
+/* bnn_output_layer on packed activations that stand for (0,1) (Section 3.2); other arguments
+ * as there. */
+BNN_API int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw,
+                               const float* b, const void* prepared, int M, int C, int H,
+                               float* logp, int ldo, int log_softmax, void* stream);
+
 /* One-time preparation of the top layer's weights for the tensor cores: each class row is
  * scaled by a power of two and split into two fp16 terms (about 22 significant bits), stored
  * in the order the MMA reads shared memory.  prepared : device buffer, 256-byte aligned, of
@@ -223,6 +248,7 @@ typedef struct bnn_model {
     int n_layers;
     int sign_mode;
     const bnn_layer* layers; /* HOST array of n_layers entries (device pointers inside) */
+    int act_values;          /* bnn_act_values of every BNN_ACT_SIGN_PACK activation */
 } bnn_model;
 
 /* Bytes of scratch for M frames.  bnn_forward_workspace_bytes is what makes bnn_forward

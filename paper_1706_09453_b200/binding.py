@@ -15,6 +15,7 @@ from . import build as _build
 
 SIGN_ZERO_POS, SIGN_ZERO_NEG = 0, 1
 ACT_NONE, ACT_SIGN_PACK, ACT_HARDTANH = 0, 1, 2
+VALUES_PM1, VALUES_01 = 0, 1
 LAYER_SIGNW, LAYER_XNOR, LAYER_REAL_OUT = 0, 1, 2
 
 
@@ -41,7 +42,8 @@ class Layer(C.Structure):
 
 
 class Model(C.Structure):
-    _fields_ = [("n_layers", C.c_int), ("sign_mode", C.c_int), ("layers", C.POINTER(Layer))]
+    _fields_ = [("n_layers", C.c_int), ("sign_mode", C.c_int), ("layers", C.POINTER(Layer)),
+                ("act_values", C.c_int)]
 
 
 _lib = None
@@ -99,6 +101,10 @@ def lib():
         L.bnn_xnor_gemm.argtypes = [p, i, p, i, i, i, i, p, i, C.POINTER(Epilogue), p]
         L.bnn_signw_gemm.argtypes = [p, i, p, i, i, i, i, p, i, C.POINTER(Epilogue), p]
         L.bnn_output_layer.argtypes = [p, i, p, i, p, i, p, p, i, i, i, p, i, i, p]
+        L.bnn_output_layer01.argtypes = [p, i, p, i, p, p, i, i, i, p, i, i, p]
+        L.bnn_output_layer01.restype = C.c_int
+        L.bnn_gemm01.argtypes = [p, i, p, i, p, i, i, i, p, i, C.POINTER(Epilogue), p]
+        L.bnn_gemm01.restype = C.c_int
         L.bnn_forward.argtypes = [C.POINTER(Model), p, i, i, p, i, p, C.c_size_t, C.POINTER(p), p]
         L.bnn_forward_static.argtypes = [C.POINTER(Model), p, i, i, p, i, p]
         L.bnn_forward_static.restype = C.c_int
@@ -253,6 +259,18 @@ def bnn_xnor_gemm_prepared(Ap, prepared, N, K, C_out=None, thr=None, flip=None, 
                                         e, _stream()), "bnn_xnor_gemm_prepared")
 
 
+def bnn_gemm01(Hp, Wp, K, N=None, prepared=None, C_out=None, thr=None, flip=None, out_bits=None):
+    """Activations in (0,1) x weights in (-1,+1); ``Wp`` and/or ``prepared`` give the weights."""
+    n = Wp.shape[0] if Wp is not None else N
+    e = None
+    if out_bits is not None:
+        e = C.byref(_epilogue(ACT_SIGN_PACK, thr=thr, flip=flip, out_bits=out_bits))
+    _check(lib().bnn_gemm01(_ptr(Hp, torch.int32), _ld(Hp), _ptr(Wp, torch.int32), _ld(Wp) if Wp is not None else 0,
+                            _ptr(prepared), Hp.shape[0], n, K,
+                            _ptr(C_out, torch.int32), _ld(C_out) if C_out is not None else 0,
+                            e, _stream()), "bnn_gemm01")
+
+
 def bnn_signw_workspace_bytes(M, K) -> int:
     return int(lib().bnn_signw_workspace_bytes(int(M), int(K)))
 
@@ -284,9 +302,15 @@ def bnn_output_prepare(Wout, prepared):
     return prepared
 
 
-def bnn_output_layer(Wout, b, logp, H, Hp=None, Hf=None, log_softmax=True, prepared=None):
+def bnn_output_layer(Wout, b, logp, H, Hp=None, Hf=None, log_softmax=True, prepared=None, values=VALUES_PM1):
     m = (Hp if Hp is not None else Hf).shape[0]
     c = Wout.shape[0]
+    if values == VALUES_01:
+        _check(lib().bnn_output_layer01(_ptr(Hp, torch.int32), _ld(Hp), _ptr(Wout, torch.float32), _ld(Wout),
+                                        _ptr(b, torch.float32), _ptr(prepared), m, c, H,
+                                        _ptr(logp, torch.float32), _ld(logp), int(log_softmax), _stream()),
+               "bnn_output_layer01")
+        return logp
     _check(lib().bnn_output_layer(_ptr(Hp, torch.int32), _ld(Hp) if Hp is not None else 0,
                                   _ptr(Hf, torch.float32), _ld(Hf) if Hf is not None else 0,
                                   _ptr(Wout, torch.float32), _ld(Wout), _ptr(b, torch.float32),
@@ -298,7 +322,7 @@ def bnn_output_layer(Wout, b, logp, H, Hp=None, Hf=None, log_softmax=True, prepa
 class ModelDesc:
     """Host-side bnn_model built from a list of layer dicts; keeps the tensors alive."""
 
-    def __init__(self, layers, sign_mode=SIGN_ZERO_POS):
+    def __init__(self, layers, sign_mode=SIGN_ZERO_POS, act_values=VALUES_PM1):
         self._keep = layers
         arr = (Layer * len(layers))()
         for a, d in zip(arr, layers):
@@ -310,7 +334,7 @@ class ModelDesc:
             a.scale, a.shift = _ptr(d.get("scale"), torch.float32), _ptr(d.get("shift"), torch.float32)
             a.thr, a.flip = _ptr(d.get("thr"), torch.int32), _ptr(d.get("flip"), torch.int32)
         self._arr = arr
-        self.c = Model(len(layers), sign_mode, arr)
+        self.c = Model(len(layers), sign_mode, arr, act_values)
         self.layers = layers
 
     def workspace_bytes(self, M: int) -> int:

@@ -49,6 +49,7 @@ int validate_model(const bnn_model* model) {
     if (L < 1) return BNN_ERR_SHAPE;
     if (model->sign_mode != BNN_SIGN_ZERO_POS && model->sign_mode != BNN_SIGN_ZERO_NEG)
         return BNN_ERR_UNSUPPORTED;
+    if (model->act_values != BNN_VALUES_PM1 && model->act_values != BNN_VALUES_01) return BNN_ERR_UNSUPPORTED;
     int prev_act = BNN_ACT_NONE;  // real-valued input h_0
     int prev_n = -1;
     for (int l = 0; l < L; ++l) {
@@ -156,7 +157,7 @@ int bnn_fold_thresholds(const float* scale, const float* shift, int N, int K, in
 // bnn_forward (both, when the layer has an image).
 static int xnor_gemm_impl(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, const void* image,
                           int M, int N, int K, int32_t* C, int ldc,
-                          const bnn_epilogue* epi, void* stream) {
+                          const bnn_epilogue* epi, int zo, void* stream) {
     if (int rc = check_dims(M, N, K)) return rc;
     if (K > kMaxK) return BNN_ERR_SHAPE;
     if (int rc = check_packed(Ap, ldap, K)) return rc;
@@ -187,20 +188,26 @@ static int xnor_gemm_impl(const uint32_t* Ap, int ldap, const uint32_t* Wp, int 
         const bool fused = !C && g_xnor_prepared != BNN_PREPARED_STREAM && xnor_res_applicable(N, K);
         const bool wide_tiles = K <= 2048;
         if (fused && (wide_tiles || !Wp || g_xnor_prepared == BNN_PREPARED_RESIDENT))
-            return launch_xnor_res(Ap, ldap, image, M, N, K, thr, flip, ob, ldob, (cudaStream_t)stream);
+            return launch_xnor_res(Ap, ldap, image, M, N, K, thr, flip, ob, ldob, zo, (cudaStream_t)stream);
         if (!Wp || g_xnor_prepared == BNN_PREPARED_STREAM)
-            return launch_xnor_img(Ap, ldap, image, M, N, K, C, ldc, thr, flip, ob, ldob, (cudaStream_t)stream);
+            return launch_xnor_img(Ap, ldap, image, M, N, K, C, ldc, thr, flip, ob, ldob, zo, (cudaStream_t)stream);
     }
     const bool tensor = g_xnor_path != BNN_PATH_CUDA_CORE && K <= kMaxKTensor;
     return (tensor ? launch_xnor_tc : launch_xnor_popc)(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip,
-                                                        ob, ldob, (cudaStream_t)stream);
+                                                        ob, ldob, zo, (cudaStream_t)stream);
 }
 
 int bnn_xnor_gemm(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp,
                   int M, int N, int K, int32_t* C, int ldc,
                   const bnn_epilogue* epi, void* stream) {
     if (!Wp) return BNN_ERR_NULL;
-    return xnor_gemm_impl(Ap, ldap, Wp, ldwp, nullptr, M, N, K, C, ldc, epi, stream);
+    return xnor_gemm_impl(Ap, ldap, Wp, ldwp, nullptr, M, N, K, C, ldc, epi, 0, stream);
+}
+
+int bnn_gemm01(const uint32_t* Hp, int ldhp, const uint32_t* Wp, int ldwp, const void* prepared,
+               int M, int N, int K, int32_t* C, int ldc, const bnn_epilogue* epi, void* stream) {
+    if (!Wp && !prepared) return BNN_ERR_NULL;
+    return xnor_gemm_impl(Hp, ldhp, Wp, ldwp, prepared, M, N, K, C, ldc, epi, 1, stream);
 }
 
 size_t bnn_xnor_prepared_bytes(int N, int K) {
@@ -223,7 +230,7 @@ int bnn_xnor_gemm_prepared(const uint32_t* Ap, int ldap, const void* prepared,
                            int M, int N, int K, int32_t* C, int ldc,
                            const bnn_epilogue* epi, void* stream) {
     if (!prepared) return BNN_ERR_NULL;
-    return xnor_gemm_impl(Ap, ldap, nullptr, 0, prepared, M, N, K, C, ldc, epi, stream);
+    return xnor_gemm_impl(Ap, ldap, nullptr, 0, prepared, M, N, K, C, ldc, epi, 0, stream);
 }
 
 size_t bnn_signw_workspace_bytes(int M, int K) {
@@ -289,7 +296,7 @@ int bnn_output_prepare(const float* Wout, int ldw, int C, int H,
 static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
                              const float* Wout, int ldw, const float* b, const void* prepared,
                              int M, int C, int H, float* logp, int ldo, int log_softmax,
-                             void* mid_event, void* stream) {
+                             int zo, void* mid_event, void* stream) {
     if (int rc = check_dims(M, C, H)) return rc;
     if (!Wout || !logp) return BNN_ERR_NULL;
     if ((Hp == nullptr) == (Hf == nullptr)) return Hp ? BNN_ERR_UNSUPPORTED : BNN_ERR_NULL;
@@ -297,7 +304,7 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
     RealGemmArgs a{};
     if (Hp) {
         if (int rc = check_packed(Hp, ldhp, H)) return rc;
-        a.Ab = Hp; a.lda = ldhp;
+        a.Ab = Hp; a.lda = ldhp; a.a_zero_one = zo;
     } else {
         if (ldhf < H) return BNN_ERR_SHAPE;
         a.Af = Hf; a.lda = ldhf;
@@ -310,7 +317,7 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
     if (prepared && (reinterpret_cast<uintptr_t>(prepared) & 255u)) return BNN_ERR_ALIGN;
     int rc;
     if (Hp && prepared && g_real_path != BNN_PATH_CUDA_CORE)
-        rc = launch_out_tc(Hp, ldhp, prepared, b, M, C, H, logp, ldo, (cudaStream_t)stream);
+        rc = launch_out_tc(Hp, ldhp, prepared, b, M, C, H, logp, ldo, zo, (cudaStream_t)stream);
     else
         rc = launch_real_gemm(a, (cudaStream_t)stream);
     if (rc) return rc;
@@ -325,7 +332,15 @@ int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
                      int M, int C, int H, float* logp, int ldo, int log_softmax,
                      void* stream) {
     return output_layer_impl(Hp, ldhp, Hf, ldhf, Wout, ldw, b, prepared, M, C, H, logp, ldo,
-                             log_softmax, nullptr, stream);
+                             log_softmax, 0, nullptr, stream);
+}
+
+int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw, const float* b,
+                       const void* prepared, int M, int C, int H, float* logp, int ldo,
+                       int log_softmax, void* stream) {
+    if (!Hp) return BNN_ERR_NULL;
+    return output_layer_impl(Hp, ldhp, nullptr, 0, Wout, ldw, b, prepared, M, C, H, logp, ldo,
+                             log_softmax, 1, nullptr, stream);
 }
 
 size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M) {
@@ -387,6 +402,7 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
             int rc = output_layer_impl(in_bits ? static_cast<const uint32_t*>(in) : nullptr, in_ld,
                                        in_bits ? nullptr : static_cast<const float*>(in), in_ld,
                                        y.W, y.ldw, y.shift, y.W_prepared, M, y.N, y.K, logp, ldo, 1,
+                                       in_bits && model->act_values == BNN_VALUES_01,
                                        events ? events[L + 1] : nullptr, stream);
             if (rc) return rc;
             if (events && events[L] &&
@@ -419,7 +435,8 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
             e.out_bits = static_cast<uint32_t*>(out); e.ldob = bnn_packed_pitch(y.N);
             const bool image = y.W_prepared && g_xnor_path != BNN_PATH_CUDA_CORE && y.K <= kMaxKTensor;
             rc = xnor_gemm_impl(static_cast<const uint32_t*>(in), in_ld, y.Wp, y.ldwp,
-                                image ? y.W_prepared : nullptr, M, y.N, y.K, nullptr, 0, &e, stream);
+                                image ? y.W_prepared : nullptr, M, y.N, y.K, nullptr, 0, &e,
+                                model->act_values == BNN_VALUES_01, stream);
             in_ld = e.ldob;
         }
         if (rc) return rc;

@@ -46,15 +46,17 @@ int launch_sign_pack(const float* X, int M, int K, int ldx, uint32_t* P, int ldp
                      cudaStream_t st);
 int launch_fold_thresholds(const float* scale, const float* shift, int N, int K, int mode,
                            int32_t* thr, uint32_t* flip, cudaStream_t st);
+// `zo` != 0 in the binary GEMMs below: the bits of the frame operand stand for (0,1) instead of
+// (-1,+1), so the result is sum_k h*w with h in {0,1} and w in {-1,+1}.
 int launch_xnor_popc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
                      int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
-                     uint32_t* out_bits, int ldob, cudaStream_t st);
+                     uint32_t* out_bits, int ldob, int zo, cudaStream_t st);
 
 // Tensor-core (tcgen05) XNOR GEMM; same contract as launch_xnor_popc.  K <= kMaxKTensor.
 constexpr int kMaxKTensor = 1 << 22;
 int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
                    int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
-                   uint32_t* out_bits, int ldob, cudaStream_t st);
+                   uint32_t* out_bits, int ldob, int zo, cudaStream_t st);
 // The same product with the unit operand given as the image launch_xnor_prepare built from the
 // packed weights (xnor_gemm_img.cu): xnor_image_bytes(N, K) bytes, 256-byte aligned.
 size_t xnor_image_bytes(int N, int K);
@@ -64,11 +66,11 @@ __host__ __device__ __forceinline__ int xnor_image_npad(int N) { return ceil_div
 // xnor_res_applicable says whether a layer of this shape fits that kernel.
 bool xnor_res_applicable(int N, int K);
 int launch_xnor_res(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
-                    const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, cudaStream_t st);
+                    const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int zo, cudaStream_t st);
 int launch_xnor_prepare(const uint32_t* Wp, int ldwp, int N, int K, void* image, cudaStream_t st);
 int launch_xnor_img(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
                     int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
-                    uint32_t* out_bits, int ldob, cudaStream_t st);
+                    uint32_t* out_bits, int ldob, int zo, cudaStream_t st);
 // Pipe micro-benchmarks (pipe_rates.cu).
 size_t pipe_rate_scratch_bytes(int which);
 int launch_pipe_rate(int which, int repeat, void* scratch, size_t scratch_bytes, double* work, cudaStream_t st);
@@ -85,6 +87,7 @@ int* tc_status_ptr();
 struct RealGemmArgs {
     const float* Af;      // fp32 A [M][lda] or nullptr
     const uint32_t* Ab;   // packed A [M][lda] or nullptr
+    int a_zero_one;       // packed A stands for (0,1) instead of (-1,+1)
     int lda;
     const float* Bf;      // fp32 B [N][ldb] or nullptr
     const uint32_t* Bb;   // packed B [N][ldb] or nullptr
@@ -110,7 +113,7 @@ int launch_signw_img(const RealGemmArgs& a, int terms, void* workspace, cudaStre
 size_t out_prepared_bytes(int C, int H);
 int launch_out_prepare(const float* W, int ldw, int C, int H, void* prepared, cudaStream_t st);
 int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const float* bias,
-                  int M, int C, int H, float* Z, int ldz, cudaStream_t st);
+                  int M, int C, int H, float* Z, int ldz, int zo, cudaStream_t st);
 int launch_log_softmax_rows(float* Z, int ldz, int M, int C, cudaStream_t st);
 
 }  // namespace bnn

@@ -108,7 +108,7 @@ __global__ void out_split_kernel(const float* __restrict__ W, int ldw, int C, in
 __global__ void __launch_bounds__(THREADS, 1)
 out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restrict__ img,
               const float* __restrict__ rs, const float* __restrict__ bias,
-              int M, int C, int H, float* __restrict__ Z, int ldz, int* __restrict__ status) {
+              int M, int C, int H, float* __restrict__ Z, int ldz, int zo, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES);
@@ -184,7 +184,13 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
                 const uint32_t nw = ~cur[q];
                 uint32_t wv[16];
 #pragma unroll
-                for (int t = 0; t < 16; ++t) wv[t] = ((nw << (15 - t)) & 0x80008000u) | 0x3C003C00u;
+                if (zo) {   // (0,1) activations: 1.0 (0x3C00) where the bit is set, +0 elsewhere
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) wv[t] = ((cur[q] >> t) & 0x00010001u) * 0x3C00u;
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) wv[t] = ((nw << (15 - t)) & 0x80008000u) | 0x3C003C00u;
+                }
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
                     sts128(st + A_BYTES + (c * FN + p + 256 * q) * 16, wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
@@ -294,7 +300,7 @@ int launch_out_prepare(const float* W, int ldw, int C, int H, void* prepared, cu
 }
 
 int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const float* bias,
-                  int M, int C, int H, float* Z, int ldz, cudaStream_t st) {
+                  int M, int C, int H, float* Z, int ldz, int zo, cudaStream_t st) {
     static bool configured = false;
     static int sms = 0;
     if (!configured) {
@@ -311,7 +317,7 @@ int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const floa
     const int tiles = ct * ceil_div(M, FN);
     int* status = tc_status_ptr();
     if (!status) return BNN_ERR_CUDA;
-    out_tc_kernel<<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(Hp, ldhp, img, rs, bias, M, C, H, Z, ldz, status);
+    out_tc_kernel<<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(Hp, ldhp, img, rs, bias, M, C, H, Z, ldz, zo, status);
     return launch_status();
 }
 

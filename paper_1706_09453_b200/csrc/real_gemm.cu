@@ -70,15 +70,16 @@ __device__ __forceinline__ void fetch(Fetch& r, const Operand& op, int row0, int
     }
 }
 
-// Registers -> shared tile S[k][row] (k-major).  Bits become +-1.0f; positions k >= K of a
-// bit operand become -1.0f, which is harmless because the fp32 operand is zero there.
+// Registers -> shared tile S[k][row] (k-major).  Bits become +1.0f / `low` (-1.0f, or 0.0f for
+// activations that stand for (0,1)); positions k >= K of a bit operand become `low`, which is
+// harmless because the fp32 operand is zero there.
 template <bool BITS>
-__device__ __forceinline__ void stash(const Fetch& r, float (*S)[PADW]) {
+__device__ __forceinline__ void stash(const Fetch& r, float (*S)[PADW], float low = -1.0f) {
     const int t = threadIdx.x;
     if (BITS) {
         if (t < TM) {
 #pragma unroll
-            for (int k = 0; k < TK; ++k) S[k][t] = ((r.word >> k) & 1u) ? 1.0f : -1.0f;
+            for (int k = 0; k < TK; ++k) S[k][t] = ((r.word >> k) & 1u) ? 1.0f : low;
         }
     } else {
         const int kq = t & 7;
@@ -114,7 +115,7 @@ real_gemm_kernel(RealGemmArgs g) {
     fetch<A_BITS>(fa, opa, m0, 0, g.K, va);
     fetch<B_BITS>(fb, opb, n0, 0, g.K, vb);
     for (int kb = 0; kb < g.K; kb += TK) {
-        stash<A_BITS>(fa, As);
+        stash<A_BITS>(fa, As, g.a_zero_one ? 0.0f : -1.0f);
         stash<B_BITS>(fb, Bs);
         __syncthreads();
         if (kb + TK < g.K) {

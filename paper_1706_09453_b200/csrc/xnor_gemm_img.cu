@@ -109,6 +109,7 @@ struct ProducerArgs {
     int tiles, nks, kw;
     uint32_t tmask;
     int lane;
+    int zo;               // the frame operand's bits stand for (0,1) instead of (-1,+1)
 };
 
 // Producer of the frame operand: thread = row `r` of every tile of this CTA, one stage per
@@ -138,7 +139,15 @@ __device__ __forceinline__ void produce_a(const ProducerArgs& a, int r) {
         // 32-bit column 4c + t of the stage = word t of chunk c: the byte order of the
         // K-major shared-memory layout of the other operand
         uint32_t wr[32];
-        if (ragged && ks == a.nks - 1) {
+        if (a.zo) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const int g = 8 * ks + c;   // index of the word in the row
+                const uint32_t valid = (!ragged || g < a.kw - 1) ? 0xFFFFFFFFu : (g == a.kw - 1 ? a.tmask : 0u);
+                const uint4 o = widen01_masked(w[c], valid);
+                wr[4 * c] = o.x; wr[4 * c + 1] = o.y; wr[4 * c + 2] = o.z; wr[4 * c + 3] = o.w;
+            }
+        } else if (ragged && ks == a.nks - 1) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const int g = 8 * ks + c;   // index of the word in the row
@@ -176,7 +185,7 @@ __global__ void __launch_bounds__(THREADS, 1)
 xnor_img_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restrict__ img,
                 int M, int N, int K, int32_t* __restrict__ C, int ldc,
                 const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
-                uint32_t* __restrict__ out_bits, int ldob, int* __restrict__ status) {
+                uint32_t* __restrict__ out_bits, int ldob, int zo, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(smem + B_STAGES * B_BYTES + GROUPS * GROUP_BYTES);
@@ -276,7 +285,7 @@ xnor_img_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
         }
         __syncwarp();
     } else if (warp >= PROD_WARP0) {
-        ProducerArgs pa{smem_u32(smem) + B_STAGES * B_BYTES, tmem, ctl, abort_flag, tiles, nks, kw, tail_mask(K), lane};
+        ProducerArgs pa{smem_u32(smem) + B_STAGES * B_BYTES, tmem, ctl, abort_flag, tiles, nks, kw, tail_mask(K), lane, zo};
         produce_a(pa, (warp & 3) * 32 + lane);
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issue: one thread
@@ -428,7 +437,7 @@ xnor_img_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
 template <bool STORE_C, bool SIGN_PACK>
 int launch_variant(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
                    int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
-                   uint32_t* out_bits, int ldob, cudaStream_t st) {
+                   uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
     auto kern = xnor_img_kernel<STORE_C, SIGN_PACK>;
     constexpr int SMEM = smem_bytes<STORE_C>();
     static bool configured = false;
@@ -448,7 +457,7 @@ int launch_variant(const uint32_t* Ap, int ldap, const void* image, int M, int N
     CUtensorMap mapA;
     if (!encode_packed_map(&mapA, Ap, ldap, M, K, BM)) return BNN_ERR_CUDA;
     kern<<<grid, THREADS, SMEM, st>>>(mapA, static_cast<const uint8_t*>(image), M, N, K, C, ldc, thr, flip,
-                                      out_bits, ldob, status);
+                                      out_bits, ldob, zo, status);
     return launch_status();
 }
 
@@ -470,11 +479,11 @@ int launch_xnor_prepare(const uint32_t* Wp, int ldwp, int N, int K, void* image,
 
 int launch_xnor_img(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
                     int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
-                    uint32_t* out_bits, int ldob, cudaStream_t st) {
+                    uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
     const bool sp = out_bits != nullptr;
-    if (C && sp) return launch_variant<true, true>(Ap, ldap, image, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
-    if (C) return launch_variant<true, false>(Ap, ldap, image, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
-    return launch_variant<false, true>(Ap, ldap, image, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
+    if (C && sp) return launch_variant<true, true>(Ap, ldap, image, M, N, K, C, ldc, thr, flip, out_bits, ldob, zo, st);
+    if (C) return launch_variant<true, false>(Ap, ldap, image, M, N, K, C, ldc, thr, flip, out_bits, ldob, zo, st);
+    return launch_variant<false, true>(Ap, ldap, image, M, N, K, C, ldc, thr, flip, out_bits, ldob, zo, st);
 }
 
 }  // namespace bnn

@@ -1,4 +1,5 @@
-// XNOR-popcount GEMM on the integer pipes: d[m][n] = K - 2*popc(a[m] xor w[n]).
+// XNOR-popcount GEMM on the integer pipes: d[m][n] = K - 2*popc(a[m] xor w[n]); with the frame
+// bits standing for (0,1) instead of (-1,+1): d[m][n] = 2*popc(a[m] and w[n]) - popc(a[m]).
 //
 // CTA tile 128 (frames) x 128 (units), 256 threads.  Warp y owns 16 frames; lane x owns the
 // four units x, x+32, x+64, x+96, so that one ballot over the warp yields a whole packed
@@ -66,7 +67,7 @@ __device__ __forceinline__ void mask_tail(Stage& s, int kw, int kbase, uint32_t 
     }
 }
 
-template <bool STORE_C, bool SIGN_PACK>
+template <bool STORE_C, bool SIGN_PACK, bool ZO>
 __global__ void __launch_bounds__(THREADS, 2)
 xnor_popc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __restrict__ Wp,
                  int ldwp, int M, int N, int K, int32_t* __restrict__ C, int ldc,
@@ -84,6 +85,9 @@ xnor_popc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __re
     for (int i = 0; i < 16; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0;
+    int ones[16];   // (0,1) frames: number of ones in the row
+#pragma unroll
+    for (int i = 0; i < 16; ++i) ones[i] = 0;
 
     load_stage(st[0], Ap, ldap, Wp, ldwp, m0, n0, M, N, kw, 0);
     cp_async_commit();
@@ -104,10 +108,15 @@ xnor_popc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __re
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const uint4 a4 = *reinterpret_cast<const uint4*>(&cur.a[wy * 16 + i][q * 4]);
+                if (ZO) ones[i] += __popc(a4.x) + __popc(a4.y) + __popc(a4.z) + __popc(a4.w);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    acc[i][j] += __popc(a4.x ^ w4[j].x) + __popc(a4.y ^ w4[j].y) +
-                                 __popc(a4.z ^ w4[j].z) + __popc(a4.w ^ w4[j].w);
+                    if (ZO)
+                        acc[i][j] += __popc(a4.x & w4[j].x) + __popc(a4.y & w4[j].y) +
+                                     __popc(a4.z & w4[j].z) + __popc(a4.w & w4[j].w);
+                    else
+                        acc[i][j] += __popc(a4.x ^ w4[j].x) + __popc(a4.y ^ w4[j].y) +
+                                     __popc(a4.z ^ w4[j].z) + __popc(a4.w ^ w4[j].w);
                 }
             }
         }
@@ -132,7 +141,7 @@ xnor_popc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __re
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int n = n0 + lane + 32 * j;
-            const int d = K - 2 * acc[i][j];
+            const int d = ZO ? 2 * acc[i][j] - ones[i] : K - 2 * acc[i][j];
             if (STORE_C) {
                 if (m < M && n < N) C[(size_t)m * ldc + n] = d;
             }
@@ -161,17 +170,25 @@ xnor_popc_kernel(const uint32_t* __restrict__ Ap, int ldap, const uint32_t* __re
 
 }  // namespace
 
-int launch_xnor_popc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
-                     int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
-                     uint32_t* out_bits, int ldob, cudaStream_t st) {
-    dim3 grid(ceil_div(M, BM), ceil_div(N, BN));
+template <bool ZO>
+static void launch_zo(dim3 grid, const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
+                      int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
+                      uint32_t* out_bits, int ldob, cudaStream_t st) {
     const bool sp = out_bits != nullptr;
     if (C && sp)
-        xnor_popc_kernel<true, true><<<grid, THREADS, 0, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob);
+        xnor_popc_kernel<true, true, ZO><<<grid, THREADS, 0, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob);
     else if (C)
-        xnor_popc_kernel<true, false><<<grid, THREADS, 0, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob);
+        xnor_popc_kernel<true, false, ZO><<<grid, THREADS, 0, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob);
     else
-        xnor_popc_kernel<false, true><<<grid, THREADS, 0, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob);
+        xnor_popc_kernel<false, true, ZO><<<grid, THREADS, 0, st>>>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob);
+}
+
+int launch_xnor_popc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
+                     int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
+                     uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
+    dim3 grid(ceil_div(M, BM), ceil_div(N, BN));
+    if (zo) launch_zo<true>(grid, Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
+    else launch_zo<false>(grid, Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
     return launch_status();
 }
 

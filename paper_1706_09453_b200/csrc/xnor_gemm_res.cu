@@ -98,6 +98,7 @@ struct ProducerArgs {
     int my_tiles, nks, kw;
     uint32_t tmask;
     int lane;
+    int zo;               // the frame operand's bits stand for (0,1) instead of (-1,+1)
 };
 
 // Producer of the frame operand: thread = row `r` of every tile of this CTA; team `team`
@@ -129,7 +130,15 @@ __device__ __forceinline__ void produce_a(const ProducerArgs& a, int r, int team
         // 32-bit column 4c + t of the stage = word t of chunk c: the byte order of the
         // K-major shared-memory layout of the other operand
         uint32_t wr[32];
-        if (ragged && ks == a.nks - 1) {
+        if (a.zo) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const int g = 8 * ks + c;   // index of the word in the row
+                const uint32_t valid = (!ragged || g < a.kw - 1) ? 0xFFFFFFFFu : (g == a.kw - 1 ? a.tmask : 0u);
+                const uint4 o = widen01_masked(w[c], valid);
+                wr[4 * c] = o.x; wr[4 * c + 1] = o.y; wr[4 * c + 2] = o.z; wr[4 * c + 3] = o.w;
+            }
+        } else if (ragged && ks == a.nks - 1) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const int g = 8 * ks + c;   // index of the word in the row
@@ -167,7 +176,7 @@ template <int BN>
 __global__ void __launch_bounds__(THREADS, 1)
 xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restrict__ img,
                 int M, int N, int K, const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
-                uint32_t* __restrict__ out_bits, int ldob, int* __restrict__ status) {
+                uint32_t* __restrict__ out_bits, int ldob, int zo, int* __restrict__ status) {
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -261,7 +270,7 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
         }
         __syncwarp();
     } else if (warp >= PROD_WARP0) {
-        ProducerArgs pa{smem_u32(smem) + B_REGION, tmem + C::TMEM_A_COL, ctl, abort_flag, share.count, nks, kw, tail_mask(K), lane};
+        ProducerArgs pa{smem_u32(smem) + B_REGION, tmem + C::TMEM_A_COL, ctl, abort_flag, share.count, nks, kw, tail_mask(K), lane, zo};
         produce_a<C::A_STAGES>(pa, (warp & 3) * 32 + lane, (warp - PROD_WARP0) / A_WARPS);
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issue: one thread
@@ -359,7 +368,7 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
 
 template <int BN>
 int launch_bn(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
-              const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int sm_count, cudaStream_t st) {
+              const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int zo, int sm_count, cudaStream_t st) {
     auto kern = xnor_res_kernel<BN>;
     static bool configured = false;
     if (!configured) {
@@ -372,7 +381,7 @@ int launch_bn(const uint32_t* Ap, int ldap, const void* image, int M, int N, int
     if (!status) return BNN_ERR_CUDA;
     CUtensorMap mapA;
     if (!encode_packed_map(&mapA, Ap, ldap, M, K, BM)) return BNN_ERR_CUDA;
-    kern<<<grid, THREADS, SMEM_BYTES, st>>>(mapA, static_cast<const uint8_t*>(image), M, N, K, thr, flip, out_bits, ldob, status);
+    kern<<<grid, THREADS, SMEM_BYTES, st>>>(mapA, static_cast<const uint8_t*>(image), M, N, K, thr, flip, out_bits, ldob, zo, status);
     return launch_status();
 }
 
@@ -404,12 +413,12 @@ bool xnor_res_applicable(int N, int K) {
 }
 
 int launch_xnor_res(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
-                    const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, cudaStream_t st) {
+                    const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
     const int sms = sm_count_of_device();
     if (sms <= 0) return BNN_ERR_CUDA;
     const int bn = tile_units(N, K, sms);
-    if (bn == 192) return launch_bn<192>(Ap, ldap, image, M, N, K, thr, flip, out_bits, ldob, sms, st);
-    if (bn == 128) return launch_bn<128>(Ap, ldap, image, M, N, K, thr, flip, out_bits, ldob, sms, st);
+    if (bn == 192) return launch_bn<192>(Ap, ldap, image, M, N, K, thr, flip, out_bits, ldob, zo, sms, st);
+    if (bn == 128) return launch_bn<128>(Ap, ldap, image, M, N, K, thr, flip, out_bits, ldob, zo, sms, st);
     return BNN_ERR_UNSUPPORTED;
 }
 

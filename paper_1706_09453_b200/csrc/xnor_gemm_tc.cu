@@ -84,12 +84,21 @@ struct ProducerArgs {
     int tiles, nks, kw;
     uint32_t tmask;
     int lane;
+    int zo;               // the frame operand's bits stand for (0,1) instead of (-1,+1)
 };
 
 // The eight 16-byte chunks of one widened row and stage; `ks` is the stage's index in the row.
+template <bool FRAMES>
 __device__ __forceinline__ void widen_stage(const ProducerArgs& a, bool ragged, int ks, const uint4& v0, const uint4& v1, uint4 (&o)[8]) {
     const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-    if (ragged && ks == a.nks - 1) {
+    if (FRAMES && a.zo) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int g = 8 * ks + c;   // index of the word in the row
+            const uint32_t valid = (!ragged || g < a.kw - 1) ? 0xFFFFFFFFu : (g == a.kw - 1 ? a.tmask : 0u);
+            o[c] = widen01_masked(w[c], valid);
+        }
+    } else if (ragged && ks == a.nks - 1) {
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
             const int g = 8 * ks + c;   // index of the word in the row
@@ -126,7 +135,7 @@ __device__ __forceinline__ void produce_a(const ProducerArgs& a, int r) {
         const uint4 v1 = lds128u(src + (((2u * gi + 1u) ^ sw) << 4));
         if (!warp_wait(smem_u32(&ctl->empty_a[s]), ph, a.abort_flag, a.lane)) break;
         uint4 o[8];
-        widen_stage(a, ragged, ks, v0, v1, o);
+        widen_stage<true>(a, ragged, ks, v0, v1, o);
         // 32-bit column 4c + t of the stage = word t of chunk c: the byte order of the
         // K-major shared-memory layout of the other operand
         uint32_t wr[32];
@@ -176,12 +185,12 @@ __device__ __forceinline__ void produce_b(const ProducerArgs& a, int r) {
         const uint32_t ph2 = s + 1 == B_STAGES ? ph ^ 1u : ph;
         if (!warp_wait(smem_u32(&ctl->empty_b[s]), ph, a.abort_flag, a.lane)) break;
         uint4 o[8];
-        widen_stage(a, ragged, 2 * kg, v0, v1, o);
+        widen_stage<false>(a, ragged, 2 * kg, v0, v1, o);
 #pragma unroll
         for (int c = 0; c < 8; ++c) sts128(dst0 + s * STAGE_BYTES + c * (BN * 16), o[c].x, o[c].y, o[c].z, o[c].w);
         if (two) {
             if (!warp_wait(smem_u32(&ctl->empty_b[s2]), ph2, a.abort_flag, a.lane)) break;
-            widen_stage(a, ragged, 2 * kg + 1, v2, v3, o);
+            widen_stage<false>(a, ragged, 2 * kg + 1, v2, v3, o);
 #pragma unroll
             for (int c = 0; c < 8; ++c) sts128(dst0 + s2 * STAGE_BYTES + c * (BN * 16), o[c].x, o[c].y, o[c].z, o[c].w);
         }
@@ -204,7 +213,7 @@ __global__ void __launch_bounds__(THREADS, 1)
 xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 int M, int N, int K, int32_t* __restrict__ C, int ldc,
                 const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
-                uint32_t* __restrict__ out_bits, int ldob, int* __restrict__ status) {
+                uint32_t* __restrict__ out_bits, int ldob, int zo, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(smem + B_STAGES * STAGE_BYTES + GROUPS * GROUP_BYTES);
@@ -259,7 +268,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     tc_fence_after_sync();
 
     if (warp >= PROD_WARP0) {
-        ProducerArgs pa{smem_u32(smem), tmem, ctl, abort_flag, tiles, nks, kw, tail_mask(K), lane};
+        ProducerArgs pa{smem_u32(smem), tmem, ctl, abort_flag, tiles, nks, kw, tail_mask(K), lane, zo};
         if (warp == TMA_WARP) {
             // ---------------- one thread feeds the staging ring, a group of two stages at a time
             if (lane == 0) {
@@ -438,7 +447,7 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 template <bool STORE_C, bool SIGN_PACK>
 int launch_variant(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N, int K,
                    int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
-                   uint32_t* out_bits, int ldob, cudaStream_t st) {
+                   uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
     auto kern = xnor_tc_kernel<STORE_C, SIGN_PACK>;
     constexpr int SMEM = smem_bytes<STORE_C>();
     static bool configured = false;
@@ -460,7 +469,7 @@ int launch_variant(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, i
     CUtensorMap mapA, mapB;
     if (!encode_packed_map(&mapA, Ap, ldap, M, K, BM) || !encode_packed_map(&mapB, Wp, ldwp, N, K, BN))
         return BNN_ERR_CUDA;
-    kern<<<grid, THREADS, SMEM, st>>>(mapA, mapB, M, N, K, C, ldc, thr, flip, out_bits, ldob, status);
+    kern<<<grid, THREADS, SMEM, st>>>(mapA, mapB, M, N, K, C, ldc, thr, flip, out_bits, ldob, zo, status);
     return launch_status();
 }
 
@@ -468,11 +477,11 @@ int launch_variant(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, i
 
 int launch_xnor_tc(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N,
                    int K, int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
-                   uint32_t* out_bits, int ldob, cudaStream_t st) {
+                   uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
     const bool sp = out_bits != nullptr;
-    if (C && sp) return launch_variant<true, true>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
-    if (C) return launch_variant<true, false>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
-    return launch_variant<false, true>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, st);
+    if (C && sp) return launch_variant<true, true>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, zo, st);
+    if (C) return launch_variant<true, false>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, zo, st);
+    return launch_variant<false, true>(Ap, ldap, Wp, ldwp, M, N, K, C, ldc, thr, flip, out_bits, ldob, zo, st);
 }
 
 }  // namespace bnn

@@ -1,5 +1,5 @@
 // Widening of packed sign bits to the 4-bit float e2m1 (+1 = nibble 0x2, -1 = nibble 0xA,
-// nothing = nibble 0x0), shared by the XNOR tensor-core kernels, and the constant of the
+// nothing = nibble 0x0; for activations that stand for (0,1): 1 = nibble 0x2, 0 = nibble 0x0), shared by the XNOR tensor-core kernels, and the constant of the
 // float -> integer trick their epilogues use.
 #pragma once
 
@@ -23,5 +23,11 @@ __device__ __forceinline__ uint4 widen_masked(uint32_t w, uint32_t valid) {
     o.w &= ((valid >> 3) & 0x11111111u) * 15u;
     return o;
 }
+
+// Activations in (0,1): bit 1 -> nibble 0x2 (+1), bit 0 -> nibble 0x0 (+0).
+__device__ __forceinline__ uint4 widen01(uint32_t w) {
+    return make_uint4((w << 1) & 0x22222222u, w & 0x22222222u, (w >> 1) & 0x22222222u, (w >> 2) & 0x22222222u);
+}
+__device__ __forceinline__ uint4 widen01_masked(uint32_t w, uint32_t valid) { return widen01(w & valid); }
 
 }  // namespace bnn

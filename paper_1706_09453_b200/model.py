@@ -26,7 +26,8 @@ def words_to_numpy(t: torch.Tensor, k: int) -> np.ndarray:
 
 
 class DeviceNet:
-    def __init__(self, net: wl.Model, sign_mode=B.SIGN_ZERO_POS, device="cuda:0", prepare_xnor=True):
+    def __init__(self, net: wl.Model, sign_mode=B.SIGN_ZERO_POS, device="cuda:0", prepare_xnor=True,
+                 act_values=B.VALUES_PM1):
         cfg = net.cfg
         self.cfg, self.sign_mode, self.device = cfg, sign_mode, device
         self.Wp, self.scale, self.shift, self.thr, self.flip, self.Wimg = [], [], [], [], [], []
@@ -62,7 +63,7 @@ class DeviceNet:
         B.bnn_output_prepare(self.Wout, self.Wout_prepared)
         layers.append(dict(kind=B.LAYER_REAL_OUT, K=cfg.hidden, N=cfg.classes, W=self.Wout,
                            W_prepared=self.Wout_prepared, shift=self.bout))
-        self.desc = B.ModelDesc(layers, sign_mode)
+        self.desc = B.ModelDesc(layers, sign_mode, act_values)
         self._ws = None
 
     def workspace(self, M: int) -> torch.Tensor:

@@ -88,6 +88,13 @@ def test_bad_arguments_are_rejected_without_a_launch(lib):
     assert rc("bnn_xnor_gemm_prepared", fake, 4, fake + 16, 1, 1, 32, fake, 1, None, None) == 3
     assert rc("bnn_xnor_gemm_prepared", fake, 4, fake, 1, 1, 32, None, 0, None, None) == 1
     assert rc("bnn_xnor_gemm_prepared", fake, 4, fake, 1, 40, 32, fake, 8, None, None) == 2
+    # (0,1) activations
+    assert rc("bnn_gemm01", fake, 4, None, 0, None, 1, 1, 32, fake, 1, None, None) == 1     # no weights at all
+    assert rc("bnn_gemm01", fake, 4, fake, 4, None, 1, 1, 32, None, 0, None, None) == 1     # no output
+    assert rc("bnn_gemm01", fake, 4, fake, 6, None, 1, 1, 32, fake, 1, None, None) == 3     # weight pitch
+    assert rc("bnn_gemm01", fake, 4, None, 0, fake + 16, 1, 1, 32, fake, 1, None, None) == 3
+    assert rc("bnn_output_layer01", None, 4, fake, 4, None, None, 1, 1, 4, fake, 1, 1, None) == 1
+    assert rc("bnn_output_layer01", fake, 4, fake, 2, None, None, 1, 1, 4, fake, 1, 1, None) == 2
     # options
     assert B.bnn_set_option(B.OPT_XNOR_PATH, B.PATH_CUDA_CORE) == 0
     assert B.bnn_set_option(B.OPT_XNOR_PATH, B.PATH_AUTO) == 1
@@ -119,6 +126,10 @@ def test_model_validation(lib):
     # fan-in mismatch
     bad, keep3 = model(layer(0, 440, 64, 1), layer(1, 32, 64, 1), layer(2, 64, 10))
     assert B.raw_call("bnn_forward", C.byref(bad), fake, 440, 8, fake, 10, fake, 1 << 20, None, None) == 2
+    # unknown activation values
+    odd, keep5 = model(layer(0, 440, 64, 1), layer(1, 64, 64, 1), layer(2, 64, 10))
+    odd.act_values = 7
+    assert B.raw_call("bnn_forward", C.byref(odd), fake, 440, 8, fake, 10, fake, 1 << 20, None, None) == 4
     # last layer must be the real-valued one
     bad, keep4 = model(layer(0, 440, 64, 1), layer(1, 64, 64, 1))
     assert B.raw_call("bnn_forward", C.byref(bad), fake, 440, 8, fake, 10, fake, 1 << 20, None, None) == 4

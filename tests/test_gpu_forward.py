@@ -27,12 +27,12 @@ def env():
     return torch, binding, model
 
 
-def run_binary_net(env, cfg, frames, mode=0, sample=None, prepare_xnor=True):
+def run_binary_net(env, cfg, frames, mode=0, sample=None, prepare_xnor=True, values=0):
     """Runs bnn_forward on `frames` frames; compares the frames in `sample` (all if None)."""
     torch, B, model = env
     net = wl.make_model(cfg)
     X = wl.make_frames(cfg, frames)
-    dn = model.DeviceNet(net, mode, prepare_xnor=prepare_xnor)
+    dn = model.DeviceNet(net, mode, prepare_xnor=prepare_xnor, act_values=values)
     outs = dn.layer_out_buffers(frames)
     logp = dn.forward(model.to_dev(X), layer_out=outs)
     torch.cuda.synchronize()
@@ -41,7 +41,7 @@ def run_binary_net(env, cfg, frames, mode=0, sample=None, prepare_xnor=True):
     glogp = logp.cpu().numpy()[idx]
     # the packed weights themselves (Eq. 3 on the GPU) must equal the oracle's
     ref = o.forward(X[idx], net.W, net.scale, net.shift, net.Wout, net.bout, o.ACT_SIGN, mode,
-                    layer1_bits=gbits[0])
+                    layer1_bits=gbits[0], values=values)
     for l, wp in enumerate(dn.Wp):
         np.testing.assert_array_equal(model.words_to_numpy(wp, net.W[l].shape[1]), ref["Wp"][l])
     # (1) first layer: equal outside the tolerance band
@@ -70,6 +70,27 @@ def test_forward_tiny_config_all_frames(env):
 def test_forward_tiny_config_weights_widened_on_the_fly(env):
     """The model without prepared images of the hidden layers' weights (bnn_xnor_gemm's kernel)."""
     run_binary_net(env, wl.CONFIGS["tiny"], 256, prepare_xnor=False)
+
+
+def test_forward_tiny_config_01_activations(env):
+    """Hidden activations in (0,1) instead of (-1,+1) (Section 3.2), on every XNOR kernel."""
+    B = env[1]
+    run_binary_net(env, wl.CONFIGS["tiny"], 256, values=1)
+    run_binary_net(env, wl.CONFIGS["tiny"], 200, values=1, prepare_xnor=False, mode=1)
+    prev = B.bnn_set_xnor_path(B.XNOR_POPC)
+    try:
+        run_binary_net(env, wl.CONFIGS["tiny"], 131, values=1)
+    finally:
+        B.bnn_set_xnor_path(prev)
+    assert B.bnn_device_status() == 0
+
+
+def test_forward_wsj_config_01_activations_sampled_frames(env):
+    cfg = wl.CONFIGS["wsj"]
+    rng = np.random.default_rng(2)
+    sample = np.unique(np.concatenate([np.arange(64), np.arange(cfg.frames - 64, cfg.frames),
+                                       rng.integers(0, cfg.frames, 200)]))
+    run_binary_net(env, cfg, cfg.frames, sample=sample, values=1)
 
 
 def test_forward_tiny_config_popcount_path(env):

@@ -264,6 +264,82 @@ def test_xnor_gemm_full_size_every_output_on_repeated_launches(B, torch_, shape,
     assert B.bnn_device_status() == 0, "a tensor-core kernel gave up on a bounded wait"
 
 
+# ------------------------------------------------------------------ (0,1) activations (Section 3.2)
+def run_gemm01(B, path, h_dev, w_dev, k, **kw):
+    """bnn_gemm01 with packed weights, or (path "prepared") with their prepared image only."""
+    if path != "prepared":
+        return B.bnn_gemm01(h_dev, w_dev, k, **kw)
+    import torch
+    n = w_dev.shape[0]
+    image = torch.empty(B.bnn_xnor_prepared_bytes(n, k), dtype=torch.uint8, device="cuda:0")
+    B.bnn_xnor_prepare(w_dev, k, image)
+    B.bnn_gemm01(h_dev, None, k, N=n, prepared=image, **kw)
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1), (5, 7, 33), (129, 130, 127), (300, 257, 1000), (256, 1024, 1024),
+                                   (131, 1024, 440), (100, 520, 4100), (700, 200, 3000)])
+@pytest.mark.parametrize("p", [0.5, 0.1])
+def test_gemm01_int32_bit_exact(B, torch_, xnor_path, shape, p):
+    m, n, k = shape
+    hp = wl.make_bit_planes(m, k, p, [7, m, n, k], B.packed_pitch(k))
+    wp = wl.make_bit_planes(n, k, 0.5, [8, m, n, k], B.packed_pitch(k))
+    # garbage in the pad bits of the frame operand must not count as ones
+    kw = (k + 31) // 32
+    hp_dirty = hp.copy()
+    if k % 32:
+        hp_dirty[:, kw - 1] |= np.uint32((0xFFFFFFFF << (k % 32)) & 0xFFFFFFFF)
+    hp_dirty[:, kw:] = 0xFFFFFFFF
+    c = torch_.full((m, n + 5), -77, dtype=torch_.int32, device="cuda:0")
+    run_gemm01(B, xnor_path, dev(hp_dirty), dev(wp), k, C_out=c[:, :n])
+    got = c.cpu().numpy()
+    np.testing.assert_array_equal(got[:, :n], o.gemm01(hp, wp, k))
+    np.testing.assert_array_equal(got[:, n:], -77)
+
+
+@pytest.mark.parametrize("shape", [(5, 7, 33), (300, 257, 1000), (256, 1024, 1024), (2100, 2048, 2048), (700, 200, 3000),
+                                   (150, 200, 5000)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_gemm01_fused_sign_pack_bit_exact(B, torch_, xnor_path, shape, mode):
+    m, n, k = shape
+    rng = np.random.default_rng(m + n + k)
+    hp = wl.make_bit_planes(m, k, 0.5, [9, m, n, k], B.packed_pitch(k))
+    wp = wl.make_bit_planes(n, k, 0.5, [10, m, n, k], B.packed_pitch(k))
+    scale = rng.uniform(0.5, 1.5, n).astype(np.float32)
+    shift = rng.normal(0, 0.1, n).astype(np.float32)
+    scale[::7] *= -1
+    shift[2::5] = np.round(shift[2::5] * 20)
+    scale[2::5] = 1.0
+    thr = torch_.empty(n, dtype=torch_.int32, device="cuda:0")
+    flip = torch_.empty((n + 31) // 32, dtype=torch_.int32, device="cuda:0")
+    B.bnn_fold_thresholds(dev(scale), dev(shift), n, k, thr, flip, mode)
+    out = packed_canary(torch_, m, n, B)
+    run_gemm01(B, xnor_path, dev(hp), dev(wp), k, thr=thr, flip=flip, out_bits=out[:, :B.packed_pitch(n)])
+    want = o.affine_sign_pack_i32(o.gemm01(hp, wp, k), scale, shift, mode)
+    got = out.cpu().numpy().view(np.uint32)
+    nw = (n + 31) // 32
+    np.testing.assert_array_equal(got[:, :nw], want)
+    np.testing.assert_array_equal(got[:, nw:], 0x5A5A5A5A)
+
+
+@pytest.mark.parametrize("c,m,h", [(2000, 70, 1024), (300, 1100, 1000), (129, 513, 33)])
+def test_output_layer_01_activations(B, torch_, real_path, c, m, h):
+    rng = np.random.default_rng(c + 1)
+    hp = wl.make_bit_planes(m, h, 0.5, 41, B.packed_pitch(h))
+    wout = rng.normal(0, 1 / np.sqrt(h), (c, h)).astype(np.float32)
+    b = rng.normal(0, 0.1, c).astype(np.float32)
+    prep = None
+    if real_path != "fp32":
+        prep = torch_.empty(B.bnn_output_prepared_bytes(c, h), dtype=torch_.uint8, device="cuda:0")
+        B.bnn_output_prepare(dev(wout), prep)
+    z = torch_.empty((m, c), dtype=torch_.float32, device="cuda:0")
+    B.bnn_output_layer(dev(wout), dev(b), z, h, Hp=dev(hp), log_softmax=False, prepared=prep, values=B.VALUES_01)
+    zr = o.real_gemm_bits01(hp, wout, b, h)
+    assert np.abs(z.cpu().numpy() - zr).max() <= FLOAT_TOL * h
+    lp = torch_.empty((m, c), dtype=torch_.float32, device="cuda:0")
+    B.bnn_output_layer(dev(wout), dev(b), lp, h, Hp=dev(hp), prepared=prep, values=B.VALUES_01)
+    assert np.abs(lp.cpu().numpy() - o.log_softmax(zr)).max() <= LOGP_TOL
+
+
 # ------------------------------------------------------------------ +-1 weights x real input
 @pytest.mark.parametrize("shape", [(1, 1, 1), (3, 5, 33), (130, 129, 440), (257, 300, 600), (64, 256, 2048),
                                    (20000, 260, 70), (300, 1300, 100)])
