@@ -274,10 +274,20 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
         produce_a<C::A_STAGES>(pa, (warp & 3) * 32 + lane, (warp - PROD_WARP0) / A_WARPS);
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issue: one thread
+        // Two stages per iteration: measured on B200, whatever this thread does between two
+        // MMAs (polls, commits, loop bookkeeping) is time the tensor pipe idles, so the waits
+        // of two stages are taken together and their eight MMAs issued back to back (12 % off
+        // the steady state against one stage per iteration).
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc_mxf4(BM, BN);
             const uint32_t sfa = tmem + C::TMEM_SF_COL, sfb = tmem + C::TMEM_SF_COL + SF_COLS / 2;
-            int it = 0;
+            // descriptor of stage 0, chunk pair 0; the address field (16-byte units) of the others
+            // is reached by plain additions: the whole region lies below 2^14 * 16 bytes
+            const uint64_t desc0 = smem_desc_kmajor(smem_u32(smem), BN * 16, 128);
+            constexpr uint32_t kStepJ = (2 * BN * 16) >> 4, kStepS = C::B_BYTES >> 4;
+            const uint32_t tmem_a = tmem + C::TMEM_A_COL;
+            int sa = 0;          // slot of the A ring and the parity its `full` barrier shows next
+            uint32_t pa = 0;
             bool ok = true;
             for (int tl = 0; tl < share.count && ok; ++tl) {
                 const int b = tl & 1;
@@ -285,21 +295,43 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d = tmem + (uint32_t)(b * BN);
-                for (int ks = 0; ks < nks; ++ks, ++it) {
-                    const int sa = it % C::A_STAGES;
-                    // the weight stage arrives once (phase 0) and then stays
-                    ok = (tl > 0 || mbar_wait(smem_u32(&ctl->full_b[ks]), 0u, abort_flag)) &&
-                         mbar_wait(smem_u32(&ctl->full_a[sa]), (uint32_t)((it / C::A_STAGES) & 1), abort_flag);
+                uint64_t db = desc0;
+                int ks = 0;
+                for (; ks + 1 < nks; ks += 2) {
+                    const int sa2 = sa + 1 == C::A_STAGES ? 0 : sa + 1;
+                    const uint32_t pa2 = sa + 1 == C::A_STAGES ? pa ^ 1u : pa;
+                    // a weight stage arrives once (phase 0) and then stays
+                    ok = (tl > 0 || (mbar_wait(smem_u32(&ctl->full_b[ks]), 0u, abort_flag) &&
+                                     mbar_wait(smem_u32(&ctl->full_b[ks + 1]), 0u, abort_flag))) &&
+                         mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag) &&
+                         mbar_wait(smem_u32(&ctl->full_a[sa2]), pa2, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t b0 = smem_u32(smem + ks * C::B_BYTES);
-                    const uint32_t ta = tmem + C::TMEM_A_COL + sa * A_COLS;
+                    const uint32_t ta = tmem_a + sa * A_COLS, ta2 = tmem_a + sa2 * A_COLS;
 #pragma unroll
-                    for (int j = 0; j < BK / 64; ++j) {   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
-                        const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (BN * 16), BN * 16, 128);
-                        mma_mxf4_ts(d, ta + 8 * j, db, idesc, sfa, sfb, (ks | j) != 0);
-                    }
+                    for (int j = 0; j < BK / 64; ++j)   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
+                        mma_mxf4_ts(d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
                     mma_commit(smem_u32(&ctl->empty_a[sa]));
+#pragma unroll
+                    for (int j = 0; j < BK / 64; ++j)
+                        mma_mxf4_ts(d, ta2 + 8 * j, db + kStepS + j * kStepJ, idesc, sfa, sfb, 1u);
+                    mma_commit(smem_u32(&ctl->empty_a[sa2]));
+                    db += 2 * kStepS;
+                    sa = sa2; pa = pa2;
+                    if (++sa == C::A_STAGES) { sa = 0; pa ^= 1u; }
+                }
+                if (ok && ks < nks) {   // odd number of stages: the last one alone
+                    ok = (tl > 0 || mbar_wait(smem_u32(&ctl->full_b[ks]), 0u, abort_flag)) &&
+                         mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        const uint32_t ta = tmem_a + sa * A_COLS;
+#pragma unroll
+                        for (int j = 0; j < BK / 64; ++j)
+                            mma_mxf4_ts(d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
+                        mma_commit(smem_u32(&ctl->empty_a[sa]));
+                        if (++sa == C::A_STAGES) { sa = 0; pa ^= 1u; }
+                    }
                 }
                 if (ok) mma_commit(smem_u32(&ctl->acc_full[b]));
             }
