@@ -105,10 +105,12 @@ __global__ void out_split_kernel(const float* __restrict__ W, int ldw, int C, in
 }
 
 // ---- the GEMM ---------------------------------------------------------------------------
+// ZO: the activation bits stand for (0,1) instead of (-1,+1).
+template <bool ZO>
 __global__ void __launch_bounds__(THREADS, 1)
 out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restrict__ img,
               const float* __restrict__ rs, const float* __restrict__ bias,
-              int M, int C, int H, float* __restrict__ Z, int ldz, int zo, int* __restrict__ status) {
+              int M, int C, int H, float* __restrict__ Z, int ldz, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES);
@@ -183,8 +185,7 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
             for (int q = 0; q < 2; ++q) {
                 const uint32_t nw = ~cur[q];
                 uint32_t wv[16];
-#pragma unroll
-                if (zo) {   // (0,1) activations: 1.0 (0x3C00) where the bit is set, +0 elsewhere
+                if (ZO) {   // (0,1) activations: 1.0 (0x3C00) where the bit is set, +0 elsewhere
 #pragma unroll
                     for (int t = 0; t < 16; ++t) wv[t] = ((cur[q] >> t) & 0x00010001u) * 0x3C00u;
                 } else {
@@ -305,7 +306,8 @@ int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const floa
     static int sms = 0;
     if (!configured) {
         int dev = 0;
-        if (cudaFuncSetAttribute(out_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        if (cudaFuncSetAttribute(out_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(out_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
             cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return BNN_ERR_CUDA;
@@ -317,7 +319,10 @@ int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const floa
     const int tiles = ct * ceil_div(M, FN);
     int* status = tc_status_ptr();
     if (!status) return BNN_ERR_CUDA;
-    out_tc_kernel<<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(Hp, ldhp, img, rs, bias, M, C, H, Z, ldz, zo, status);
+    if (zo)
+        out_tc_kernel<true><<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(Hp, ldhp, img, rs, bias, M, C, H, Z, ldz, status);
+    else
+        out_tc_kernel<false><<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(Hp, ldhp, img, rs, bias, M, C, H, Z, ldz, status);
     return launch_status();
 }
 
