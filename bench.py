@@ -234,6 +234,10 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
     if real_path == "tensor" and cfg.act == 1:
         rows.append(dict(name="output_gemm", kernel="out_tc_kernel", work=owork, unit="TFLOP/s", bound="tensor",
                          peak=peaks["bf16_tflops_sustained"], passes=2))
+    elif real_path == "tensor":
+        # fp32 activations: both operands in two fp16 terms, three MMAs per step
+        rows.append(dict(name="output_gemm", kernel="h_split_kernel+outf_tc_kernel", work=owork, unit="TFLOP/s",
+                         bound="tensor", peak=peaks["bf16_tflops_sustained"], passes=3))
     else:
         rows.append(dict(name="output_gemm", kernel="real_gemm_kernel", work=owork, unit="TFLOP/s", bound="alu",
                          peak=fp32_peak))

@@ -53,8 +53,8 @@ typedef enum {
 typedef enum { BNN_SIGN_ZERO_POS = 0, BNN_SIGN_ZERO_NEG = 1 } bnn_sign_mode;
 
 /* What a stored bit of a binarised ACTIVATION matrix stands for in the layer that reads it.
- * The paper works with the pair (-1,+1) and also reports binary activations in (0,1), "the
- * hard version of Sigmoid" (Section 3.2, Table 3; Section 3.3, Table 4).  The decision that
+ * The paper works with the pair (-1,+1) and also reports binary activations in (0,1), which it
+ * likens to a Sigmoid with a hard step (Section 3.2, Table 3; Section 3.3, Table 4).  The decision that
  * sets the bit is the same in both (pre-activation positive, or zero under
  * BNN_SIGN_ZERO_POS); only the value the next layer multiplies differs.  Weights are always
  * (-1,+1): the paper's (0,1) weights did not train (Table 3). */
@@ -209,6 +209,20 @@ BNN_API int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, 
                                const float* b, const void* prepared, int M, int C, int H,
                                float* logp, int ldo, int log_softmax, void* stream);
 
+/* bnn_output_layer on fp32 activations (the last hidden layer of a binary-weights-only network,
+ * Algorithm 1) with scratch.  With `prepared` and a `workspace` (device, 256-byte aligned) of at
+ * least bnn_output_workspace_bytes(M, H) bytes the product runs on the tensor cores: the
+ * activations are split once per call into two fp16 terms (scratch image), the weights are the
+ * two fp16 terms of `prepared`, three MMAs per step:
+ *   |z - exact| <= ~3 * 2^-22 * sum_h |Hf[m][h]| |Wout[c][h]|  (+ fp32 accumulation rounding).
+ * Activations must be finite with |Hf| < 65504 (hardtanh outputs lie in [-1, 1]).  Without
+ * `prepared` or with too little workspace it behaves exactly like bnn_output_layer (FP32 pipe). */
+BNN_API size_t bnn_output_workspace_bytes(int M, int H);
+BNN_API int bnn_output_layer_ws(const float* Hf, int ldhf, const float* Wout, int ldw,
+                                const float* b, const void* prepared, int M, int C, int H,
+                                float* logp, int ldo, int log_softmax,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
 /* One-time preparation of the top layer's weights for the tensor cores: each class row is
  * scaled by a power of two and split into two fp16 terms (about 22 significant bits), stored
  * in the order the MMA reads shared memory.  prepared : device buffer, 256-byte aligned, of
@@ -253,7 +267,8 @@ typedef struct bnn_model {
 
 /* Bytes of scratch for M frames.  bnn_forward_workspace_bytes is what makes bnn_forward
  * fastest: two ping-pong activation buffers plus the split-activation image of the widest
- * sign-weight layer (see bnn_signw_gemm_ws).  bnn_forward_min_workspace_bytes is the least it
+ * sign-weight layer (see bnn_signw_gemm_ws) or of a top layer fed with fp32 activations (see
+ * bnn_output_layer_ws).  bnn_forward_min_workspace_bytes is the least it
  * accepts (the two buffers only; sign-weight layers then run without the image). */
 BNN_API size_t bnn_forward_workspace_bytes(const bnn_model* model, int M);
 BNN_API size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M);

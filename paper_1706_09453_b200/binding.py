@@ -103,6 +103,10 @@ def lib():
         L.bnn_output_layer.argtypes = [p, i, p, i, p, i, p, p, i, i, i, p, i, i, p]
         L.bnn_output_layer01.argtypes = [p, i, p, i, p, p, i, i, i, p, i, i, p]
         L.bnn_output_layer01.restype = C.c_int
+        L.bnn_output_workspace_bytes.argtypes = [i, i]
+        L.bnn_output_workspace_bytes.restype = C.c_size_t
+        L.bnn_output_layer_ws.argtypes = [p, i, p, i, p, p, i, i, i, p, i, i, p, C.c_size_t, p]
+        L.bnn_output_layer_ws.restype = C.c_int
         L.bnn_gemm01.argtypes = [p, i, p, i, p, i, i, i, p, i, C.POINTER(Epilogue), p]
         L.bnn_gemm01.restype = C.c_int
         L.bnn_forward.argtypes = [C.POINTER(Model), p, i, i, p, i, p, C.c_size_t, C.POINTER(p), p]
@@ -302,9 +306,22 @@ def bnn_output_prepare(Wout, prepared):
     return prepared
 
 
-def bnn_output_layer(Wout, b, logp, H, Hp=None, Hf=None, log_softmax=True, prepared=None, values=VALUES_PM1):
+def bnn_output_workspace_bytes(M, H) -> int:
+    return int(lib().bnn_output_workspace_bytes(int(M), int(H)))
+
+
+def bnn_output_layer(Wout, b, logp, H, Hp=None, Hf=None, log_softmax=True, prepared=None, values=VALUES_PM1,
+                     workspace=None):
+    """``workspace`` (uint8 CUDA tensor) with fp32 activations ``Hf`` calls bnn_output_layer_ws."""
     m = (Hp if Hp is not None else Hf).shape[0]
     c = Wout.shape[0]
+    if workspace is not None:
+        _check(lib().bnn_output_layer_ws(_ptr(Hf, torch.float32), _ld(Hf), _ptr(Wout, torch.float32), _ld(Wout),
+                                         _ptr(b, torch.float32), _ptr(prepared), m, c, H,
+                                         _ptr(logp, torch.float32), _ld(logp), int(log_softmax),
+                                         _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+               "bnn_output_layer_ws")
+        return logp
     if values == VALUES_01:
         _check(lib().bnn_output_layer01(_ptr(Hp, torch.int32), _ld(Hp), _ptr(Wout, torch.float32), _ld(Wout),
                                         _ptr(b, torch.float32), _ptr(prepared), m, c, H,

@@ -296,7 +296,7 @@ int bnn_output_prepare(const float* Wout, int ldw, int C, int H,
 static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
                              const float* Wout, int ldw, const float* b, const void* prepared,
                              int M, int C, int H, float* logp, int ldo, int log_softmax,
-                             int zo, void* mid_event, void* stream) {
+                             int zo, void* workspace, size_t workspace_bytes, void* mid_event, void* stream) {
     if (int rc = check_dims(M, C, H)) return rc;
     if (!Wout || !logp) return BNN_ERR_NULL;
     if ((Hp == nullptr) == (Hf == nullptr)) return Hp ? BNN_ERR_UNSUPPORTED : BNN_ERR_NULL;
@@ -318,6 +318,9 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
     int rc;
     if (Hp && prepared && g_real_path != BNN_PATH_CUDA_CORE)
         rc = launch_out_tc(Hp, ldhp, prepared, b, M, C, H, logp, ldo, zo, (cudaStream_t)stream);
+    else if (Hf && prepared && g_real_path != BNN_PATH_CUDA_CORE && workspace &&
+             !(reinterpret_cast<uintptr_t>(workspace) & 255u) && workspace_bytes >= outf_image_bytes(M, H))
+        rc = launch_outf_tc(Hf, ldhf, prepared, b, M, C, H, logp, ldo, workspace, (cudaStream_t)stream);
     else
         rc = launch_real_gemm(a, (cudaStream_t)stream);
     if (rc) return rc;
@@ -332,7 +335,20 @@ int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
                      int M, int C, int H, float* logp, int ldo, int log_softmax,
                      void* stream) {
     return output_layer_impl(Hp, ldhp, Hf, ldhf, Wout, ldw, b, prepared, M, C, H, logp, ldo,
-                             log_softmax, 0, nullptr, stream);
+                             log_softmax, 0, nullptr, 0, nullptr, stream);
+}
+
+size_t bnn_output_workspace_bytes(int M, int H) {
+    if (M < 1 || H < 1) return 0;
+    return outf_image_bytes(M, H);
+}
+
+int bnn_output_layer_ws(const float* Hf, int ldhf, const float* Wout, int ldw, const float* b,
+                        const void* prepared, int M, int C, int H, float* logp, int ldo,
+                        int log_softmax, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!Hf) return BNN_ERR_NULL;
+    return output_layer_impl(nullptr, 0, Hf, ldhf, Wout, ldw, b, prepared, M, C, H, logp, ldo,
+                             log_softmax, 0, workspace, workspace_bytes, nullptr, stream);
 }
 
 int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw, const float* b,
@@ -340,7 +356,7 @@ int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw,
                        int log_softmax, void* stream) {
     if (!Hp) return BNN_ERR_NULL;
     return output_layer_impl(Hp, ldhp, nullptr, 0, Wout, ldw, b, prepared, M, C, H, logp, ldo,
-                             log_softmax, 1, nullptr, stream);
+                             log_softmax, 1, nullptr, 0, nullptr, stream);
 }
 
 size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M) {
@@ -357,11 +373,15 @@ size_t bnn_forward_workspace_bytes(const bnn_model* model, int M) {
     const size_t base = bnn_forward_min_workspace_bytes(model, M);
     if (base == 0) return 0;
     size_t img = 0;
-    for (int l = 0; l < model->n_layers; ++l)
-        if (model->layers[l].kind == BNN_LAYER_SIGNW) {
-            const size_t b = signw_image_bytes(M, model->layers[l].K, 3);  // room for either term count
-            if (b > img) img = b;
-        }
+    for (int l = 0; l < model->n_layers; ++l) {
+        const bnn_layer& y = model->layers[l];
+        size_t b = 0;
+        if (y.kind == BNN_LAYER_SIGNW)
+            b = signw_image_bytes(M, y.K, 3);  // room for either term count
+        else if (y.kind == BNN_LAYER_REAL_OUT && l > 0 && model->layers[l - 1].act == BNN_ACT_HARDTANH)
+            b = outf_image_bytes(M, y.K);      // fp32 activations into the top layer
+        if (b > img) img = b;
+    }
     return base + round256(img);
 }
 
@@ -402,7 +422,7 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
             int rc = output_layer_impl(in_bits ? static_cast<const uint32_t*>(in) : nullptr, in_ld,
                                        in_bits ? nullptr : static_cast<const float*>(in), in_ld,
                                        y.W, y.ldw, y.shift, y.W_prepared, M, y.N, y.K, logp, ldo, 1,
-                                       in_bits && model->act_values == BNN_VALUES_01,
+                                       in_bits && model->act_values == BNN_VALUES_01, img, img_bytes,
                                        events ? events[L + 1] : nullptr, stream);
             if (rc) return rc;
             if (events && events[L] &&

@@ -37,6 +37,34 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
 }
 
+// Programmatic dependent launch, used by the kernel of the binary hidden layers: it starts with
+// pdl_trigger() (the kernel after it in the stream may be scheduled as soon as all CTAs of this
+// one have got that far and SM resources free up), does what does not depend on the kernel
+// before it (set-up, the copy of its weight slice) and calls pdl_wait() before it reads that
+// kernel's output: the wait returns once the kernel before it has completed and its writes are
+// visible.  A kernel of this kind cannot finish before its wait returns, so completion of one
+// implies completion of everything before it in the stream.  (Measured on B200: giving the
+// other kernels of the forward the same treatment, with the wait right after their set-up,
+// made the step 1 % slower instead of faster, so they are launched the ordinary way.)
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Launch with programmatic stream serialisation allowed (see above).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline int launch_status() { return cudaGetLastError() == cudaSuccess ? BNN_OK : BNN_ERR_CUDA; }
@@ -114,6 +142,11 @@ size_t out_prepared_bytes(int C, int H);
 int launch_out_prepare(const float* W, int ldw, int C, int H, void* prepared, cudaStream_t st);
 int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const float* bias,
                   int M, int C, int H, float* Z, int ldz, int zo, cudaStream_t st);
+// The top layer on fp32 activations (finite, |a| < 65504) with both operands split into fp16
+// terms (out_gemm_f32_tc.cu): `workspace` holds outf_image_bytes(M, H) bytes, 256-byte aligned.
+size_t outf_image_bytes(int M, int H);
+int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float* bias,
+                   int M, int C, int H, float* Z, int ldz, void* workspace, cudaStream_t st);
 int launch_log_softmax_rows(float* Z, int ldz, int M, int C, cudaStream_t st);
 
 }  // namespace bnn

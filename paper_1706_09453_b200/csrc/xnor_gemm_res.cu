@@ -183,11 +183,10 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
     Control* ctl = reinterpret_cast<Control*>(smem + B_REGION + GROUPS * GROUP_BYTES);
     volatile int* abort_flag = &ctl->abort;
 
-    // Programmatic dependent launch: the kernel that follows in the stream may be scheduled as
-    // soon as this one's CTAs leave their SMs.  Its own set-up and the copy of its weight slice
-    // need nothing this kernel writes; it waits (griddepcontrol.wait, below) before it touches
-    // the frames.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // The kernel that follows in the stream may be scheduled as soon as this one's CTAs leave
+    // their SMs.  This kernel's own set-up and the copy of its weight slice need nothing the
+    // kernel before it writes; it waits (pdl_wait, below) before it touches the frames.
+    pdl_trigger();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kw = words_for(K);
@@ -271,7 +270,7 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
             }
             // the frames are the previous kernel's output: wait until that kernel has completed
             // and its writes are visible (returns at once when there is no such dependency)
-            asm volatile("griddepcontrol.wait;" ::: "memory");
+            pdl_wait();
             for (; gc < GROUPS && gc < total_groups; ++gc) load_group(gc);
             for (; gc < total_groups; ++gc) {
                 if (!mbar_wait_relaxed(smem_u32(&ctl->group_empty[gc % GROUPS]), (uint32_t)(((gc / GROUPS) - 1) & 1), abort_flag)) break;
@@ -423,23 +422,8 @@ int launch_bn(const uint32_t* Ap, int ldap, const void* image, int M, int N, int
     if (!status) return BNN_ERR_CUDA;
     CUtensorMap mapA;
     if (!encode_packed_map(&mapA, Ap, ldap, M, K, BM)) return BNN_ERR_CUDA;
-    // launched with programmatic stream serialisation: it may start while the kernel before it
-    // in the stream drains (see the kernel's first statement)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(THREADS);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-#ifdef BNN_XNOR_NO_PDL
-    attr[0].val.programmaticStreamSerializationAllowed = 0;
-#else
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-#endif
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, mapA, static_cast<const uint8_t*>(image), M, N, K, thr, flip, out_bits, ldob, zo, status) != cudaSuccess)
+    if (launch_pdl(kern, dim3(grid), dim3(THREADS), SMEM_BYTES, st, mapA, static_cast<const uint8_t*>(image), M, N, K,
+                   thr, flip, out_bits, ldob, zo, status) != cudaSuccess)
         return BNN_ERR_CUDA;
     return launch_status();
 }

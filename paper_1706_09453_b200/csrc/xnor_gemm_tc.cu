@@ -298,34 +298,56 @@ xnor_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             produce_b(pa, (warp - PROD_WARP0 - A_WARPS) * 32 + lane);
         }
     } else if (warp == MMA_WARP) {
-        // ---------------- MMA issue: one thread
+        // ---------------- MMA issue: one thread.  Two stages per iteration: whatever this thread
+        // does between two MMAs (polls, commits, bookkeeping) is time the tensor pipe idles, so
+        // the waits of two stages are taken together and their eight MMAs issued back to back.
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc_mxf4(BM, BN);
             const uint32_t sfa = tmem + TMEM_SF_COL, sfb = tmem + TMEM_SF_COL + SF_COLS / 2;
-            int it = 0;
+            const uint32_t smem0 = smem_u32(smem);
+            int sa = 0, sb = 0;        // ring slots and the parities their `full` barriers show next
+            uint32_t pa = 0, pb = 0;
             int tl = 0;
             bool ok = true;
+            auto issue = [&](uint32_t d, int slot_a, int slot_b, bool first) {
+                const uint32_t b0 = smem0 + slot_b * STAGE_BYTES;
+                const uint32_t ta = tmem + TMEM_A_COL + slot_a * A_COLS;
+#pragma unroll
+                for (int j = 0; j < BK / 64; ++j) {   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
+                    const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (BN * 16), BN * 16, 128);
+                    mma_mxf4_ts(d, ta + 8 * j, db, idesc, sfa, sfb, !(first && j == 0));
+                }
+                mma_commit(smem_u32(&ctl->empty_a[slot_a]));
+                mma_commit(smem_u32(&ctl->empty_b[slot_b]));
+            };
             for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
                 const int b = tl & 1;
                 ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), (uint32_t)(((tl >> 1) & 1) ^ 1), abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d = tmem + (uint32_t)(b * BN);
-                for (int ks = 0; ks < nks; ++ks, ++it) {
-                    const int sa = it % A_STAGES, sb = it % B_STAGES;
-                    ok = mbar_wait(smem_u32(&ctl->full_b[sb]), (uint32_t)((it / B_STAGES) & 1), abort_flag) &&
-                         mbar_wait(smem_u32(&ctl->full_a[sa]), (uint32_t)((it / A_STAGES) & 1), abort_flag);
+                int ks = 0;
+                for (; ks + 1 < nks; ks += 2) {
+                    const int sa2 = sa + 1 == A_STAGES ? 0 : sa + 1, sb2 = sb + 1 == B_STAGES ? 0 : sb + 1;
+                    const uint32_t pa2 = sa + 1 == A_STAGES ? pa ^ 1u : pa, pb2 = sb + 1 == B_STAGES ? pb ^ 1u : pb;
+                    ok = mbar_wait(smem_u32(&ctl->full_b[sb]), pb, abort_flag) && mbar_wait(smem_u32(&ctl->full_b[sb2]), pb2, abort_flag) &&
+                         mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag) && mbar_wait(smem_u32(&ctl->full_a[sa2]), pa2, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t b0 = smem_u32(smem + sb * STAGE_BYTES);
-                    const uint32_t ta = tmem + TMEM_A_COL + sa * A_COLS;
-#pragma unroll
-                    for (int j = 0; j < BK / 64; ++j) {   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
-                        const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (BN * 16), BN * 16, 128);
-                        mma_mxf4_ts(d, ta + 8 * j, db, idesc, sfa, sfb, (ks | j) != 0);
+                    issue(d, sa, sb, ks == 0);
+                    issue(d, sa2, sb2, false);
+                    sa = sa2; pa = pa2; sb = sb2; pb = pb2;
+                    if (++sa == A_STAGES) { sa = 0; pa ^= 1u; }
+                    if (++sb == B_STAGES) { sb = 0; pb ^= 1u; }
+                }
+                if (ok && ks < nks) {   // odd number of stages: the last one alone
+                    ok = mbar_wait(smem_u32(&ctl->full_b[sb]), pb, abort_flag) && mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        issue(d, sa, sb, ks == 0);
+                        if (++sa == A_STAGES) { sa = 0; pa ^= 1u; }
+                        if (++sb == B_STAGES) { sb = 0; pb ^= 1u; }
                     }
-                    mma_commit(smem_u32(&ctl->empty_a[sa]));
-                    mma_commit(smem_u32(&ctl->empty_b[sb]));
                 }
                 if (ok) mma_commit(smem_u32(&ctl->acc_full[b]));
             }

@@ -88,6 +88,10 @@ def test_bad_arguments_are_rejected_without_a_launch(lib):
     assert rc("bnn_xnor_gemm_prepared", fake, 4, fake + 16, 1, 1, 32, fake, 1, None, None) == 3
     assert rc("bnn_xnor_gemm_prepared", fake, 4, fake, 1, 1, 32, None, 0, None, None) == 1
     assert rc("bnn_xnor_gemm_prepared", fake, 4, fake, 1, 40, 32, fake, 8, None, None) == 2
+    # top layer with scratch
+    assert B.bnn_output_workspace_bytes(8192, 2048) == 32 * 64 * 32768
+    assert rc("bnn_output_layer_ws", None, 4, fake, 4, None, None, 1, 1, 4, fake, 1, 1, None, 0, None) == 1
+    assert rc("bnn_output_layer_ws", fake, 2, fake, 4, None, None, 1, 1, 4, fake, 1, 1, None, 0, None) == 2
     # (0,1) activations
     assert rc("bnn_gemm01", fake, 4, None, 0, None, 1, 1, 32, fake, 1, None, None) == 1     # no weights at all
     assert rc("bnn_gemm01", fake, 4, fake, 4, None, 1, 1, 32, None, 0, None, None) == 1     # no output

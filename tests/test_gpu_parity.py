@@ -455,6 +455,34 @@ def test_output_layer_real_activations(B, torch_):
     assert np.abs(lp.cpu().numpy() - want).max() <= LOGP_TOL
 
 
+@pytest.mark.parametrize("m,h,c", [(33, 300, 257), (600, 2048, 3400), (257, 33, 129), (1, 1, 1)])
+def test_output_layer_real_activations_tensor_path(B, torch_, m, h, c):
+    """fp32 activations x fp32 weights with both split into fp16 terms (bnn_output_layer_ws):
+    the operand split costs at most 3 * 2^-22 * sum|a||w|; with the fp32 accumulation of 3 * H
+    products on top the logits are tested at 2^-17 * sum|a||w|, the log-probs at 1e-4."""
+    rng = np.random.default_rng(m + h + c)
+    hf = rng.uniform(-1, 1, (m, h)).astype(np.float32)
+    hf[rng.random(hf.shape) < 0.2] = 1.0          # hardtanh saturates often
+    hf[rng.random(hf.shape) < 0.2] = -1.0
+    hf[0, 0] = np.float32(1e-7)                   # below the fp16 normal range
+    wout = rng.normal(0, 1 / np.sqrt(h), (c, h)).astype(np.float32)
+    b = rng.normal(0, 0.1, c).astype(np.float32)
+    prep = torch_.empty(B.bnn_output_prepared_bytes(c, h), dtype=torch_.uint8, device="cuda:0")
+    B.bnn_output_prepare(dev(wout), prep)
+    ws = torch_.empty(B.bnn_output_workspace_bytes(m, h), dtype=torch_.uint8, device="cuda:0")
+    z = torch_.full((m, c + 1), 9.0, dtype=torch_.float32, device="cuda:0")
+    B.bnn_output_layer(dev(wout), dev(b), z[:, :c], h, Hf=dev(hf), log_softmax=False, prepared=prep, workspace=ws)
+    zr = o.real_gemm_f32(hf, wout, b)
+    bound = 2.0 ** -17 * (np.abs(hf).astype(np.float64) @ np.abs(wout).astype(np.float64).T) + 1e-6
+    got = z.cpu().numpy()
+    assert (np.abs(got[:, :c] - zr) <= bound).all(), np.abs(got[:, :c] - zr).max()
+    np.testing.assert_array_equal(got[:, c], 9.0)
+    lp = torch_.empty((m, c), dtype=torch_.float32, device="cuda:0")
+    B.bnn_output_layer(dev(wout), dev(b), lp, h, Hf=dev(hf), prepared=prep, workspace=ws)
+    assert np.abs(lp.cpu().numpy() - o.log_softmax(zr)).max() <= LOGP_TOL
+    assert B.bnn_device_status() == 0
+
+
 def test_output_layer_wide_dynamic_range_weights(B, torch_):
     """Rows whose magnitudes differ by many orders: the per-row power-of-two scaling of the
     prepared fp16 terms must keep every row accurate."""
