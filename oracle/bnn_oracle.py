@@ -200,8 +200,23 @@ def log_softmax(Z):
     return LP
 
 
+def splice(F, left, right):
+    """Context window of the feature front end (Section 3: frames spliced over a context of 11):
+    row m of the result is the concatenation of rows m - left .. m + right of F; rows outside the
+    matrix are replaced by the nearest existing one (the paper does not say how edges are padded;
+    this is the reading taken).  Written out as plain loops."""
+    F = _f32(F)
+    M, D = F.shape
+    out = np.empty((M, (left + right + 1) * D), dtype=np.float32)
+    for m in range(M):
+        for j, t in enumerate(range(-left, right + 1)):
+            r = min(max(m + t, 0), M - 1)
+            out[m, j * D:(j + 1) * D] = F[r]
+    return out
+
+
 def forward(X, W, scale, shift, Wout, bout, act=ACT_SIGN, mode=SIGN_ZERO_POS,
-            layer1_bits=None, values=VALUES_PM1):
+            layer1_bits=None, values=VALUES_PM1, log_prior=None):
     """Whole forward pass, layer by layer in the order of Algorithms 1 and 2.
 
     W: list of real-valued weight matrices [N_l][K_l]; they are binarised with Eq. 3 first.
@@ -245,4 +260,6 @@ def forward(X, W, scale, shift, Wout, bout, act=ACT_SIGN, mode=SIGN_ZERO_POS,
         Z = real_gemm_f32(Hf, Wout, bout)
     taps["logits"] = Z
     taps["logp"] = log_softmax(Z)
+    if log_prior is not None:   # scaled log-likelihoods for a hybrid decoder: log p(s|x) - log p(s)
+        taps["logp"] = taps["logp"] - np.asarray(log_prior, dtype=np.float64)[None, :]
     return taps

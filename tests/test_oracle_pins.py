@@ -359,3 +359,42 @@ def test_forward_with_01_activations_against_numpy():
     # and it is a different function from the (-1,+1) network on this input
     t2 = o.forward(X, W, [None] * 3, r, Wout, bout, o.ACT_SIGN, o.SIGN_ZERO_NEG)
     assert np.abs(t["logp"] - t2["logp"]).max() > 1e-3
+
+
+# ---------------------------------------------------------------- front and back of a hybrid model
+def test_splice_context_window():
+    """The 11-frame context of Section 3: interior rows are plain concatenations of the
+    neighbouring frames, edges repeat the first / last frame, no context is the identity."""
+    rng = np.random.default_rng(3)
+    F = rng.standard_normal((9, 4)).astype(np.float32)
+    np.testing.assert_array_equal(o.splice(F, 0, 0), F)
+    S = o.splice(F, 2, 1)
+    assert S.shape == (9, 16)
+    np.testing.assert_array_equal(S[4], np.concatenate([F[2], F[3], F[4], F[5]]))
+    np.testing.assert_array_equal(S[0], np.concatenate([F[0], F[0], F[0], F[1]]))
+    np.testing.assert_array_equal(S[1], np.concatenate([F[0], F[0], F[1], F[2]]))
+    np.testing.assert_array_equal(S[8], np.concatenate([F[6], F[7], F[8], F[8]]))
+    # the same window through numpy's own edge padding
+    P = np.pad(F, ((2, 1), (0, 0)), mode="edge")
+    np.testing.assert_array_equal(S, np.concatenate([P[t:t + 9] for t in range(4)], axis=1))
+    # a window longer than the matrix still only repeats existing rows
+    one = o.splice(F[:1], 5, 5)
+    np.testing.assert_array_equal(one, np.tile(F[:1], (1, 11)))
+
+
+def test_forward_log_prior_is_subtracted_from_log_posteriors():
+    rng = np.random.default_rng(6)
+    dims = [12, 20, 16]
+    X = rng.standard_normal((5, dims[0])).astype(np.float32)
+    W = [rng.standard_normal((dims[i + 1], dims[i])).astype(np.float32) for i in range(2)]
+    sc = [np.ones(dims[i + 1], np.float32) for i in range(2)]
+    sh = [np.zeros(dims[i + 1], np.float32) for i in range(2)]
+    Wout = rng.standard_normal((7, dims[-1])).astype(np.float32)
+    bout = rng.standard_normal(7).astype(np.float32)
+    prior = rng.dirichlet(np.ones(7))
+    lp = np.log(prior).astype(np.float32)
+    a = o.forward(X, W, sc, sh, Wout, bout)
+    b = o.forward(X, W, sc, sh, Wout, bout, log_prior=lp)
+    np.testing.assert_allclose(b["logp"], a["logp"] - lp.astype(np.float64)[None, :], atol=1e-12)
+    # posterior / prior, summed with the prior as weights, is 1 again
+    np.testing.assert_allclose((np.exp(b["logp"]) * np.exp(lp.astype(np.float64))).sum(1), 1.0, atol=1e-9)
