@@ -263,6 +263,21 @@ typedef struct bnn_model {
     int sign_mode;
     const bnn_layer* layers; /* HOST array of n_layers entries (device pointers inside) */
     int act_values;          /* bnn_act_values of every BNN_ACT_SIGN_PACK activation */
+    /* Front and back of a hybrid acoustic model, both optional (0, 0, NULL = off).
+     * splice_left/right: the network's input is a window of splice_left + 1 + splice_right
+     * consecutive feature frames (Section 3: 11 frames of 40 filter-bank features).  With a
+     * window, X holds ONE frame per row, K_0 / (left + right + 1) features wide, and input row m
+     * of the first layer is the concatenation of rows m - left .. m + right of X, rows outside
+     * [0, M) replaced by the nearest one (one call = one utterance or chunk of it).  The window
+     * is formed while the first layer loads its input, so the spliced matrix never exists in
+     * memory; this needs the full bnn_forward_workspace_bytes workspace (else
+     * BNN_ERR_WORKSPACE).  The paper only says that the features are spliced; the edge rule is
+     * this library's.
+     * log_prior: device [C] or NULL; subtracted from every row of log-probabilities, which turns
+     * the state posteriors into the scaled likelihoods a hybrid HMM decoder consumes
+     * (the paper decodes with Kaldi, Section 3; it does not print this step). */
+    int splice_left, splice_right;
+    const float* log_prior;
 } bnn_model;
 
 /* Bytes of scratch for M frames.  bnn_forward_workspace_bytes is what makes bnn_forward

@@ -43,7 +43,8 @@ class Layer(C.Structure):
 
 class Model(C.Structure):
     _fields_ = [("n_layers", C.c_int), ("sign_mode", C.c_int), ("layers", C.POINTER(Layer)),
-                ("act_values", C.c_int)]
+                ("act_values", C.c_int), ("splice_left", C.c_int), ("splice_right", C.c_int),
+                ("log_prior", C.c_void_p)]
 
 
 _lib = None
@@ -339,8 +340,8 @@ def bnn_output_layer(Wout, b, logp, H, Hp=None, Hf=None, log_softmax=True, prepa
 class ModelDesc:
     """Host-side bnn_model built from a list of layer dicts; keeps the tensors alive."""
 
-    def __init__(self, layers, sign_mode=SIGN_ZERO_POS, act_values=VALUES_PM1):
-        self._keep = layers
+    def __init__(self, layers, sign_mode=SIGN_ZERO_POS, act_values=VALUES_PM1, splice=(0, 0), log_prior=None):
+        self._keep = (layers, log_prior)
         arr = (Layer * len(layers))()
         for a, d in zip(arr, layers):
             a.kind, a.K, a.N, a.act = d["kind"], d["K"], d["N"], d.get("act", ACT_NONE)
@@ -351,7 +352,7 @@ class ModelDesc:
             a.scale, a.shift = _ptr(d.get("scale"), torch.float32), _ptr(d.get("shift"), torch.float32)
             a.thr, a.flip = _ptr(d.get("thr"), torch.int32), _ptr(d.get("flip"), torch.int32)
         self._arr = arr
-        self.c = Model(len(layers), sign_mode, arr, act_values)
+        self.c = Model(len(layers), sign_mode, arr, act_values, splice[0], splice[1], _ptr(log_prior, torch.float32))
         self.layers = layers
 
     def workspace_bytes(self, M: int) -> int:

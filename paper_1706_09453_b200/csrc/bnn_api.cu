@@ -244,17 +244,21 @@ int bnn_signw_gemm(const float* X, int ldx, const uint32_t* Wp, int ldwp,
     return bnn_signw_gemm_ws(X, ldx, Wp, ldwp, M, N, K, Y, ldy, epi, nullptr, 0, stream);
 }
 
-int bnn_signw_gemm_ws(const float* X, int ldx, const uint32_t* Wp, int ldwp,
+// splice_dim > 0: X is [M][ldx] with splice_dim features per frame and row m of the product's
+// input is the concatenation of frames m - splice_left .. (K / splice_dim frames), clamped to
+// the batch; only the path that splits the activations into a scratch image forms it.
+static int signw_impl(const float* X, int ldx, const uint32_t* Wp, int ldwp,
                       int M, int N, int K, float* Y, int ldy,
                       const bnn_epilogue* epi, void* workspace, size_t workspace_bytes,
-                      void* stream) {
+                      int splice_dim, int splice_left, void* stream) {
     if (int rc = check_dims(M, N, K)) return rc;
     if (!X) return BNN_ERR_NULL;
-    if (ldx < K) return BNN_ERR_SHAPE;
+    if (ldx < (splice_dim > 0 ? splice_dim : K)) return BNN_ERR_SHAPE;
     if (int rc = check_packed(Wp, ldwp, K)) return rc;
     if (Y && ldy < N) return BNN_ERR_SHAPE;
     RealGemmArgs a{};
     a.Af = X; a.lda = ldx; a.Bb = Wp; a.ldb = ldwp;
+    a.splice_dim = splice_dim; a.splice_left = splice_left;
     a.M = M; a.N = N; a.K = K;
     a.Y = Y; a.ldy = ldy;
     a.act = BNN_ACT_NONE; a.sign_mode = BNN_SIGN_ZERO_POS;
@@ -274,9 +278,18 @@ int bnn_signw_gemm_ws(const float* X, int ldx, const uint32_t* Wp, int ldwp,
         if (workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255u) &&
             workspace_bytes >= signw_image_bytes(M, K, g_signw_terms))
             return launch_signw_img(a, g_signw_terms, workspace, (cudaStream_t)stream);
+        if (splice_dim > 0) return BNN_ERR_WORKSPACE;
         return launch_signw_tc(a, g_signw_terms, (cudaStream_t)stream);
     }
+    if (splice_dim > 0) return BNN_ERR_UNSUPPORTED;
     return launch_real_gemm(a, (cudaStream_t)stream);
+}
+
+int bnn_signw_gemm_ws(const float* X, int ldx, const uint32_t* Wp, int ldwp,
+                      int M, int N, int K, float* Y, int ldy,
+                      const bnn_epilogue* epi, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+    return signw_impl(X, ldx, Wp, ldwp, M, N, K, Y, ldy, epi, workspace, workspace_bytes, 0, 0, stream);
 }
 
 size_t bnn_output_prepared_bytes(int C, int H) {
@@ -296,7 +309,8 @@ int bnn_output_prepare(const float* Wout, int ldw, int C, int H,
 static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
                              const float* Wout, int ldw, const float* b, const void* prepared,
                              int M, int C, int H, float* logp, int ldo, int log_softmax,
-                             int zo, void* workspace, size_t workspace_bytes, void* mid_event, void* stream) {
+                             int zo, void* workspace, size_t workspace_bytes, const float* log_prior,
+                             void* mid_event, void* stream) {
     if (int rc = check_dims(M, C, H)) return rc;
     if (!Wout || !logp) return BNN_ERR_NULL;
     if ((Hp == nullptr) == (Hf == nullptr)) return Hp ? BNN_ERR_UNSUPPORTED : BNN_ERR_NULL;
@@ -326,7 +340,7 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
     if (rc) return rc;
     if (mid_event && cudaEventRecord((cudaEvent_t)mid_event, (cudaStream_t)stream) != cudaSuccess)
         return BNN_ERR_CUDA;
-    if (log_softmax) return launch_log_softmax_rows(logp, ldo, M, C, (cudaStream_t)stream);
+    if (log_softmax) return launch_log_softmax_rows(logp, ldo, M, C, log_prior, (cudaStream_t)stream);
     return BNN_OK;
 }
 
@@ -335,7 +349,7 @@ int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
                      int M, int C, int H, float* logp, int ldo, int log_softmax,
                      void* stream) {
     return output_layer_impl(Hp, ldhp, Hf, ldhf, Wout, ldw, b, prepared, M, C, H, logp, ldo,
-                             log_softmax, 0, nullptr, 0, nullptr, stream);
+                             log_softmax, 0, nullptr, 0, nullptr, nullptr, stream);
 }
 
 size_t bnn_output_workspace_bytes(int M, int H) {
@@ -348,7 +362,7 @@ int bnn_output_layer_ws(const float* Hf, int ldhf, const float* Wout, int ldw, c
                         int log_softmax, void* workspace, size_t workspace_bytes, void* stream) {
     if (!Hf) return BNN_ERR_NULL;
     return output_layer_impl(nullptr, 0, Hf, ldhf, Wout, ldw, b, prepared, M, C, H, logp, ldo,
-                             log_softmax, 0, workspace, workspace_bytes, nullptr, stream);
+                             log_softmax, 0, workspace, workspace_bytes, nullptr, nullptr, stream);
 }
 
 int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw, const float* b,
@@ -356,7 +370,7 @@ int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw,
                        int log_softmax, void* stream) {
     if (!Hp) return BNN_ERR_NULL;
     return output_layer_impl(Hp, ldhp, nullptr, 0, Wout, ldw, b, prepared, M, C, H, logp, ldo,
-                             log_softmax, 1, nullptr, 0, nullptr, stream);
+                             log_softmax, 1, nullptr, 0, nullptr, nullptr, stream);
 }
 
 size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M) {
@@ -397,7 +411,12 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                        void* const* layer_out, void* const* events, void* stream) {
     if (int rc = validate_model(model)) return rc;
     if (!X || !logp) return BNN_ERR_NULL;
-    if (M < 1 || ldx < model->layers[0].K) return BNN_ERR_SHAPE;
+    // context window formed inside the first layer: X holds K / (left + right + 1) features per frame
+    const int ctx = model->splice_left + model->splice_right + 1;
+    if (model->splice_left < 0 || model->splice_right < 0) return BNN_ERR_SHAPE;
+    if (ctx > 1 && (model->layers[0].K % ctx != 0 || model->layers[0].kind != BNN_LAYER_SIGNW)) return BNN_ERR_SHAPE;
+    const int splice_dim = ctx > 1 ? model->layers[0].K / ctx : 0;
+    if (M < 1 || ldx < (ctx > 1 ? splice_dim : model->layers[0].K)) return BNN_ERR_SHAPE;
     const int L = model->n_layers;
     if (ldo < model->layers[L - 1].N) return BNN_ERR_SHAPE;
     const size_t need = bnn_forward_min_workspace_bytes(model, M);
@@ -423,7 +442,7 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                                        in_bits ? nullptr : static_cast<const float*>(in), in_ld,
                                        y.W, y.ldw, y.shift, y.W_prepared, M, y.N, y.K, logp, ldo, 1,
                                        in_bits && model->act_values == BNN_VALUES_01, img, img_bytes,
-                                       events ? events[L + 1] : nullptr, stream);
+                                       model->log_prior, events ? events[L + 1] : nullptr, stream);
             if (rc) return rc;
             if (events && events[L] &&
                 cudaEventRecord((cudaEvent_t)events[L], (cudaStream_t)stream) != cudaSuccess)
@@ -447,8 +466,8 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                 yf = static_cast<float*>(out);
                 out_ld = y.N;
             }
-            rc = bnn_signw_gemm_ws(static_cast<const float*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
-                                   yf, y.N, &e, img, img_bytes, stream);
+            rc = signw_impl(static_cast<const float*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
+                            yf, y.N, &e, img, img_bytes, l == 0 ? splice_dim : 0, model->splice_left, stream);
             in_ld = out_ld;
         } else {
             e.thr = y.thr; e.flip = y.flip;

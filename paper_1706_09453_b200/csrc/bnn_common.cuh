@@ -114,6 +114,8 @@ int* tc_status_ptr();
 // either fp32 or packed +-1 bits.
 struct RealGemmArgs {
     const float* Af;      // fp32 A [M][lda] or nullptr
+    int splice_dim;       // > 0: row m of A is the concatenation of rows clamp(m - splice_left + t)
+    int splice_left;      //      (t = 0 .. K/splice_dim - 1) of an fp32 matrix [M][lda] of splice_dim columns
     const uint32_t* Ab;   // packed A [M][lda] or nullptr
     int a_zero_one;       // packed A stands for (0,1) instead of (-1,+1)
     int lda;
@@ -147,6 +149,7 @@ int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const floa
 size_t outf_image_bytes(int M, int H);
 int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float* bias,
                    int M, int C, int H, float* Z, int ldz, void* workspace, cudaStream_t st);
-int launch_log_softmax_rows(float* Z, int ldz, int M, int C, cudaStream_t st);
+// Z <- log softmax of each row, minus prior[c] when `prior` (device, [C]) is given.
+int launch_log_softmax_rows(float* Z, int ldz, int M, int C, const float* prior, cudaStream_t st);
 
 }  // namespace bnn

@@ -224,7 +224,7 @@ __device__ __forceinline__ float block_logsumexp(float mx, float s, float* sm, f
 
 // One CTA per row, any C: online (max, sum exp) in one sweep, then z - logsumexp in a second.
 __global__ void __launch_bounds__(256)
-log_softmax_rows_kernel(float* __restrict__ Z, int ldz, int M, int C) {
+log_softmax_rows_kernel(float* __restrict__ Z, int ldz, int M, int C, const float* __restrict__ prior) {
     __shared__ float sm[8], ss[8];
     for (int row = blockIdx.x; row < M; row += gridDim.x) {
         float* z = Z + (size_t)row * ldz;
@@ -235,7 +235,7 @@ log_softmax_rows_kernel(float* __restrict__ Z, int ldz, int M, int C) {
             s += expf(v - mx);
         }
         const float lse = block_logsumexp(mx, s, sm, ss);
-        for (int c = threadIdx.x; c < C; c += blockDim.x) z[c] -= lse;
+        for (int c = threadIdx.x; c < C; c += blockDim.x) z[c] = z[c] - lse - (prior ? prior[c] : 0.f);
     }
 }
 
@@ -252,7 +252,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // multiply, one ex2 and one add; the sum is reduced the same way.
 template <int V>
 __global__ void __launch_bounds__(256)
-log_softmax_rows_reg_kernel(float* __restrict__ Z, int ldz, int M, int C) {
+log_softmax_rows_reg_kernel(float* __restrict__ Z, int ldz, int M, int C, const float* __restrict__ prior) {
     __shared__ float sm[2][8], ss[2][8];
     const int c4 = C >> 2;  // C % 4 == 0
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -294,7 +294,12 @@ log_softmax_rows_reg_kernel(float* __restrict__ Z, int ldz, int M, int C) {
 #pragma unroll
         for (int i = 0; i < V; ++i) {
             const int c = threadIdx.x + i * 256;
-            if (c < c4) z[c] = make_float4(v[i].x - lse, v[i].y - lse, v[i].z - lse, v[i].w - lse);
+            if (c < c4) {
+                // optional log-prior of each class (16-byte aligned, C % 4 == 0): a hybrid decoder
+                // wants log p(state | frame) - log p(state)
+                const float4 pr = prior ? __ldg(reinterpret_cast<const float4*>(prior) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+                z[c] = make_float4(v[i].x - lse - pr.x, v[i].y - lse - pr.y, v[i].z - lse - pr.z, v[i].w - lse - pr.w);
+            }
         }
     }
 }
@@ -314,15 +319,15 @@ int launch_real_gemm(const RealGemmArgs& a, cudaStream_t st) {
     return launch_status();
 }
 
-int launch_log_softmax_rows(float* Z, int ldz, int M, int C, cudaStream_t st) {
+int launch_log_softmax_rows(float* Z, int ldz, int M, int C, const float* prior, cudaStream_t st) {
     const int blocks = M < 148 * 8 ? M : 148 * 8;
-    const bool reg = (C % 4 == 0) && (ldz % 4 == 0) && aligned16(Z) && C <= 256 * 4 * 4;
+    const bool reg = (C % 4 == 0) && (ldz % 4 == 0) && aligned16(Z) && C <= 256 * 4 * 4 && (!prior || aligned16(prior));
     if (reg && C <= 256 * 4 * 2)
-        log_softmax_rows_reg_kernel<2><<<blocks, 256, 0, st>>>(Z, ldz, M, C);
+        log_softmax_rows_reg_kernel<2><<<blocks, 256, 0, st>>>(Z, ldz, M, C, prior);
     else if (reg)
-        log_softmax_rows_reg_kernel<4><<<blocks, 256, 0, st>>>(Z, ldz, M, C);
+        log_softmax_rows_reg_kernel<4><<<blocks, 256, 0, st>>>(Z, ldz, M, C, prior);
     else
-        log_softmax_rows_kernel<<<blocks, 256, 0, st>>>(Z, ldz, M, C);
+        log_softmax_rows_kernel<<<blocks, 256, 0, st>>>(Z, ldz, M, C, prior);
     return launch_status();
 }
 

@@ -66,12 +66,16 @@ __device__ __forceinline__ float bf16_hi_as_float(uint32_t w) { return __uint_as
 // ---- split: one CTA per (frame tile, stage): 128 rows x 32 floats -> NT planes of 8 KB ------
 template <int NT>
 __global__ void __launch_bounds__(256)
-x_split_kernel(const float* __restrict__ X, int ldx, int M, int K, int nks, uint8_t* __restrict__ img) {
+x_split_kernel(const float* __restrict__ X, int ldx, int M, int K, int nks, uint8_t* __restrict__ img,
+               int sdim, int sleft) {
     __shared__ float raw[BM][BK + 1];
     const int mt = blockIdx.x / nks, ks = blockIdx.x % nks;
     const int t = threadIdx.x;
-    // coalesced read: 8 consecutive threads fetch the 32 floats of one row segment
-    const bool vec = (ldx % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0);
+    // coalesced read: 8 consecutive threads fetch the 32 floats of one row segment.  With splicing
+    // (sdim > 0, a multiple of 4 on the vector path) position k of row m is feature k % sdim of
+    // input row m - sleft + k / sdim, clamped to the rows that exist: the context window of the
+    // feature front end, formed here instead of being materialised in memory.
+    const bool vec = (ldx % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15) == 0) && (sdim % 4 == 0);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int row = (t >> 3) + 32 * i, m = mt * BM + row;
@@ -79,13 +83,30 @@ x_split_kernel(const float* __restrict__ X, int ldx, int M, int K, int nks, uint
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (m < M) {
             const float* src = X + (size_t)m * ldx + k;
+            if (sdim > 0) {
+                int r = m - sleft + k / sdim;
+                r = r < 0 ? 0 : (r >= M ? M - 1 : r);
+                src = X + (size_t)r * ldx + k % sdim;
+            }
             if (vec && k + 3 < K) {
                 v = __ldg(reinterpret_cast<const float4*>(src));
             } else {
-                if (k + 0 < K) v.x = __ldg(src + 0);
-                if (k + 1 < K) v.y = __ldg(src + 1);
-                if (k + 2 < K) v.z = __ldg(src + 2);
-                if (k + 3 < K) v.w = __ldg(src + 3);
+                if (sdim > 0) {   // the four positions may straddle two input rows
+                    float e[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (k + q < K) {
+                            int r = m - sleft + (k + q) / sdim;
+                            r = r < 0 ? 0 : (r >= M ? M - 1 : r);
+                            e[q] = __ldg(X + (size_t)r * ldx + (k + q) % sdim);
+                        }
+                    v = make_float4(e[0], e[1], e[2], e[3]);
+                } else {
+                    if (k + 0 < K) v.x = __ldg(src + 0);
+                    if (k + 1 < K) v.y = __ldg(src + 1);
+                    if (k + 2 < K) v.z = __ldg(src + 2);
+                    if (k + 3 < K) v.w = __ldg(src + 3);
+                }
             }
         }
         raw[row][c4 + 0] = v.x; raw[row][c4 + 1] = v.y; raw[row][c4 + 2] = v.z; raw[row][c4 + 3] = v.w;
@@ -354,7 +375,7 @@ int launch_nt(const RealGemmArgs& r, void* workspace, cudaStream_t st) {
     }
     const int nks = ceil_div(r.K, BK), mt = ceil_div(r.M, BM);
     uint8_t* img = static_cast<uint8_t*>(workspace);
-    x_split_kernel<NT><<<mt * nks, 256, 0, st>>>(r.Af, r.lda, r.M, r.K, nks, img);
+    x_split_kernel<NT><<<mt * nks, 256, 0, st>>>(r.Af, r.lda, r.M, r.K, nks, img, r.splice_dim, r.splice_left);
     Args a{img, r.Bb, r.ldb, r.M, r.N, r.K, r.scale, r.shift, r.act, r.sign_mode, r.Y, r.ldy, r.out_bits, r.ldob,
            tc_status_ptr()};
     if (!a.status) return BNN_ERR_CUDA;

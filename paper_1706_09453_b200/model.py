@@ -27,7 +27,7 @@ def words_to_numpy(t: torch.Tensor, k: int) -> np.ndarray:
 
 class DeviceNet:
     def __init__(self, net: wl.Model, sign_mode=B.SIGN_ZERO_POS, device="cuda:0", prepare_xnor=True,
-                 act_values=B.VALUES_PM1):
+                 act_values=B.VALUES_PM1, splice=(0, 0), log_prior=None):
         cfg = net.cfg
         self.cfg, self.sign_mode, self.device = cfg, sign_mode, device
         self.Wp, self.scale, self.shift, self.thr, self.flip, self.Wimg = [], [], [], [], [], []
@@ -63,7 +63,8 @@ class DeviceNet:
         B.bnn_output_prepare(self.Wout, self.Wout_prepared)
         layers.append(dict(kind=B.LAYER_REAL_OUT, K=cfg.hidden, N=cfg.classes, W=self.Wout,
                            W_prepared=self.Wout_prepared, shift=self.bout))
-        self.desc = B.ModelDesc(layers, sign_mode, act_values)
+        self.log_prior = to_dev(log_prior, device) if log_prior is not None else None
+        self.desc = B.ModelDesc(layers, sign_mode, act_values, splice, self.log_prior)
         self._ws = None
 
     def workspace(self, M: int) -> torch.Tensor:

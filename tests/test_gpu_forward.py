@@ -202,3 +202,48 @@ def test_forward_binary_weights_only_wsj_config_sampled(env):
     sample = np.unique(np.concatenate([np.arange(64), np.arange(cfg.frames - 64, cfg.frames),
                                        rng.integers(0, cfg.frames, 128)]))
     run_bw_net(env, cfg, cfg.frames, sample=sample)
+
+
+@pytest.mark.parametrize("frames", [300, 3])
+def test_forward_spliced_input_and_log_prior(env, frames):
+    """The context window formed inside the first layer (one 40-dim frame per input row, 5 + 1 + 5
+    frames of context, edge frames repeated) and the log-prior subtracted after the log-softmax:
+    equal to the oracle run on the explicitly spliced input."""
+    torch, B, model = env
+    cfg = wl.CONFIGS["tiny"]
+    net = wl.make_model(cfg)
+    rng = np.random.default_rng(frames)
+    F = rng.standard_normal((frames, 40)).astype(np.float32)
+    prior = rng.dirichlet(np.ones(cfg.classes) * 5.0)
+    log_prior = np.log(prior).astype(np.float32)
+    dn = model.DeviceNet(net, splice=(5, 5), log_prior=log_prior)
+    outs = dn.layer_out_buffers(frames)
+    Fd = torch.full((frames, 44), 7.0, dtype=torch.float32, device="cuda:0")   # pitch 44: 16-byte aligned rows
+    Fd[:, :40] = model.to_dev(F)
+    logp = dn.forward(Fd[:, :40], layer_out=outs)
+    torch.cuda.synchronize()
+    X = o.splice(F, 5, 5)
+    assert X.shape == (frames, cfg.in_dim)
+    g1 = model.words_to_numpy(outs[0], cfg.hidden)
+    ref = o.forward(X, net.W, net.scale, net.shift, net.Wout, net.bout, o.ACT_SIGN, 0, layer1_bits=g1,
+                    log_prior=log_prior)
+    band = FLOAT_TOL * np.abs(net.scale[0])[None, :] * ref["sumabs"][:, None]
+    decided = np.abs(ref["pre"][0]) > band
+    np.testing.assert_array_equal(o.unpack_pm1(g1, cfg.hidden)[decided],
+                                  o.unpack_pm1(ref["bits_own_layer1"], cfg.hidden)[decided])
+    assert decided.mean() > 0.995
+    for l in range(1, cfg.n_hidden):
+        np.testing.assert_array_equal(model.words_to_numpy(outs[l], cfg.hidden), ref["bits"][l])
+    assert np.abs(logp.cpu().numpy() - ref["logp"]).max() <= LOGP_TOL
+    # an unaligned pitch takes the scalar path of the splitting kernel: same bits
+    Fu = torch.full((frames, 41), 7.0, dtype=torch.float32, device="cuda:0")
+    Fu[:, :40] = model.to_dev(F)
+    outs2 = dn.layer_out_buffers(frames)
+    logp2 = dn.forward(Fu[:, :40], layer_out=outs2)
+    assert torch.equal(outs2[0], outs[0]) and torch.equal(logp2, logp)
+    # the window needs the scratch image: the minimal workspace is refused
+    small = torch.empty(dn.desc.min_workspace_bytes(frames), dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(B.BnnError) as e:
+        B.bnn_forward(dn.desc, Fd[:, :40], logp, small)
+    assert e.value.status == 5
+    assert B.bnn_device_status() == 0
