@@ -29,6 +29,7 @@
 #define ACT_NONE 0
 #define ACT_SIGN 1
 #define ACT_HARDTANH 2
+#define ACT_SIGMOID 3  /* the hidden units of the paper's real-valued layers (Section 3) */
 
 int oracle_num_threads(void) {
 #ifdef _OPENMP
@@ -142,6 +143,25 @@ void oracle_affine_sign_pack_i32(const int32_t* D, long ldd, long M, long N,
 }
 
 /*
+ * A binary layer whose output stays real-valued: h = Sigmoid(scale*d + shift), the last hidden
+ * layer of the paper's best systems (Table 2: Sigmoid on the first and last hidden layer, binary
+ * in between).  The affine is the same single fp32 fused multiply-add as in the Sign layers; the
+ * Sigmoid of that fp32 value is evaluated in double.  Yhat (optional) receives the fp32 value.
+ */
+void oracle_affine_sigmoid_i32(const int32_t* D, long ldd, long M, long N,
+                               const float* scale, const float* shift,
+                               double* H, long ldh, float* Yhat, long ldy) {
+    for (long m = 0; m < M; ++m)
+        for (long n = 0; n < N; ++n) {
+            float s = scale ? scale[n] : 1.0f;
+            float b = shift ? shift[n] : 0.0f;
+            float y = fmaf(s, (float)D[m * ldd + n], b);
+            if (Yhat) Yhat[m * ldy + n] = y;
+            H[m * ldh + n] = 1.0 / (1.0 + exp(-(double)y));
+        }
+}
+
+/*
  * Binary weights against real-valued activations (Algorithm 1 forward, without the bias):
  * y[m][n] = sum_k w^b[n][k] * x[m][k], w^b in {-1,+1}, accumulated in double.
  * sumabs[m] (optional) = sum_k |x[m][k]|, the scale of the comparison tolerance.
@@ -189,6 +209,8 @@ void oracle_affine_act_f64(const double* Y, long ldy, long M, long N,
                 if (P && sg == 1) P[m * ldp + n / 32] |= (uint32_t)1 << (n % 32);
             } else if (act == ACT_HARDTANH) {
                 h = v < -1.0 ? -1.0 : (v > 1.0 ? 1.0 : v);
+            } else if (act == ACT_SIGMOID) {
+                h = 1.0 / (1.0 + exp(-v));
             }
             if (H) H[m * ldh + n] = h;
         }

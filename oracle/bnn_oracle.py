@@ -200,6 +200,59 @@ def log_softmax(Z):
     return LP
 
 
+ACT_SIGMOID = 3
+
+
+def affine_sigmoid_i32(D, scale, shift):
+    """h = Sigmoid(fma(scale, d, shift)) for integer dot products d; float64 [M][N]."""
+    D = np.ascontiguousarray(D, dtype=np.int32)
+    M, N = D.shape
+    scale, shift = _f32(scale), _f32(shift)
+    H = np.empty((M, N), dtype=np.float64)
+    lib().oracle_affine_sigmoid_i32(_p(D), _L(N), _L(M), _L(N), _p(scale), _p(shift), _p(H), _L(N), None, _L(0))
+    return H
+
+
+def forward_mixed(X, W, scale, shift, Wout, bout, mode=SIGN_ZERO_POS, layer2_bits=None):
+    """Forward pass of the paper's most accurate topology (Table 2, Section 3.2; with the binary
+    weights of Section 2.3 in the middle): layer 1 keeps real-valued weights and Sigmoid units,
+    layer 2 has +-1 weights on those real activations and Sign units, layers 3 .. L-1 are
+    +-1 x +-1 with Sign units, layer L is +-1 x +-1 with Sigmoid units, the Softmax layer is
+    real-valued.  W[0] is used as it is (bias shift[0], scale[0] must be None); W[1:] are
+    binarised with Eq. 3.  ``layer2_bits`` replaces the oracle's own layer-2 bits (see forward).
+    """
+    X = _f32(X)
+    L = len(W)
+    assert L >= 3 and scale[0] is None
+    taps = {"pre": [], "bits": []}
+    Wp = [None] + [sign_pack(w, mode) for w in W[1:]]
+    taps["Wp"] = Wp
+    # layer 1: real weights, Sigmoid (Eq. 1-2 with f = Sigmoid), in double, handed on as fp32
+    Y1 = real_gemm_f32(X, W[0], shift[0])
+    _, H1, _ = affine_act_f64(Y1, None, None, ACT_SIGMOID, mode)
+    taps["h1"] = H1
+    h1 = H1.astype(np.float32)
+    # layer 2: +-1 weights on real activations, Sign
+    Y2, sumabs = signw_gemm(h1, Wp[1], W[1].shape[1])
+    Yh, _, P = affine_act_f64(Y2, scale[1], shift[1], ACT_SIGN, mode)
+    taps["sumabs2"], taps["pre2"], taps["bits_own_layer2"] = sumabs, Yh, P
+    if layer2_bits is not None:
+        P = np.ascontiguousarray(layer2_bits, dtype=np.uint32)[:, :words(W[1].shape[0])]
+    taps["bits"].append(P)
+    for l in range(2, L - 1):
+        D = xnor_gemm(P, Wp[l], W[l].shape[1])
+        P = affine_sign_pack_i32(D, scale[l], shift[l], mode)
+        taps["bits"].append(P)
+    # layer L: +-1 x +-1, Sigmoid units
+    D = xnor_gemm(P, Wp[L - 1], W[L - 1].shape[1])
+    HL = affine_sigmoid_i32(D, scale[L - 1], shift[L - 1])
+    taps["hL"] = HL
+    Z = real_gemm_f32(HL.astype(np.float32), Wout, bout)
+    taps["logits"] = Z
+    taps["logp"] = log_softmax(Z)
+    return taps
+
+
 def splice(F, left, right):
     """Context window of the feature front end (Section 3: frames spliced over a context of 11):
     row m of the result is the concatenation of rows m - left .. m + right of F; rows outside the

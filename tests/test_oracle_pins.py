@@ -398,3 +398,48 @@ def test_forward_log_prior_is_subtracted_from_log_posteriors():
     np.testing.assert_allclose(b["logp"], a["logp"] - lp.astype(np.float64)[None, :], atol=1e-12)
     # posterior / prior, summed with the prior as weights, is 1 again
     np.testing.assert_allclose((np.exp(b["logp"]) * np.exp(lp.astype(np.float64))).sum(1), 1.0, atol=1e-9)
+
+
+# ---------------------------------------------------------------- Sigmoid layers, mixed topology
+def test_sigmoid_activation_pins():
+    from scipy.special import expit
+    y = np.array([[0.0, 1.0, -1.0, 30.0, -30.0, 1e-3, -745.0, 710.0]])
+    _, H, _ = o.affine_act_f64(y, None, None, o.ACT_SIGMOID)
+    np.testing.assert_allclose(H, expit(y), rtol=1e-15, atol=0)
+    assert H[0, 0] == 0.5
+    np.testing.assert_allclose(H[0, 1] + H[0, 2], 1.0, atol=1e-16)   # sigma(-x) = 1 - sigma(x)
+    # integer dot products through the fp32 affine
+    d = np.array([[-5, 0, 3, 100]], dtype=np.int32)
+    sc = np.array([0.5, 1.0, -2.0, 0.25], dtype=np.float32)
+    sh = np.array([0.25, 0.0, 1.0, -25.0], dtype=np.float32)
+    np.testing.assert_allclose(o.affine_sigmoid_i32(d, sc, sh), expit(np.array([[-2.25, 0.0, -5.0, 0.0]])), rtol=1e-15)
+
+
+def test_forward_mixed_topology_against_numpy():
+    """(Sigmoid, Sign, Sign, Sigmoid, Softmax) with real first-layer and Softmax weights, written
+    again with numpy on values whose layer-2 pre-activations are far from zero."""
+    from scipy.special import expit
+    rng = np.random.default_rng(12)
+    dims = [23, 40, 36, 32, 28]
+    X = rng.standard_normal((7, dims[0])).astype(np.float32)
+    W = [rng.standard_normal((dims[i + 1], dims[i])).astype(np.float32) for i in range(4)]
+    sc = [None] + [rng.uniform(0.5, 1.5, dims[i + 1]).astype(np.float32) for i in range(1, 4)]
+    sh = [rng.standard_normal(dims[i + 1]).astype(np.float32) * 0.3 for i in range(4)]
+    Wout = rng.standard_normal((9, dims[-1])).astype(np.float32)
+    bout = rng.standard_normal(9).astype(np.float32)
+    t = o.forward_mixed(X, W, sc, sh, Wout, bout, o.SIGN_ZERO_NEG)
+    f64 = lambda a: a.astype(np.float64)
+    h = expit(f64(X) @ f64(W[0]).T + f64(sh[0])).astype(np.float32)
+    y = (f64(h) @ np.where(W[1] > 0, 1.0, -1.0).T) * f64(sc[1]) + f64(sh[1])
+    assert np.abs(y).min() > 1e-6
+    a = np.where(y > 0, 1.0, -1.0)
+    d = a @ np.where(W[2] > 0, 1.0, -1.0).T
+    a = np.where((np.float32(1) * (sc[2] * d.astype(np.float32) + sh[2])) > 0, 1.0, -1.0)
+    d = a @ np.where(W[3] > 0, 1.0, -1.0).T
+    hL = expit(f64((sc[3] * d.astype(np.float32) + sh[3]).astype(np.float32))).astype(np.float32)
+    z = f64(hL) @ f64(Wout).T + f64(bout)
+    z = z - z.max(1, keepdims=True)
+    want = z - np.log(np.exp(z).sum(1, keepdims=True))
+    # two roundings instead of one fma can move a value by an ulp: far inside the tolerance
+    np.testing.assert_allclose(t["logp"], want, atol=1e-5)
+    np.testing.assert_array_equal(o.unpack_pm1(t["bits"][0], dims[2]), np.where(y > 0, 1, -1))
