@@ -35,7 +35,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="wsj", choices=["tiny", "wsj", "wsj_bw", "ami"])
+    ap.add_argument("--config", default="wsj", choices=["tiny", "wsj", "wsj_bw", "ami", "wsj_mixed"])
     ap.add_argument("--frames", type=int, default=None, help="override the batch size (frames per step)")
     ap.add_argument("--cpu-frames", type=int, default=16384, help="frames of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -81,6 +81,8 @@ def load_peaks():
 # ------------------------------------------------------------------ CPU oracle arm
 def oracle_step(cfg, net, X):
     from oracle import bnn_oracle as o
+    if getattr(cfg, "mixed", False):
+        return o.forward_mixed(X, net.W, net.scale, net.shift, net.Wout, net.bout, o.SIGN_ZERO_POS)
     return o.forward(X, net.W, net.scale, net.shift, net.Wout, net.bout,
                      o.ACT_SIGN if cfg.act == 1 else o.ACT_HARDTANH, o.SIGN_ZERO_POS)
 
@@ -196,10 +198,23 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
     fp32_peak = SMS * 128 * 2 * clk / 1e12          # TFLOP/s on the FP32 pipe
     rows = []
     k = cfg.in_dim
+    mixed = getattr(cfg, "mixed", False)
     for l in range(cfg.n_hidden):
-        xnor = cfg.act == 1 and l > 0
+        xnor = cfg.act == 1 and l > (1 if mixed else 0)
         work = 2.0 * frames * cfg.hidden * k
-        if xnor and xnor_path in ("tensor", "tensor-unprepared"):
+        if mixed and l == 0:
+            # real-valued Sigmoid layer: both operands in two fp16 terms, three MMAs per step
+            if real_path == "tensor":
+                rows.append(dict(name="real_1", kernel="h_split_kernel+outf_tc_kernel", work=work, unit="TFLOP/s",
+                                 bound="tensor", peak=peaks["bf16_tflops_sustained"], passes=3))
+            else:
+                rows.append(dict(name="real_1", kernel="real_gemm_kernel", work=work, unit="TFLOP/s", bound="alu",
+                                 peak=fp32_peak))
+        elif xnor and mixed and l == cfg.n_hidden - 1 and xnor_path != "popc":
+            # binary layer with Sigmoid units: int32 dot products, then one pointwise pass
+            rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_tc_kernel+affine_sigmoid_i32_kernel", work=work,
+                             unit="Tbop/s", bound="tensor", peak=4.0 * peaks["bf16_tflops_sustained"]))
+        elif xnor and xnor_path in ("tensor", "tensor-unprepared"):
             # 4-bit (e2m1, kind::mxf4) tensor-core MACs: 4 x the measured bf16 rate (nominal ratio
             # 9 : 2.25 PFLOP/s), sustained figure because the kernel is timed inside a long step;
             # 1 bit-MAC = 2 bop.  smem_bytes: what the kernel moves through the SM's shared
@@ -234,7 +249,7 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
                              bound="alu", peak=fp32_peak))
         k = cfg.hidden
     owork = 2.0 * frames * cfg.classes * cfg.hidden
-    if real_path == "tensor" and cfg.act == 1:
+    if real_path == "tensor" and cfg.act == 1 and not mixed:
         rows.append(dict(name="output_gemm", kernel="out_tc_kernel", work=owork, unit="TFLOP/s", bound="tensor",
                          peak=peaks["bf16_tflops_sustained"], passes=2))
     elif real_path == "tensor":
@@ -492,9 +507,9 @@ def run_ours(args):
         "e2e": {"value": e2e_fps, "unit": UNIT, "h2d_bytes_per_step": int(Xp.numel() * 4),
                 "d2h_bytes_per_step": int(Lp.numel() * 4), "steps": Ke,
                 "overlap": "copy-in, forward and copy-out of consecutive steps on three streams"},
-        # per step: one kernel per binary hidden layer, two per sign-weight layer (split + GEMM),
-        # top-layer GEMM and log-softmax
-        "gpu_launches": K * (cfg.n_hidden + 2 + (1 if cfg.act == 1 else cfg.n_hidden) * (1 if args.real_path == "tensor" else 0)),
+        # per step: the kernels named in the layer table (one per binary hidden layer, two per
+        # sign-weight layer: split + GEMM, top-layer GEMM, log-softmax)
+        "gpu_launches": K * sum(r["kernel"].count("+") + 1 for r in rows),
         "paths": {"xnor": args.xnor_path, "real": args.real_path},
         "roofline": roofline,
         "forward_roofline": forward_roofline,

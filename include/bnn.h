@@ -64,7 +64,10 @@ typedef enum { BNN_VALUES_PM1 = 0, BNN_VALUES_01 = 1 } bnn_act_values;
 typedef enum {
     BNN_ACT_NONE = 0,      /* write the value itself */
     BNN_ACT_SIGN_PACK = 1, /* f = Sign (Algorithm 2), written as packed bits */
-    BNN_ACT_HARDTANH = 2   /* f = clamp to [-1, 1], written as fp32 */
+    BNN_ACT_HARDTANH = 2,  /* f = clamp to [-1, 1], written as fp32 */
+    BNN_ACT_SIGMOID = 3    /* f = 1 / (1 + exp(-x)), written as fp32: the real-valued hidden units of
+                              the paper's networks (Section 3; Table 2 keeps them on the first and
+                              last hidden layer) */
 } bnn_act;
 
 /*
@@ -223,6 +226,22 @@ BNN_API int bnn_output_layer_ws(const float* Hf, int ldhf, const float* Wout, in
                                 float* logp, int ldo, int log_softmax,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* A hidden layer with real-valued weights (Eq. 1-2): Y = f(Hf W^T + bias), f = BNN_ACT_SIGMOID,
+ * BNN_ACT_HARDTANH or BNN_ACT_NONE.  Hf : fp32 [M][ldhf].  W : fp32 [N][ldw].  Y : fp32 [M][ldy].
+ * With `prepared` (bnn_output_prepare image of W) and `workspace` (bnn_output_workspace_bytes(M, K)
+ * bytes, 256-byte aligned) it runs on the tensor cores like bnn_output_layer_ws, same bound before
+ * f; otherwise on the FP32 pipe. */
+BNN_API int bnn_real_layer(const float* Hf, int ldhf, const float* W, int ldw, const float* bias,
+                           const void* prepared, int M, int N, int K, float* Y, int ldy, int act,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* Sigmoid units on a binary layer: Y[m][n] = Sigmoid(fma(scale[n], D[m][n], shift[n])) for the
+ * integer dot products D of bnn_xnor_gemm (the last hidden layer of the paper's mixed networks,
+ * Table 2).  scale, shift : [N] or NULL.  Y may be the same buffer as D when ldy == ldd.  The
+ * affine is the same single fp32 fused multiply-add as in the Sign layers. */
+BNN_API int bnn_affine_sigmoid_i32(const int32_t* D, int ldd, const float* scale, const float* shift,
+                                   int M, int N, float* Y, int ldy, void* stream);
+
 /* One-time preparation of the top layer's weights for the tensor cores: each class row is
  * scaled by a power of two and split into two fp16 terms (about 22 significant bits), stored
  * in the order the MMA reads shared memory.  prepared : device buffer, 256-byte aligned, of
@@ -239,7 +258,9 @@ typedef enum {
     BNN_LAYER_SIGNW = 0,   /* +-1 weights x real input (first layer; every hidden layer of
                               a binary-weights-only network) */
     BNN_LAYER_XNOR = 1,    /* +-1 weights x +-1 activations */
-    BNN_LAYER_REAL_OUT = 2 /* real-valued top layer + log-softmax; must be last */
+    BNN_LAYER_REAL_OUT = 2,/* real-valued top layer + log-softmax; must be last */
+    BNN_LAYER_REAL = 3     /* real-valued weights x real input + bias, SIGMOID or HARDTANH units: the
+                              input layer the paper keeps real-valued in its best systems (Table 2) */
 } bnn_layer_kind;
 
 typedef struct bnn_layer {
@@ -247,15 +268,17 @@ typedef struct bnn_layer {
     int K, N;              /* fan-in, fan-out */
     const uint32_t* Wp;    /* SIGNW, XNOR: packed weights [N][ldwp] */
     int ldwp;
-    const float* W;        /* REAL_OUT: fp32 weights [N][ldw] */
+    const float* W;        /* REAL_OUT, REAL: fp32 weights [N][ldw] */
     int ldw;
-    const void* W_prepared;/* REAL_OUT: bnn_output_prepare image of W, or NULL;
+    const void* W_prepared;/* REAL_OUT, REAL: bnn_output_prepare image of W, or NULL;
                               XNOR: bnn_xnor_prepare image of Wp, or NULL */
     const float* scale;    /* SIGNW: per-unit scale or NULL */
-    const float* shift;    /* SIGNW: per-unit shift or NULL; REAL_OUT: bias or NULL */
+    const float* shift;    /* SIGNW: per-unit shift or NULL; REAL_OUT, REAL: bias or NULL;
+                              XNOR with SIGMOID units: scale and shift of the affine */
     const int32_t* thr;    /* XNOR: folded thresholds [N] */
     const uint32_t* flip;  /* XNOR: [ceil(N/32)] */
-    int act;               /* SIGNW: BNN_ACT_SIGN_PACK or BNN_ACT_HARDTANH; XNOR: SIGN_PACK */
+    int act;               /* SIGNW: SIGN_PACK, HARDTANH or SIGMOID; XNOR: SIGN_PACK (thr, flip) or
+                              SIGMOID (scale, shift; fp32 output); REAL: SIGMOID or HARDTANH */
 } bnn_layer;
 
 typedef struct bnn_model {
@@ -296,8 +319,10 @@ BNN_API size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M);
  *   hidden layer l write its output there instead of into the workspace (packed bits with
  *   pitch bnn_packed_pitch(N_l) words, or fp32 [M][N_l] for HARDTANH layers), which lets a
  *   caller inspect every layer at no cost.
- * Layer kinds must chain: SIGNW+SIGN_PACK -> XNOR; SIGNW+HARDTANH -> SIGNW or REAL_OUT;
- * XNOR -> XNOR or REAL_OUT; the last layer is REAL_OUT.  Otherwise BNN_ERR_UNSUPPORTED.
+ * Layer kinds must chain: a layer with SIGN_PACK units feeds XNOR or REAL_OUT; a layer with
+ * fp32 units (HARDTANH, SIGMOID) feeds SIGNW, REAL or REAL_OUT; the last layer is REAL_OUT.
+ * Otherwise BNN_ERR_UNSUPPORTED.  The paper's mixed topology (Table 2) is
+ * REAL+SIGMOID -> SIGNW+SIGN_PACK -> XNOR+SIGN_PACK ... -> XNOR+SIGMOID -> REAL_OUT.
  */
 BNN_API int bnn_forward(const bnn_model* model, const float* X, int ldx, int M,
                 float* logp, int ldo, void* workspace, size_t workspace_bytes,

@@ -14,9 +14,9 @@ import torch
 from . import build as _build
 
 SIGN_ZERO_POS, SIGN_ZERO_NEG = 0, 1
-ACT_NONE, ACT_SIGN_PACK, ACT_HARDTANH = 0, 1, 2
+ACT_NONE, ACT_SIGN_PACK, ACT_HARDTANH, ACT_SIGMOID = 0, 1, 2, 3
 VALUES_PM1, VALUES_01 = 0, 1
-LAYER_SIGNW, LAYER_XNOR, LAYER_REAL_OUT = 0, 1, 2
+LAYER_SIGNW, LAYER_XNOR, LAYER_REAL_OUT, LAYER_REAL = 0, 1, 2, 3
 
 
 class BnnError(RuntimeError):
@@ -108,6 +108,10 @@ def lib():
         L.bnn_output_workspace_bytes.restype = C.c_size_t
         L.bnn_output_layer_ws.argtypes = [p, i, p, i, p, p, i, i, i, p, i, i, p, C.c_size_t, p]
         L.bnn_output_layer_ws.restype = C.c_int
+        L.bnn_real_layer.argtypes = [p, i, p, i, p, p, i, i, i, p, i, i, p, C.c_size_t, p]
+        L.bnn_real_layer.restype = C.c_int
+        L.bnn_affine_sigmoid_i32.argtypes = [p, i, p, p, i, i, p, i, p]
+        L.bnn_affine_sigmoid_i32.restype = C.c_int
         L.bnn_gemm01.argtypes = [p, i, p, i, p, i, i, i, p, i, C.POINTER(Epilogue), p]
         L.bnn_gemm01.restype = C.c_int
         L.bnn_forward.argtypes = [C.POINTER(Model), p, i, i, p, i, p, C.c_size_t, C.POINTER(p), p]
@@ -305,6 +309,26 @@ def bnn_output_prepare(Wout, prepared):
     _check(lib().bnn_output_prepare(_ptr(Wout, torch.float32), _ld(Wout), c, h, _ptr(prepared),
                                     prepared.numel() * prepared.element_size(), _stream()), "bnn_output_prepare")
     return prepared
+
+
+def bnn_real_layer(Hf, W, bias, Y, act=ACT_SIGMOID, prepared=None, workspace=None):
+    """Y = act(Hf W^T + bias) with real-valued weights; tensor cores with ``prepared`` and ``workspace``."""
+    m, k = Hf.shape
+    _check(lib().bnn_real_layer(_ptr(Hf, torch.float32), _ld(Hf), _ptr(W, torch.float32), _ld(W),
+                                _ptr(bias, torch.float32), _ptr(prepared), m, W.shape[0], k,
+                                _ptr(Y, torch.float32), _ld(Y), act, _ptr(workspace),
+                                workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                _stream()), "bnn_real_layer")
+    return Y
+
+
+def bnn_affine_sigmoid_i32(D, scale, shift, Y):
+    """Y = Sigmoid(fma(scale, D, shift)); ``Y`` may be a float32 view of ``D``'s own memory."""
+    m, n = D.shape
+    _check(lib().bnn_affine_sigmoid_i32(_ptr(D, torch.int32), _ld(D), _ptr(scale, torch.float32),
+                                        _ptr(shift, torch.float32), m, n, _ptr(Y, torch.float32), _ld(Y),
+                                        _stream()), "bnn_affine_sigmoid_i32")
+    return Y
 
 
 def bnn_output_workspace_bytes(M, H) -> int:

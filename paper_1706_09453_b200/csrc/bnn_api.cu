@@ -60,14 +60,25 @@ int validate_model(const bnn_model* model) {
         switch (y.kind) {
             case BNN_LAYER_SIGNW:
                 if (in_bits || l == L - 1) return BNN_ERR_UNSUPPORTED;
-                if (y.act != BNN_ACT_SIGN_PACK && y.act != BNN_ACT_HARDTANH) return BNN_ERR_UNSUPPORTED;
+                if (y.act != BNN_ACT_SIGN_PACK && y.act != BNN_ACT_HARDTANH && y.act != BNN_ACT_SIGMOID)
+                    return BNN_ERR_UNSUPPORTED;
                 if (int rc = check_packed(y.Wp, y.ldwp, y.K)) return rc;
                 break;
             case BNN_LAYER_XNOR:
                 if (!in_bits || l == L - 1) return BNN_ERR_UNSUPPORTED;
-                if (y.act != BNN_ACT_SIGN_PACK) return BNN_ERR_UNSUPPORTED;
-                if (!y.thr || !y.flip) return BNN_ERR_NULL;
+                if (y.act == BNN_ACT_SIGN_PACK) {
+                    if (!y.thr || !y.flip) return BNN_ERR_NULL;
+                } else if (y.act != BNN_ACT_SIGMOID) {
+                    return BNN_ERR_UNSUPPORTED;
+                }
                 if (int rc = check_packed(y.Wp, y.ldwp, y.K)) return rc;
+                break;
+            case BNN_LAYER_REAL:
+                if (in_bits || l == L - 1) return BNN_ERR_UNSUPPORTED;
+                if (y.act != BNN_ACT_SIGMOID && y.act != BNN_ACT_HARDTANH) return BNN_ERR_UNSUPPORTED;
+                if (!y.W) return BNN_ERR_NULL;
+                if (y.ldw < y.K) return BNN_ERR_SHAPE;
+                if (y.scale) return BNN_ERR_UNSUPPORTED;   // Eq. 1 as printed: weights and a bias
                 break;
             case BNN_LAYER_REAL_OUT:
                 if (l != L - 1) return BNN_ERR_UNSUPPORTED;
@@ -263,7 +274,8 @@ static int signw_impl(const float* X, int ldx, const uint32_t* Wp, int ldwp,
     a.Y = Y; a.ldy = ldy;
     a.act = BNN_ACT_NONE; a.sign_mode = BNN_SIGN_ZERO_POS;
     if (epi) {
-        if (epi->act != BNN_ACT_NONE && epi->act != BNN_ACT_SIGN_PACK && epi->act != BNN_ACT_HARDTANH)
+        if (epi->act != BNN_ACT_NONE && epi->act != BNN_ACT_SIGN_PACK && epi->act != BNN_ACT_HARDTANH &&
+            epi->act != BNN_ACT_SIGMOID)
             return BNN_ERR_UNSUPPORTED;
         if (epi->sign_mode != BNN_SIGN_ZERO_POS && epi->sign_mode != BNN_SIGN_ZERO_NEG)
             return BNN_ERR_UNSUPPORTED;
@@ -310,8 +322,10 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
                              const float* Wout, int ldw, const float* b, const void* prepared,
                              int M, int C, int H, float* logp, int ldo, int log_softmax,
                              int zo, void* workspace, size_t workspace_bytes, const float* log_prior,
-                             void* mid_event, void* stream) {
+                             int act, void* mid_event, void* stream) {
     if (int rc = check_dims(M, C, H)) return rc;
+    if (act != BNN_ACT_NONE && (Hp || log_softmax || (act != BNN_ACT_SIGMOID && act != BNN_ACT_HARDTANH)))
+        return BNN_ERR_UNSUPPORTED;
     if (!Wout || !logp) return BNN_ERR_NULL;
     if ((Hp == nullptr) == (Hf == nullptr)) return Hp ? BNN_ERR_UNSUPPORTED : BNN_ERR_NULL;
     if (ldw < H || ldo < C) return BNN_ERR_SHAPE;
@@ -326,7 +340,7 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
     a.Bf = Wout; a.ldb = ldw;
     a.M = M; a.N = C; a.K = H;
     a.shift = b;
-    a.act = BNN_ACT_NONE;
+    a.act = act;
     a.Y = logp; a.ldy = ldo;
     if (prepared && (reinterpret_cast<uintptr_t>(prepared) & 255u)) return BNN_ERR_ALIGN;
     int rc;
@@ -334,7 +348,7 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
         rc = launch_out_tc(Hp, ldhp, prepared, b, M, C, H, logp, ldo, zo, (cudaStream_t)stream);
     else if (Hf && prepared && g_real_path != BNN_PATH_CUDA_CORE && workspace &&
              !(reinterpret_cast<uintptr_t>(workspace) & 255u) && workspace_bytes >= outf_image_bytes(M, H))
-        rc = launch_outf_tc(Hf, ldhf, prepared, b, M, C, H, logp, ldo, workspace, (cudaStream_t)stream);
+        rc = launch_outf_tc(Hf, ldhf, prepared, b, M, C, H, logp, ldo, act, workspace, (cudaStream_t)stream);
     else
         rc = launch_real_gemm(a, (cudaStream_t)stream);
     if (rc) return rc;
@@ -349,7 +363,23 @@ int bnn_output_layer(const uint32_t* Hp, int ldhp, const float* Hf, int ldhf,
                      int M, int C, int H, float* logp, int ldo, int log_softmax,
                      void* stream) {
     return output_layer_impl(Hp, ldhp, Hf, ldhf, Wout, ldw, b, prepared, M, C, H, logp, ldo,
-                             log_softmax, 0, nullptr, 0, nullptr, nullptr, stream);
+                             log_softmax, 0, nullptr, 0, nullptr, BNN_ACT_NONE, nullptr, stream);
+}
+
+int bnn_real_layer(const float* Hf, int ldhf, const float* W, int ldw, const float* bias,
+                   const void* prepared, int M, int N, int K, float* Y, int ldy, int act,
+                   void* workspace, size_t workspace_bytes, void* stream) {
+    if (!Hf) return BNN_ERR_NULL;
+    return output_layer_impl(nullptr, 0, Hf, ldhf, W, ldw, bias, prepared, M, N, K, Y, ldy, 0, 0,
+                             workspace, workspace_bytes, nullptr, act, nullptr, stream);
+}
+
+int bnn_affine_sigmoid_i32(const int32_t* D, int ldd, const float* scale, const float* shift,
+                           int M, int N, float* Y, int ldy, void* stream) {
+    if (!D || !Y) return BNN_ERR_NULL;
+    if (M < 1 || N < 1 || ldd < N || ldy < N) return BNN_ERR_SHAPE;
+    if (static_cast<const void*>(D) == static_cast<const void*>(Y) && ldd != ldy) return BNN_ERR_SHAPE;
+    return launch_affine_sigmoid_i32(D, ldd, scale, shift, M, N, Y, ldy, (cudaStream_t)stream);
 }
 
 size_t bnn_output_workspace_bytes(int M, int H) {
@@ -362,7 +392,7 @@ int bnn_output_layer_ws(const float* Hf, int ldhf, const float* Wout, int ldw, c
                         int log_softmax, void* workspace, size_t workspace_bytes, void* stream) {
     if (!Hf) return BNN_ERR_NULL;
     return output_layer_impl(nullptr, 0, Hf, ldhf, Wout, ldw, b, prepared, M, C, H, logp, ldo,
-                             log_softmax, 0, workspace, workspace_bytes, nullptr, nullptr, stream);
+                             log_softmax, 0, workspace, workspace_bytes, nullptr, BNN_ACT_NONE, nullptr, stream);
 }
 
 int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw, const float* b,
@@ -370,7 +400,7 @@ int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw,
                        int log_softmax, void* stream) {
     if (!Hp) return BNN_ERR_NULL;
     return output_layer_impl(Hp, ldhp, nullptr, 0, Wout, ldw, b, prepared, M, C, H, logp, ldo,
-                             log_softmax, 1, nullptr, 0, nullptr, nullptr, stream);
+                             log_softmax, 1, nullptr, 0, nullptr, BNN_ACT_NONE, nullptr, stream);
 }
 
 size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M) {
@@ -392,8 +422,9 @@ size_t bnn_forward_workspace_bytes(const bnn_model* model, int M) {
         size_t b = 0;
         if (y.kind == BNN_LAYER_SIGNW)
             b = signw_image_bytes(M, y.K, 3);  // room for either term count
-        else if (y.kind == BNN_LAYER_REAL_OUT && l > 0 && model->layers[l - 1].act == BNN_ACT_HARDTANH)
-            b = outf_image_bytes(M, y.K);      // fp32 activations into the top layer
+        else if (y.kind == BNN_LAYER_REAL ||
+                 (y.kind == BNN_LAYER_REAL_OUT && l > 0 && model->layers[l - 1].act != BNN_ACT_SIGN_PACK))
+            b = outf_image_bytes(M, y.K);      // fp32 activations into a real-valued layer
         if (b > img) img = b;
     }
     return base + round256(img);
@@ -442,7 +473,7 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                                        in_bits ? nullptr : static_cast<const float*>(in), in_ld,
                                        y.W, y.ldw, y.shift, y.W_prepared, M, y.N, y.K, logp, ldo, 1,
                                        in_bits && model->act_values == BNN_VALUES_01, img, img_bytes,
-                                       model->log_prior, events ? events[L + 1] : nullptr, stream);
+                                       model->log_prior, BNN_ACT_NONE, events ? events[L + 1] : nullptr, stream);
             if (rc) return rc;
             if (events && events[L] &&
                 cudaEventRecord((cudaEvent_t)events[L], (cudaStream_t)stream) != cudaSuccess)
@@ -469,6 +500,23 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
             rc = signw_impl(static_cast<const float*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
                             yf, y.N, &e, img, img_bytes, l == 0 ? splice_dim : 0, model->splice_left, stream);
             in_ld = out_ld;
+        } else if (y.kind == BNN_LAYER_REAL) {
+            if (l == 0 && splice_dim > 0) return BNN_ERR_UNSUPPORTED;
+            rc = output_layer_impl(nullptr, 0, static_cast<const float*>(in), in_ld, y.W, y.ldw, y.shift,
+                                   y.W_prepared, M, y.N, y.K, static_cast<float*>(out), y.N, 0, 0,
+                                   img, img_bytes, nullptr, y.act, nullptr, stream);
+            in_ld = y.N;
+        } else if (y.act == BNN_ACT_SIGMOID) {
+            // binary layer with Sigmoid units: the integer dot products go to the output buffer
+            // and are turned into fp32 activations in place
+            const bool image = y.W_prepared && g_xnor_path != BNN_PATH_CUDA_CORE && y.K <= kMaxKTensor;
+            rc = xnor_gemm_impl(static_cast<const uint32_t*>(in), in_ld, y.Wp, y.ldwp,
+                                image ? y.W_prepared : nullptr, M, y.N, y.K, static_cast<int32_t*>(out), y.N,
+                                nullptr, model->act_values == BNN_VALUES_01, stream);
+            if (!rc)
+                rc = launch_affine_sigmoid_i32(static_cast<const int32_t*>(out), y.N, y.scale, y.shift, M, y.N,
+                                               static_cast<float*>(out), y.N, (cudaStream_t)stream);
+            in_ld = y.N;
         } else {
             e.thr = y.thr; e.flip = y.flip;
             e.out_bits = static_cast<uint32_t*>(out); e.ldob = bnn_packed_pitch(y.N);

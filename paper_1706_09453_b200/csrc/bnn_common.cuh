@@ -147,8 +147,12 @@ int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const floa
 // The top layer on fp32 activations (finite, |a| < 65504) with both operands split into fp16
 // terms (out_gemm_f32_tc.cu): `workspace` holds outf_image_bytes(M, H) bytes, 256-byte aligned.
 size_t outf_image_bytes(int M, int H);
+// `act`: bnn_act applied after the bias (NONE, SIGMOID, HARDTANH).
 int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float* bias,
-                   int M, int C, int H, float* Z, int ldz, void* workspace, cudaStream_t st);
+                   int M, int C, int H, float* Z, int ldz, int act, void* workspace, cudaStream_t st);
+// Y = Sigmoid(fma(scale, D, shift)) element by element (Y may alias D when the pitches agree).
+int launch_affine_sigmoid_i32(const int32_t* D, int ldd, const float* scale, const float* shift,
+                              int M, int N, float* Y, int ldy, cudaStream_t st);
 // Z <- log softmax of each row, minus prior[c] when `prior` (device, [C]) is given.
 int launch_log_softmax_rows(float* Z, int ldz, int M, int C, const float* prior, cudaStream_t st);
 

@@ -1,6 +1,8 @@
-// Real-valued top layer on real-valued activations (the binary-weights-only networks of
-// Algorithm 1, whose last hidden layer hands on fp32 values), on the tensor cores:
-//   z[m][c] = sum_h Wout[c][h] * a[m][h] + b[c].
+// Real-valued layer on real-valued activations, on the tensor cores: the top layer of the
+// binary-weights-only networks of Algorithm 1 (whose last hidden layer hands on fp32 values) and
+// the real-valued hidden layers of the paper's mixed networks (Table 2), with an optional
+// activation f (Sigmoid, clamp):
+//   z[m][c] = f( sum_h Wout[c][h] * a[m][h] + b[c] ).
 //
 // Both operands are split into two fp16 terms.  The weights use the image bnn_output_prepare
 // builds (per-row power-of-two scaling, w * 2^e = w1 + w2, about 22 significant bits).  The
@@ -96,7 +98,7 @@ h_split_kernel(const float* __restrict__ Hf, int ldh, int M, int H, int nks, uin
 __global__ void __launch_bounds__(THREADS, 1)
 outf_tc_kernel(const uint8_t* __restrict__ himg, const uint8_t* __restrict__ wimg,
                const float* __restrict__ rs, const float* __restrict__ bias,
-               int M, int C, int H, float* __restrict__ Z, int ldz, int* __restrict__ status) {
+               int M, int C, int H, float* __restrict__ Z, int ldz, int act, int* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES);
@@ -211,7 +213,12 @@ outf_tc_kernel(const uint8_t* __restrict__ himg, const uint8_t* __restrict__ wim
                     float* dst = Z + (size_t)(f0 + gi * 32) * ldz + c;
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (f0 + gi * 32 + j < M) dst[(size_t)j * ldz] = fmaf(__uint_as_float(acc[j]), scl, bia);
+                        if (f0 + gi * 32 + j < M) {
+                            float v = fmaf(__uint_as_float(acc[j]), scl, bia);
+                            if (act == BNN_ACT_SIGMOID) v = 1.0f / (1.0f + expf(-v));
+                            else if (act == BNN_ACT_HARDTANH) v = fminf(fmaxf(v, -1.0f), 1.0f);
+                            dst[(size_t)j * ldz] = v;
+                        }
                 }
             }
             tc_fence_before_sync();
@@ -236,7 +243,7 @@ size_t outf_image_bytes(int M, int H) {
 }
 
 int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float* bias,
-                   int M, int C, int H, float* Z, int ldz, void* workspace, cudaStream_t st) {
+                   int M, int C, int H, float* Z, int ldz, int act, void* workspace, cudaStream_t st) {
     static bool configured = false;
     static int sms = 0;
     if (!configured) {
@@ -256,7 +263,7 @@ int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float*
     if (!status) return BNN_ERR_CUDA;
     h_split_kernel<<<ft * hs, FN, 0, st>>>(Hf, ldhf, M, H, hs, himg);
     const int tiles = ct * ft;
-    outf_tc_kernel<<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(himg, wimg, rs, bias, M, C, H, Z, ldz, status);
+    outf_tc_kernel<<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(himg, wimg, rs, bias, M, C, H, Z, ldz, act, status);
     return launch_status();
 }
 

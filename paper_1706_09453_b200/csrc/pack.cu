@@ -100,4 +100,25 @@ int launch_fold_thresholds(const float* scale, const float* shift, int N, int K,
     return launch_status();
 }
 
+// Binary layer with Sigmoid units: y = Sigmoid(fma(scale[n], d, shift[n])) for the integer dot
+// products d; Y may alias D (same pitch): every element is read and written by one thread.
+__global__ void affine_sigmoid_i32_kernel(const int32_t* D, int ldd, const float* __restrict__ scale,
+                                          const float* __restrict__ shift, int M, int N, float* Y, int ldy) {
+    const long long total = (long long)M * N;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int m = (int)(i / N), n = (int)(i % N);
+        const float v = fmaf(scale ? scale[n] : 1.0f, (float)D[(size_t)m * ldd + n], shift ? shift[n] : 0.0f);
+        Y[(size_t)m * ldy + n] = 1.0f / (1.0f + expf(-v));
+    }
+}
+
+int launch_affine_sigmoid_i32(const int32_t* D, int ldd, const float* scale, const float* shift,
+                              int M, int N, float* Y, int ldy, cudaStream_t st) {
+    const long long total = (long long)M * N;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    affine_sigmoid_i32_kernel<<<(int)blocks, 256, 0, st>>>(D, ldd, scale, shift, M, N, Y, ldy);
+    return launch_status();
+}
+
 }  // namespace bnn

@@ -161,6 +161,7 @@ real_gemm_kernel(RealGemmArgs g) {
             for (int j = 0; j < 4; ++j) {
                 y[j] = fmaf(sc[j], acc[i][jh * 4 + j], sh[j]);
                 if (g.act == BNN_ACT_HARDTANH) y[j] = fminf(fmaxf(y[j], -1.0f), 1.0f);
+                if (g.act == BNN_ACT_SIGMOID) y[j] = 1.0f / (1.0f + expf(-y[j]));
             }
             if (pack) {
 #pragma unroll

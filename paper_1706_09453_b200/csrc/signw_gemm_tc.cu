@@ -250,6 +250,7 @@ __global__ void __launch_bounds__(THREADS, 1) signw_tc_kernel(Args g) {
                 for (int j = 0; j < 32; ++j) {
                     float v = fmaf(ctl->sc[gi * 32 + j], __uint_as_float(acc[j]), ctl->sh[gi * 32 + j]);
                     if (g.act == BNN_ACT_HARDTANH) v = fminf(fmaxf(v, -1.0f), 1.0f);
+                    if (g.act == BNN_ACT_SIGMOID) v = 1.0f / (1.0f + expf(-v));
                     y[j] = v;
                     wd |= (uint32_t)(nb + j < N && sign_is_pos(v, g.sign_mode)) << j;
                 }

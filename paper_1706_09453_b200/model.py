@@ -33,19 +33,34 @@ class DeviceNet:
         self.Wp, self.scale, self.shift, self.thr, self.flip, self.Wimg = [], [], [], [], [], []
         layers = []
         binary_act = cfg.act == wl.ACT_SIGN
+        mixed = getattr(cfg, "mixed", False)
+        self.W0 = self.W0_prepared = None
         for l, w in enumerate(net.W):
             n, k = w.shape
             wd = to_dev(w, device)
+            if mixed and l == 0:
+                # real-valued Sigmoid layer: the weights as they are, prepared for the tensor cores
+                self.W0 = wd
+                self.W0_prepared = torch.empty(B.bnn_output_prepared_bytes(n, k), dtype=torch.uint8, device=device)
+                B.bnn_output_prepare(wd, self.W0_prepared)
+                sh = to_dev(net.shift[l], device)
+                self.Wp.append(None); self.scale.append(None); self.shift.append(sh)
+                self.thr.append(None); self.flip.append(None)
+                layers.append(dict(kind=B.LAYER_REAL, K=k, N=n, W=wd, W_prepared=self.W0_prepared, shift=sh,
+                                   act=B.ACT_SIGMOID))
+                continue
             wp = packed_empty(n, k, device)
             B.bnn_pack_weights(wd, wp, sign_mode)
             del wd
             sc, sh = to_dev(net.scale[l], device), to_dev(net.shift[l], device)
             self.Wp.append(wp); self.scale.append(sc); self.shift.append(sh)
-            if l == 0 or not binary_act:
+            first_binary = l == (1 if mixed else 0)
+            if first_binary or not binary_act:
                 layers.append(dict(kind=B.LAYER_SIGNW, K=k, N=n, Wp=wp, scale=sc, shift=sh,
                                    act=B.ACT_SIGN_PACK if binary_act else B.ACT_HARDTANH))
                 self.thr.append(None); self.flip.append(None)
             else:
+                last_sigmoid = mixed and l == len(net.W) - 1
                 thr = torch.empty(n, dtype=torch.int32, device=device)
                 flip = torch.empty((n + 31) // 32, dtype=torch.int32, device=device)
                 B.bnn_fold_thresholds(sc, sh, n, k, thr, flip, sign_mode)
@@ -56,7 +71,8 @@ class DeviceNet:
                     B.bnn_xnor_prepare(wp, k, img)
                 self.Wimg.append(img)
                 layers.append(dict(kind=B.LAYER_XNOR, K=k, N=n, Wp=wp, thr=thr, flip=flip, W_prepared=img,
-                                   act=B.ACT_SIGN_PACK))
+                                   scale=sc, shift=sh,
+                                   act=B.ACT_SIGMOID if last_sigmoid else B.ACT_SIGN_PACK))
         self.Wout, self.bout = to_dev(net.Wout, device), to_dev(net.bout, device)
         self.Wout_prepared = torch.empty(B.bnn_output_prepared_bytes(cfg.classes, cfg.hidden),
                                          dtype=torch.uint8, device=device)

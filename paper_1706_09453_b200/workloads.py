@@ -36,6 +36,8 @@ class Config:
     classes: int         # C
     act: int = ACT_SIGN  # hidden activation
     per_layer_alpha: bool = False  # binary-weights-only variant: scale = alpha_l, shift = 0
+    mixed: bool = False  # the paper's most accurate topology (Table 2): real-valued Sigmoid first layer,
+                         # binary layers with Sign units in between, binary last hidden layer with Sigmoid units
 
 
 CONFIGS = {
@@ -47,6 +49,8 @@ CONFIGS = {
     "wsj_bw": Config("wsj_bw", 2, 8192, 440, 2048, 6, 3400, ACT_HARDTANH, True),
     # AMI-scale: 600 -> 6 x 3072 -> 4000
     "ami": Config("ami", 3, 65536, 600, 3072, 6, 4000),
+    # mixed topology at the WSJ shape (sigma, b, b, b, b, sigma, softmax); first-layer weights ~ N(0, 1/K)
+    "wsj_mixed": Config("wsj_mixed", 5, 8192, 440, 2048, 6, 3400, mixed=True),
 }
 
 # Isolated XNOR GEMM sweep.
@@ -79,7 +83,13 @@ def make_model(cfg: Config, seed: int | None = None) -> Model:
     rng = np.random.Generator(np.random.PCG64(cfg.seed if seed is None else seed))
     m = Model(cfg)
     k = cfg.in_dim
-    for _ in range(cfg.n_hidden):
+    for l in range(cfg.n_hidden):
+        if cfg.mixed and l == 0:   # real-valued layer: weights and a bias (Eq. 1), no scale
+            m.W.append(rng.normal(0.0, 1.0 / np.sqrt(k), size=(cfg.hidden, k)).astype(np.float32))
+            m.scale.append(None)
+            m.shift.append(rng.normal(0.0, 0.1, size=cfg.hidden).astype(np.float32))
+            k = cfg.hidden
+            continue
         m.W.append(_signed_weights(rng, cfg.hidden, k))
         if cfg.per_layer_alpha:
             alpha = np.float32(rng.uniform(0.01, 0.1))

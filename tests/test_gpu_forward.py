@@ -247,3 +247,49 @@ def test_forward_spliced_input_and_log_prior(env, frames):
         B.bnn_forward(dn.desc, Fd[:, :40], logp, small)
     assert e.value.status == 5
     assert B.bnn_device_status() == 0
+
+
+def run_mixed_net(env, cfg, frames, sample=None, mode=0):
+    """The paper's mixed topology through bnn_forward: real-valued Sigmoid first layer, +-1 weights
+    with Sign units, +-1 x +-1 with Sign units, +-1 x +-1 with Sigmoid units, real Softmax layer."""
+    torch, B, model = env
+    net = wl.make_model(cfg)
+    X = wl.make_frames(cfg, frames)
+    dn = model.DeviceNet(net, mode)
+    outs = dn.layer_out_buffers(frames)
+    logp = dn.forward(model.to_dev(X), layer_out=outs)
+    torch.cuda.synchronize()
+    idx = np.arange(frames) if sample is None else np.asarray(sample)
+    g2 = model.words_to_numpy(outs[1], cfg.hidden)[idx]
+    ref = o.forward_mixed(X[idx], net.W, net.scale, net.shift, net.Wout, net.bout, mode, layer2_bits=g2)
+    # layer 1: Sigmoid units; the pre-activation is within 2^-17 sum|x||w| and |d sigmoid| <= |dz| / 4
+    bound = 0.25 * 2.0 ** -17 * (np.abs(X[idx]).astype(np.float64) @ np.abs(net.W[0]).astype(np.float64).T) + 2e-7
+    assert (np.abs(outs[0].cpu().numpy()[idx] - ref["h1"]) <= bound).all()
+    # layer 2: bits equal outside the float tolerance band
+    band = FLOAT_TOL * np.abs(net.scale[1])[None, :] * ref["sumabs2"][:, None]
+    decided = np.abs(ref["pre2"]) > band
+    np.testing.assert_array_equal(o.unpack_pm1(g2, cfg.hidden)[decided],
+                                  o.unpack_pm1(ref["bits_own_layer2"], cfg.hidden)[decided])
+    assert decided.mean() > 0.99, decided.mean()
+    # downstream of the GPU's own layer-2 bits: binary layers bit-exact, Sigmoid units and log-probs close
+    for l in range(2, cfg.n_hidden - 1):
+        np.testing.assert_array_equal(model.words_to_numpy(outs[l], cfg.hidden)[idx], ref["bits"][l - 1])
+    assert np.abs(outs[-1].cpu().numpy()[idx] - ref["hL"]).max() <= 1e-6
+    err = np.abs(logp.cpu().numpy()[idx] - ref["logp"]).max()
+    assert err <= LOGP_TOL, err
+    assert B.bnn_device_status() == 0
+
+
+def test_forward_mixed_topology_small(env):
+    import dataclasses
+    cfg = dataclasses.replace(wl.CONFIGS["wsj_mixed"], hidden=512, classes=700, frames=300, n_hidden=4)
+    run_mixed_net(env, cfg, 300)
+    run_mixed_net(env, cfg, 77, mode=1)
+
+
+def test_forward_mixed_topology_wsj_shape_sampled(env):
+    cfg = wl.CONFIGS["wsj_mixed"]
+    rng = np.random.default_rng(3)
+    sample = np.unique(np.concatenate([np.arange(64), np.arange(cfg.frames - 64, cfg.frames),
+                                       rng.integers(0, cfg.frames, 128)]))
+    run_mixed_net(env, cfg, cfg.frames, sample=sample)

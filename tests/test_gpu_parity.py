@@ -538,3 +538,45 @@ def test_pipe_rate_launches_run_and_report_their_work(B, torch_):
         B.bnn_pipe_rate(99, 1, scratch)               # unknown kind
     with pytest.raises(B.BnnError):
         B.bnn_pipe_rate(0, 1, scratch[:1024])         # scratch too small
+
+
+# ------------------------------------------------------------------ Sigmoid units (Table 2 topology)
+@pytest.mark.parametrize("m,k,n", [(300, 440, 1024), (33, 77, 129), (700, 2048, 520)])
+@pytest.mark.parametrize("tensor", [False, True])
+def test_real_layer_sigmoid(B, torch_, m, k, n, tensor):
+    """Real-valued weights x real input + bias, Sigmoid units (Eq. 1-2), FP32 pipe and tensor cores."""
+    rng = np.random.default_rng(m + k + n)
+    x = rng.standard_normal((m, k)).astype(np.float32)
+    w = rng.normal(0, 1 / np.sqrt(k), (n, k)).astype(np.float32)
+    b = rng.normal(0, 0.1, n).astype(np.float32)
+    prep = ws = None
+    if tensor:
+        prep = torch_.empty(B.bnn_output_prepared_bytes(n, k), dtype=torch_.uint8, device="cuda:0")
+        B.bnn_output_prepare(dev(w), prep)
+        ws = torch_.empty(B.bnn_output_workspace_bytes(m, k), dtype=torch_.uint8, device="cuda:0")
+    y = torch_.full((m, n + 2), 5.0, dtype=torch_.float32, device="cuda:0")
+    B.bnn_real_layer(dev(x), dev(w), dev(b), y[:, :n], B.ACT_SIGMOID, prepared=prep, workspace=ws)
+    _, want, _ = o.affine_act_f64(o.real_gemm_f32(x, w, b), None, None, o.ACT_SIGMOID)
+    got = y.cpu().numpy()
+    # |d sigmoid| <= |dz| / 4; the pre-activation is within 2^-17 sum|x||w| (tensor) or fp32 rounding
+    bound = 0.25 * 2.0 ** -17 * (np.abs(x).astype(np.float64) @ np.abs(w).astype(np.float64).T) + 2e-7
+    assert (np.abs(got[:, :n] - want) <= bound).all(), np.abs(got[:, :n] - want).max()
+    np.testing.assert_array_equal(got[:, n:], 5.0)
+    assert B.bnn_device_status() == 0
+
+
+def test_affine_sigmoid_i32_in_place(B, torch_):
+    rng = np.random.default_rng(77)
+    m, n = 130, 200
+    d = rng.integers(-2048, 2049, (m, n)).astype(np.int32)
+    sc = rng.uniform(-0.01, 0.01, n).astype(np.float32)
+    sh = rng.normal(0, 0.5, n).astype(np.float32)
+    want = o.affine_sigmoid_i32(d, sc, sh)
+    dd = dev(d)
+    y = torch_.empty((m, n), dtype=torch_.float32, device="cuda:0")
+    B.bnn_affine_sigmoid_i32(dd, dev(sc), dev(sh), y)
+    assert np.abs(y.cpu().numpy() - want).max() <= 2e-7
+    B.bnn_affine_sigmoid_i32(dd, dev(sc), dev(sh), dd.view(torch_.float32))     # same memory
+    assert torch_.equal(dd.view(torch_.float32), y)
+    B.bnn_affine_sigmoid_i32(dev(d), None, None, y)
+    assert np.abs(y.cpu().numpy() - o.affine_sigmoid_i32(d, None, None)).max() <= 2e-7
