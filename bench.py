@@ -259,6 +259,18 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
     else:
         rows.append(dict(name="output_gemm", kernel="real_gemm_kernel", work=owork, unit="TFLOP/s", bound="alu",
                          peak=fp32_peak))
+    if frames <= 16 and cfg.act == 1 and not mixed and xnor_path != "popc":
+        # a handful of frames: bnn_forward runs the matrix-vector kernels (one warp per unit), which
+        # are bound by reading each layer's weights once
+        for r in rows:
+            if r["name"].startswith("signw"):
+                r.update(kernel="small_signw_kernel", bound="alu", peak=fp32_peak, passes=1)
+            elif r["name"].startswith("xnor"):
+                r.update(kernel="small_xnor_kernel", bound="alu", peak=popc_peak)
+                r.pop("smem_bytes", None)
+            elif r["name"] == "output_gemm":
+                r.update(kernel="small_out_kernel", bound="hbm", unit="GB/s", peak=peaks["hbm_gbs"], scale=1e9, passes=1,
+                         work=4.0 * cfg.classes * cfg.hidden + 4.0 * frames * cfg.classes)
     # log-softmax: one read and one write of the [frames][classes] fp32 matrix
     rows.append(dict(name="log_softmax", kernel="log_softmax_rows_kernel", work=2.0 * frames * cfg.classes * 4,
                      unit="GB/s", bound="hbm", peak=peaks["hbm_gbs"], scale=1e9))

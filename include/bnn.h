@@ -374,9 +374,15 @@ BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, 
  *                        layers) runs for a fused Sign layer: BNN_PREPARED_STREAM reads the
  *                        weight image from L2 for every tile of frames; BNN_PREPARED_RESIDENT
  *                        keeps a tile of units' weights in shared memory for the whole launch
- *                        (needs K <= 3072; other shapes stream); AUTO picks by shape. */
+ *                        (needs K <= 3072; other shapes stream); AUTO picks by shape.
+ *   BNN_OPT_SMALL_BATCH: 1 (default) lets bnn_forward run batches of up to 16 frames -- the
+ *                        matrix-vector regime the paper has in mind for embedded recognisers
+ *                        (Section 1) -- on kernels that spread each layer's weights over all SMs,
+ *                        one warp per output unit, on the integer / FP32 pipes, instead of the
+ *                        tiled tensor-core kernels (about 4x lower latency); 0 turns that off.
+ *                        Integers and bits are identical; the fp32 sums differ by rounding order. */
 typedef enum { BNN_OPT_XNOR_PATH = 0, BNN_OPT_REAL_PATH = 1, BNN_OPT_SIGNW_TERMS = 2,
-               BNN_OPT_XNOR_PREPARED = 3 } bnn_option;
+               BNN_OPT_XNOR_PREPARED = 3, BNN_OPT_SMALL_BATCH = 4 } bnn_option;
 typedef enum { BNN_PATH_AUTO = 0, BNN_PATH_CUDA_CORE = 1, BNN_PATH_TENSOR = 2 } bnn_path;
 typedef enum { BNN_PREPARED_AUTO = 0, BNN_PREPARED_STREAM = 1, BNN_PREPARED_RESIDENT = 2 } bnn_prepared_kernel;
 BNN_API int bnn_set_option(int option, int value);

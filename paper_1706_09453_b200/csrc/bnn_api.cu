@@ -11,6 +11,7 @@ constexpr int kMaxK = 1 << 24;
 int g_xnor_path = BNN_PATH_AUTO;
 int g_real_path = BNN_PATH_AUTO;
 int g_xnor_prepared = BNN_PREPARED_AUTO;
+int g_small_batch = 1;  // batches of up to kSmallBatchMax frames take the matrix-vector kernels
 int g_signw_terms = 2;  // |dot| <= K stays exact in every accumulator type used
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
@@ -114,10 +115,13 @@ int bnn_set_option(int option, int value) {
         case BNN_OPT_REAL_PATH: slot = &g_real_path; break;
         case BNN_OPT_SIGNW_TERMS: slot = &g_signw_terms; break;
         case BNN_OPT_XNOR_PREPARED: slot = &g_xnor_prepared; break;
+        case BNN_OPT_SMALL_BATCH: slot = &g_small_batch; break;
         default: return -1;
     }
     if (option == BNN_OPT_SIGNW_TERMS) {
         if (value != 2 && value != 3) return -1;
+    } else if (option == BNN_OPT_SMALL_BATCH) {
+        if (value != 0 && value != 1) return -1;
     } else if (option == BNN_OPT_XNOR_PREPARED) {
         if (value != BNN_PREPARED_AUTO && value != BNN_PREPARED_STREAM && value != BNN_PREPARED_RESIDENT) return -1;
     } else if (value != BNN_PATH_AUTO && value != BNN_PATH_CUDA_CORE && value != BNN_PATH_TENSOR) {
@@ -463,11 +467,28 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
     const void* in = X;
     int in_ld = ldx;
     bool in_bits = false;
+    // A handful of frames: the layers made of packed bits take the matrix-vector kernels, which
+    // spread the weights over all SMs instead of tiling the frames (small_batch.cu).
+    const bool small = g_small_batch && M <= kSmallBatchMax;
+    const int zo01 = model->act_values == BNN_VALUES_01;
     for (int l = 0; l < L; ++l) {
         const bnn_layer& y = model->layers[l];
         if (events && events[l] &&
             cudaEventRecord((cudaEvent_t)events[l], (cudaStream_t)stream) != cudaSuccess)
             return BNN_ERR_CUDA;
+        if (y.kind == BNN_LAYER_REAL_OUT && small && in_bits && small_fits_bits(y.K)) {
+            if (int rc = check_packed(in, in_ld, y.K)) return rc;
+            if (int rc = launch_small_out(static_cast<const uint32_t*>(in), in_ld, y.W, y.ldw, y.shift, M, y.N, y.K,
+                                          logp, ldo, zo01, (cudaStream_t)stream)) return rc;
+            if (events && events[L + 1] &&
+                cudaEventRecord((cudaEvent_t)events[L + 1], (cudaStream_t)stream) != cudaSuccess)
+                return BNN_ERR_CUDA;
+            if (int rc = launch_log_softmax_rows(logp, ldo, M, y.N, model->log_prior, (cudaStream_t)stream)) return rc;
+            if (events && events[L] &&
+                cudaEventRecord((cudaEvent_t)events[L], (cudaStream_t)stream) != cudaSuccess)
+                return BNN_ERR_CUDA;
+            return BNN_OK;
+        }
         if (y.kind == BNN_LAYER_REAL_OUT) {
             int rc = output_layer_impl(in_bits ? static_cast<const uint32_t*>(in) : nullptr, in_ld,
                                        in_bits ? nullptr : static_cast<const float*>(in), in_ld,
@@ -486,7 +507,18 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
         e.act = y.act;
         e.sign_mode = model->sign_mode;
         int rc;
-        if (y.kind == BNN_LAYER_SIGNW) {
+        if (small && y.act == BNN_ACT_SIGN_PACK && y.kind == BNN_LAYER_SIGNW && !(l == 0 && splice_dim > 0) &&
+            small_fits_real(y.K)) {
+            const int ldob = bnn_packed_pitch(y.N);
+            rc = launch_small_signw(static_cast<const float*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K, y.scale, y.shift,
+                                    model->sign_mode, static_cast<uint32_t*>(out), ldob, (cudaStream_t)stream);
+            in_ld = ldob;
+        } else if (small && y.act == BNN_ACT_SIGN_PACK && y.kind == BNN_LAYER_XNOR && small_fits_bits(y.K)) {
+            const int ldob = bnn_packed_pitch(y.N);
+            rc = launch_small_xnor(static_cast<const uint32_t*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K, y.thr, y.flip,
+                                   static_cast<uint32_t*>(out), ldob, zo01, (cudaStream_t)stream);
+            in_ld = ldob;
+        } else if (y.kind == BNN_LAYER_SIGNW) {
             e.scale = y.scale; e.shift = y.shift;
             float* yf = nullptr;
             int out_ld;

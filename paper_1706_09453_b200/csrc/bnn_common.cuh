@@ -99,6 +99,21 @@ int launch_xnor_prepare(const uint32_t* Wp, int ldwp, int N, int K, void* image,
 int launch_xnor_img(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
                     int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
                     uint32_t* out_bits, int ldob, int zo, cudaStream_t st);
+// Small batches (small_batch.cu): plain kernels that spread a layer's weights over all SMs, one
+// warp per output unit, for M <= kSmallBatchMax frames.
+constexpr int kSmallBatchMax = 16;
+// Whether a layer of fan-in K fits those kernels (they stage the batch's operand in 48 KB of
+// shared memory: 16 x K floats for real input, 16 x K bits for packed input).
+inline bool small_fits_real(int K) { return (size_t)kSmallBatchMax * K * sizeof(float) <= 48 * 1024; }
+inline bool small_fits_bits(int K) { return (size_t)kSmallBatchMax * words_for(K) * sizeof(uint32_t) <= 48 * 1024; }
+int launch_small_signw(const float* X, int ldx, const uint32_t* Wp, int ldwp, int M, int N, int K,
+                       const float* scale, const float* shift, int sign_mode,
+                       uint32_t* out_bits, int ldob, cudaStream_t st);
+int launch_small_xnor(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp, int M, int N, int K,
+                      const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int zo,
+                      cudaStream_t st);
+int launch_small_out(const uint32_t* Hp, int ldhp, const float* W, int ldw, const float* bias,
+                     int M, int C, int H, float* Z, int ldz, int zo, cudaStream_t st);
 // Pipe micro-benchmarks (pipe_rates.cu).
 size_t pipe_rate_scratch_bytes(int which);
 int launch_pipe_rate(int which, int repeat, void* scratch, size_t scratch_bytes, double* work, cudaStream_t st);

@@ -103,6 +103,8 @@ def test_bad_arguments_are_rejected_without_a_launch(lib):
     assert B.bnn_set_option(B.OPT_XNOR_PATH, B.PATH_CUDA_CORE) == 0
     assert B.bnn_set_option(B.OPT_XNOR_PATH, B.PATH_AUTO) == 1
     assert rc("bnn_set_option", 9, 0) == -1 and rc("bnn_set_option", 2, 4) == -1
+    assert B.bnn_set_option(B.OPT_SMALL_BATCH, 0) == 1 and B.bnn_set_option(B.OPT_SMALL_BATCH, 1) == 0
+    assert rc("bnn_set_option", 4, 2) == -1
     assert rc("bnn_fold_thresholds", None, None, 4, 4, 0, None, fake, None) == 1
 
 

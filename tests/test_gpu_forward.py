@@ -293,3 +293,24 @@ def test_forward_mixed_topology_wsj_shape_sampled(env):
     sample = np.unique(np.concatenate([np.arange(64), np.arange(cfg.frames - 64, cfg.frames),
                                        rng.integers(0, cfg.frames, 128)]))
     run_mixed_net(env, cfg, cfg.frames, sample=sample)
+
+
+@pytest.mark.parametrize("frames", [1, 5, 16])
+@pytest.mark.parametrize("values", [0, 1])
+def test_forward_small_batch_kernels(env, frames, values):
+    """Batches of up to 16 frames run on the matrix-vector kernels (one warp per unit): same parity
+    with the oracle as the tiled kernels, for both activation value sets and both Sign conventions,
+    and on sizes that are not multiples of 32."""
+    import dataclasses
+    B = env[1]
+    assert B.bnn_set_option(B.OPT_SMALL_BATCH, 1) in (0, 1)
+    run_binary_net(env, wl.CONFIGS["tiny"], frames, values=values)
+    odd = dataclasses.replace(wl.CONFIGS["tiny"], hidden=1000, classes=3307, in_dim=441)
+    run_binary_net(env, odd, frames, values=values, mode=1)
+    # the tiled kernels on the same batch (option off) still agree with the oracle
+    prev = B.bnn_set_option(B.OPT_SMALL_BATCH, 0)
+    try:
+        run_binary_net(env, wl.CONFIGS["tiny"], frames, values=values)
+    finally:
+        B.bnn_set_option(B.OPT_SMALL_BATCH, prev)
+    assert B.bnn_device_status() == 0
