@@ -47,7 +47,7 @@ typedef enum {
     BNN_ERR_CUDA = 6         /* the CUDA runtime reported an error at launch */
 } bnn_status;
 
-/* Value of Sign at zero.  Eq. 3 of the paper reads "+1 if x > 0, -1 otherwise", i.e.
+/* Value of Sign at zero.  Eq. 3 of the paper gives +1 for x > 0 and -1 for everything else, i.e.
  * BNN_SIGN_ZERO_NEG.  BNN_SIGN_ZERO_POS is the other common convention (x >= 0 -> +1).
  * NaN maps to -1 in both modes (every comparison with NaN is false). */
 typedef enum { BNN_SIGN_ZERO_POS = 0, BNN_SIGN_ZERO_NEG = 1 } bnn_sign_mode;
