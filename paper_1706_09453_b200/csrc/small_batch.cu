@@ -148,9 +148,12 @@ small_out_kernel(const uint32_t* __restrict__ Hp, int ldhp, const float* __restr
     const int c = blockIdx.x * 8 + warp;
     if (c >= C) return;
     const float* w = W + (size_t)c * ldw;
-    float acc[MT];
+    // acc[m] = sum of the weights at the positions where frame m's bit is set (one predicated add
+    // per weight and frame); with +-1 activations z = 2 acc - (sum of all weights of the class).
+    float acc[MT], tot = 0.f;
 #pragma unroll
     for (int m = 0; m < MT; ++m) acc[m] = 0.f;
+    const uint32_t lanebit = 1u << lane;
     // eight independent loads of the class's weights in flight per lane: this kernel is bound by
     // how fast the 4 bytes per weight arrive
     for (int g0 = 0; g0 < hw; g0 += 8) {
@@ -163,19 +166,20 @@ small_out_kernel(const uint32_t* __restrict__ Hp, int ldhp, const float* __restr
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             if (g0 + u < hw) {
+                tot += wv[u];
 #pragma unroll
-                for (int m = 0; m < MT; ++m) {
-                    const bool one = (hs[m * hw + g0 + u] >> lane) & 1u;
-                    acc[m] += one ? wv[u] : (ZO ? 0.f : -wv[u]);
-                }
+                for (int m = 0; m < MT; ++m)
+                    if (hs[m * hw + g0 + u] & lanebit) acc[m] += wv[u];
             }
         }
     }
     const float b = bias ? bias[c] : 0.f;
+    tot = warp_sum(tot);
 #pragma unroll
     for (int m = 0; m < MT; ++m)
         if (m < M) {
-            const float z = warp_sum(acc[m]) + b;
+            const float s1 = warp_sum(acc[m]);
+            const float z = (ZO ? s1 : 2.0f * s1 - tot) + b;
             if (lane == 0) Z[(size_t)m * ldz + c] = z;
         }
 }
