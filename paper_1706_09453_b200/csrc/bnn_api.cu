@@ -476,7 +476,7 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
         if (events && events[l] &&
             cudaEventRecord((cudaEvent_t)events[l], (cudaStream_t)stream) != cudaSuccess)
             return BNN_ERR_CUDA;
-        if (y.kind == BNN_LAYER_REAL_OUT && small && in_bits && small_fits_bits(y.K)) {
+        if (y.kind == BNN_LAYER_REAL_OUT && small && in_bits && small_fits_out(y.K)) {
             if (int rc = check_packed(in, in_ld, y.K)) return rc;
             if (int rc = launch_small_out(static_cast<const uint32_t*>(in), in_ld, y.W, y.ldw, y.shift, M, y.N, y.K,
                                           logp, ldo, zo01, (cudaStream_t)stream)) return rc;

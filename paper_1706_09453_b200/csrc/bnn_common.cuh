@@ -106,6 +106,7 @@ constexpr int kSmallBatchMax = 16;
 // shared memory: 16 x K floats for real input, 16 x K bits for packed input).
 inline bool small_fits_real(int K) { return (size_t)kSmallBatchMax * K * sizeof(float) <= 48 * 1024; }
 inline bool small_fits_bits(int K) { return (size_t)kSmallBatchMax * words_for(K) * sizeof(uint32_t) <= 48 * 1024; }
+inline bool small_fits_out(int H) { return (size_t)words_for(H) * 32 * sizeof(uint16_t) <= 48 * 1024; }
 int launch_small_signw(const float* X, int ldx, const uint32_t* Wp, int ldwp, int M, int N, int K,
                        const float* scale, const float* shift, int sign_mode,
                        uint32_t* out_bits, int ldob, cudaStream_t st);

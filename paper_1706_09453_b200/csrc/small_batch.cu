@@ -52,6 +52,7 @@ small_signw_kernel(const float* __restrict__ X, int ldx, const uint32_t* __restr
                    int sign_mode, uint32_t* __restrict__ out_bits, int ldob) {
     __shared__ unsigned char dec[32][MAXM];
     extern __shared__ float xs[];   // the batch's input, [MT][K]; rows >= M are zero
+    __shared__ float xsum[MT];      // sum_k x[m][k], the same for every unit
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * 32, n = n0 + warp;
     for (int i = threadIdx.x; i < MT * K; i += blockDim.x) {
@@ -59,6 +60,15 @@ small_signw_kernel(const float* __restrict__ X, int ldx, const uint32_t* __restr
         xs[i] = m < M ? __ldg(X + (size_t)m * ldx + k) : 0.f;
     }
     __syncthreads();
+    if (warp < MT) {   // warp m adds up row m
+        float t = 0.f;
+        for (int k = lane; k < K; k += 32) t += xs[warp * K + k];
+        t = warp_sum(t);
+        if (lane == 0) xsum[warp] = t;
+    }
+    __syncthreads();
+    // sum_k w x = 2 * (sum of x where the weight bit is set) - sum_k x: one predicated add per
+    // position and frame
     float acc[MT];
 #pragma unroll
     for (int m = 0; m < MT; ++m) acc[m] = 0.f;
@@ -67,12 +77,9 @@ small_signw_kernel(const float* __restrict__ X, int ldx, const uint32_t* __restr
         for (int k0 = 0; k0 < K; k0 += 32) {
             const int k = k0 + lane;
             const bool plus = (__ldg(w + (k0 >> 5)) >> lane) & 1u;
-            if (k < K) {
+            if (k < K && plus) {
 #pragma unroll
-                for (int m = 0; m < MT; ++m) {
-                    const float x = xs[m * K + k];
-                    acc[m] += plus ? x : -x;
-                }
+                for (int m = 0; m < MT; ++m) acc[m] += xs[m * K + k];
             }
         }
     }
@@ -80,7 +87,7 @@ small_signw_kernel(const float* __restrict__ X, int ldx, const uint32_t* __restr
 #pragma unroll
     for (int m = 0; m < MT; ++m)
         if (m < M) {
-            const float y = fmaf(sc, warp_sum(acc[m]), sh);
+            const float y = fmaf(sc, 2.0f * warp_sum(acc[m]) - xsum[m], sh);
             if (lane == 0) dec[warp][m] = sign_is_pos(y, sign_mode);
         }
     __syncthreads();
@@ -137,12 +144,18 @@ template <bool ZO, int MT>
 __global__ void __launch_bounds__(256)
 small_out_kernel(const uint32_t* __restrict__ Hp, int ldhp, const float* __restrict__ W, int ldw,
                  const float* __restrict__ bias, int M, int C, int H, float* __restrict__ Z, int ldz) {
-    extern __shared__ uint32_t hs[];   // the batch's packed activations, [MT][hw]; rows >= M are zero
+    // fm[g][lane]: bit m set <=> frame m has a one at position 32 g + lane (frames >= M: clear).
+    // Built once per block; the inner loop then needs one shared-memory load per weight.
+    extern __shared__ uint16_t fm[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hw = words_for(H);
-    for (int i = threadIdx.x; i < MT * hw; i += blockDim.x) {
-        const int m = i / hw, g = i - m * hw;
-        hs[i] = m < M ? __ldg(Hp + (size_t)m * ldhp + g) : 0u;
+    for (int i = threadIdx.x; i < hw * 32; i += blockDim.x) {
+        const int g = i >> 5, l = i & 31;
+        uint32_t t = 0u;
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (m < M) t |= ((__ldg(Hp + (size_t)m * ldhp + g) >> l) & 1u) << m;
+        fm[i] = (uint16_t)t;
     }
     __syncthreads();
     const int c = blockIdx.x * 8 + warp;
@@ -153,7 +166,6 @@ small_out_kernel(const uint32_t* __restrict__ Hp, int ldhp, const float* __restr
     float acc[MT], tot = 0.f;
 #pragma unroll
     for (int m = 0; m < MT; ++m) acc[m] = 0.f;
-    const uint32_t lanebit = 1u << lane;
     // eight independent loads of the class's weights in flight per lane: this kernel is bound by
     // how fast the 4 bytes per weight arrive
     for (int g0 = 0; g0 < hw; g0 += 8) {
@@ -167,9 +179,10 @@ small_out_kernel(const uint32_t* __restrict__ Hp, int ldhp, const float* __restr
         for (int u = 0; u < 8; ++u) {
             if (g0 + u < hw) {
                 tot += wv[u];
+                const uint32_t t = fm[(g0 + u) * 32 + lane];
 #pragma unroll
                 for (int m = 0; m < MT; ++m)
-                    if (hs[m * hw + g0 + u] & lanebit) acc[m] += wv[u];
+                    if (t & (1u << m)) acc[m] += wv[u];
             }
         }
     }
@@ -217,7 +230,7 @@ int launch_small_xnor(const uint32_t* Ap, int ldap, const uint32_t* Wp, int ldwp
 
 int launch_small_out(const uint32_t* Hp, int ldhp, const float* W, int ldw, const float* bias,
                      int M, int C, int H, float* Z, int ldz, int zo, cudaStream_t st) {
-    const size_t smem = (size_t)frames_bound(M) * words_for(H) * sizeof(uint32_t);
+    const size_t smem = (size_t)words_for(H) * 32 * sizeof(uint16_t);
     if (M > MAXM || smem > kSmallSmemMax) return BNN_ERR_UNSUPPORTED;
     if (zo)
         BNN_SMALL_DISPATCH(M, (small_out_kernel<true, MT><<<ceil_div(C, 8), 256, smem, st>>>(Hp, ldhp, W, ldw, bias, M, C, H, Z, ldz)));
