@@ -314,3 +314,14 @@ def test_forward_small_batch_kernels(env, frames, values):
     finally:
         B.bnn_set_option(B.OPT_SMALL_BATCH, prev)
     assert B.bnn_device_status() == 0
+
+
+def test_forward_small_batch_other_topologies(env):
+    """A few frames through the networks whose layers only partly have matrix-vector kernels
+    (fp32 activations, Sigmoid units): small and tiled kernels chain on the same buffers."""
+    import dataclasses
+    bw = dataclasses.replace(wl.CONFIGS["wsj_bw"], hidden=512, classes=700, frames=5)
+    run_bw_net(env, bw, 5)
+    mixed = dataclasses.replace(wl.CONFIGS["wsj_mixed"], hidden=512, classes=700, frames=7, n_hidden=4)
+    run_mixed_net(env, mixed, 7)
+    run_mixed_net(env, wl.CONFIGS["wsj_mixed"], 3)
