@@ -37,6 +37,15 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
 }
 
+// 16-byte read-only global load issued exactly where it is written (a volatile asm keeps its place
+// among the other volatile statements: barrier waits, shared-memory stores).  Producer warps use it
+// to fetch operands for later pipeline stages while they work on the current one.
+__device__ __forceinline__ uint4 ldg_nc_u4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
 // Programmatic dependent launch, used by the kernel of the binary hidden layers: it starts with
 // pdl_trigger() (the kernel after it in the stream may be scheduled as soon as all CTAs of this
 // one have got that far and SM resources free up), does what does not depend on the kernel

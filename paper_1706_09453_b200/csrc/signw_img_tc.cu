@@ -44,7 +44,7 @@ template <int NT> struct Cfg {
 
 struct Control {
     float sc[UN], sh[UN];
-    uint64_t full[4], empty[4], acc_full, acc_empty;
+    uint64_t full[4], empty[4], acc_full, acc_empty[2];
     uint32_t tmem_base;
     int abort;
 };
@@ -69,6 +69,7 @@ __global__ void __launch_bounds__(256)
 x_split_kernel(const float* __restrict__ X, int ldx, int M, int K, int nks, uint8_t* __restrict__ img,
                int sdim, int sleft) {
     __shared__ float raw[BM][BK + 1];
+    pdl_trigger();   // the GEMM may be scheduled as SMs free up; it waits before it reads the image
     const int mt = blockIdx.x / nks, ks = blockIdx.x % nks;
     const int t = threadIdx.x;
     // coalesced read: 8 consecutive threads fetch the 32 floats of one row segment.  With splicing
@@ -135,6 +136,131 @@ x_split_kernel(const float* __restrict__ X, int ldx, int M, int K, int nks, uint
     }
 }
 
+
+// TMEM -> registers: lane i of the warp reads 16 columns of TMEM lane (base lane + i).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+
+// Sign of 16 affine outputs: bit j = (Sign(fma(sc[j], acc[j], sh[j])) is +1).
+// sc / sh: 16-byte aligned shared memory.
+template <bool ZERO_NEG>
+__device__ __forceinline__ uint32_t sign_bits16(const uint32_t (&acc)[16], const float* sc, const float* sh) {
+    const float4* s4 = reinterpret_cast<const float4*>(sc);
+    const float4* h4 = reinterpret_cast<const float4*>(sh);
+    uint32_t wd = 0u;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float4 s = s4[q], h = h4[q];
+        const float v0 = fmaf(s.x, __uint_as_float(acc[4 * q + 0]), h.x);
+        const float v1 = fmaf(s.y, __uint_as_float(acc[4 * q + 1]), h.y);
+        const float v2 = fmaf(s.z, __uint_as_float(acc[4 * q + 2]), h.z);
+        const float v3 = fmaf(s.w, __uint_as_float(acc[4 * q + 3]), h.w);
+        wd |= (uint32_t)(ZERO_NEG ? v0 > 0.0f : v0 >= 0.0f) << (4 * q + 0);
+        wd |= (uint32_t)(ZERO_NEG ? v1 > 0.0f : v1 >= 0.0f) << (4 * q + 1);
+        wd |= (uint32_t)(ZERO_NEG ? v2 > 0.0f : v2 >= 0.0f) << (4 * q + 2);
+        wd |= (uint32_t)(ZERO_NEG ? v3 > 0.0f : v3 >= 0.0f) << (4 * q + 3);
+    }
+    return wd;
+}
+
+template <int ACT>
+__device__ __forceinline__ float activate(float v) {
+    if (ACT == BNN_ACT_HARDTANH) return fminf(fmaxf(v, -1.0f), 1.0f);
+    if (ACT == BNN_ACT_SIGMOID) return 1.0f / (1.0f + expf(-v));
+    return v;
+}
+
+// Epilogue of one 256-column accumulator for a layer that hands on nothing but bits.
+template <bool ZERO_NEG>
+__device__ __forceinline__ void epilogue_bits(uint32_t taddr, const float* sc, const float* sh, int cols_left,
+                                              uint32_t* dst, int words_left, bool row_ok) {
+    // (loads of columns beyond the layer's last unit stay inside the accumulator; their bits are
+    // masked to zero and never stored)
+    uint32_t a0[16], a1[16];
+    tmem_ld16(taddr, a0);
+#pragma unroll 1
+    for (int q4 = 0; q4 < 2; ++q4) {              // 128 columns = four words = one 16-byte store
+        if (q4 * 128 >= cols_left) break;         // uniform over the CTA
+        uint32_t words[4];
+#pragma unroll
+        for (int gq = 0; gq < 4; ++gq) {
+            const int c = q4 * 128 + gq * 32;
+            tmem_ld_wait();
+            tmem_ld16(taddr + c + 16, a1);
+            uint32_t wd = sign_bits16<ZERO_NEG>(a0, sc + c, sh + c);
+            tmem_ld_wait();
+            if (c + 32 < 256) tmem_ld16(taddr + c + 32, a0);
+            wd |= sign_bits16<ZERO_NEG>(a1, sc + c + 16, sh + c + 16) << 16;
+            const int valid = cols_left - c;
+            words[gq] = valid >= 32 ? wd : (valid > 0 ? (wd & ((1u << valid) - 1u)) : 0u);
+        }
+        if (row_ok) {
+            if (q4 * 4 + 4 <= words_left) {
+                *reinterpret_cast<uint4*>(dst + q4 * 4) = make_uint4(words[0], words[1], words[2], words[3]);
+            } else {
+#pragma unroll
+                for (int gq = 0; gq < 4; ++gq)
+                    if (q4 * 4 + gq < words_left) dst[q4 * 4 + gq] = words[gq];
+            }
+        }
+    }
+    tmem_ld_wait();
+}
+
+// Epilogue of one 256-column accumulator with an fp32 output (and packed bits as well when the
+// activation is Sign).
+template <int ACT>
+__device__ __forceinline__ void epilogue_real(uint32_t taddr, const float* sc, const float* sh, int cols_left,
+                                              float* y, bool vec, uint32_t* bits, int words_left, bool row_ok,
+                                              int sign_mode) {
+    uint32_t a0[16], a1[16];
+    tmem_ld16(taddr, a0);
+    auto emit = [&](uint32_t (&a)[16], int c) -> uint32_t {   // columns c .. c+15 of the accumulator
+        uint32_t wd = 0u;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float v = activate<ACT>(fmaf(sc[c + j], __uint_as_float(a[j]), sh[c + j]));
+            a[j] = __float_as_uint(v);
+            if (ACT == BNN_ACT_SIGN_PACK) wd |= (uint32_t)sign_is_pos(v, sign_mode) << j;
+        }
+        if (y && row_ok && c < cols_left) {
+            if (vec && c + 16 <= cols_left) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    reinterpret_cast<float4*>(y + c)[q] = make_float4(__uint_as_float(a[4 * q]), __uint_as_float(a[4 * q + 1]),
+                                                                      __uint_as_float(a[4 * q + 2]), __uint_as_float(a[4 * q + 3]));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (c + j < cols_left) y[c + j] = __uint_as_float(a[j]);
+            }
+        }
+        return wd;
+    };
+#pragma unroll 1
+    for (int gi = 0; gi < 8; ++gi) {              // one packed word per iteration
+        const int c = gi * 32;
+        if (c >= cols_left) break;                // uniform over the CTA
+        tmem_ld_wait();
+        tmem_ld16(taddr + c + 16, a1);
+        uint32_t wd = emit(a0, c);
+        tmem_ld_wait();
+        if (c + 32 < 256) tmem_ld16(taddr + c + 32, a0);
+        wd |= emit(a1, c + 16) << 16;
+        if (ACT == BNN_ACT_SIGN_PACK && bits && row_ok && gi < words_left) {
+            const int valid = cols_left - c;
+            bits[gi] = valid >= 32 ? wd : (wd & ((1u << valid) - 1u));
+        }
+    }
+    tmem_ld_wait();
+}
+
 struct Args {
     const uint8_t* img;
     const uint32_t* Wp; int ldwp;
@@ -166,7 +292,8 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->acc_full), 1);
-        mbar_init(smem_u32(&ctl->acc_empty), EPI_WARPS);
+        mbar_init(smem_u32(&ctl->acc_empty[0]), EPI_WARPS);
+        mbar_init(smem_u32(&ctl->acc_empty[1]), EPI_WARPS);
         ctl->abort = 0;
         mbar_init_fence();
     }
@@ -197,7 +324,7 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int n = n0 + p + 256 * q;
-                if (n < N) o[q] = __ldg(reinterpret_cast<const uint4*>(g.Wp + (size_t)n * g.ldwp) + pf_g);
+                if (n < N) o[q] = ldg_nc_u4(reinterpret_cast<const uint4*>(g.Wp + (size_t)n * g.ldwp) + pf_g);
             }
             if (++pf_g == ngroups) { pf_g = 0; pf_tile += gridDim.x; --pf_left; }
         };
@@ -215,6 +342,9 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
             if (!warp_wait(smem_u32(&ctl->empty[s]), ph, abort_flag, lane)) break;
             const uint32_t st = smem_u32(smem) + s * C::STAGE_BYTES;
             if (p == 0) {
+                // the image is the output of the kernel before this one in the stream: wait until that
+                // kernel has completed and its writes are visible (the weights do not depend on it)
+                if (it == 0) pdl_wait();
                 const int mt = tile % m_tiles;
                 mbar_expect_tx(smem_u32(&ctl->full[s]), C::A_BYTES);
                 bulk_g2s(st, g.img + ((size_t)mt * nks + ks) * C::A_BYTES, C::A_BYTES, smem_u32(&ctl->full[s]));
@@ -243,32 +373,55 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
     } else if (warp == MMA_WARP) {
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc(kAccF32, kFmtBF16, kFmtBF16, BM, 256);
+            // MMAs of one stage into accumulator `sub` (units [256 sub, 256 sub + 256) of the tile)
+            auto issue = [&](int s, int sub, int ks) {
+                const uint32_t a0 = smem_u32(smem + s * C::STAGE_BYTES);
+                const uint32_t b0 = a0 + C::A_BYTES;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (UN * 16) + sub * 256 * 16, UN * 16, 128);
+#pragma unroll
+                    for (int q = 0; q < NT; ++q) {
+                        const uint64_t da = smem_desc_kmajor(a0 + q * A_PLANE + 2 * j * (BM * 16), BM * 16, 128);
+                        mma_f16(tmem + sub * 256, da, db, idesc, (ks | j | q) != 0);
+                    }
+                }
+            };
             int it = 0, tl = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
-                ok = mbar_wait(smem_u32(&ctl->acc_empty), (uint32_t)((tl & 1) ^ 1), abort_flag);
+                const uint32_t par = (uint32_t)((tl & 1) ^ 1);
+                // The epilogue hands accumulator 0 back first.  The first stages go into it alone
+                // (their slots stay occupied) until accumulator 1 is free as well; then accumulator 1
+                // catches up and the stages are released.
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[0]), par, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
-                for (int ks = 0; ks < nks; ++ks, ++it) {
+                const int lead = nks < C::STAGES ? nks : C::STAGES;
+                for (int ks = 0; ks < lead && ok; ++ks) {
+                    const int s = (it + ks) % C::STAGES;
+                    ok = mbar_wait(smem_u32(&ctl->full[s]), (uint32_t)(((it + ks) / C::STAGES) & 1), abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue(s, 0, ks);
+                }
+                if (!ok) break;
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[1]), par, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int ks = 0; ks < lead; ++ks) {
+                    const int s = (it + ks) % C::STAGES;
+                    issue(s, 1, ks);
+                    mma_commit(smem_u32(&ctl->empty[s]));
+                }
+                it += lead;
+                for (int ks = lead; ks < nks; ++ks, ++it) {
                     const int s = it % C::STAGES;
                     ok = mbar_wait(smem_u32(&ctl->full[s]), (uint32_t)((it / C::STAGES) & 1), abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t a0 = smem_u32(smem + s * C::STAGE_BYTES);
-                    const uint32_t b0 = a0 + C::A_BYTES;
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-#pragma unroll
-                        for (int sub = 0; sub < 2; ++sub) {
-                            // rows [256 sub, 256 sub + 256) of the unit tile
-                            const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (UN * 16) + sub * 256 * 16, UN * 16, 128);
-#pragma unroll
-                            for (int q = 0; q < NT; ++q) {
-                                const uint64_t da = smem_desc_kmajor(a0 + q * A_PLANE + 2 * j * (BM * 16), BM * 16, 128);
-                                mma_f16(tmem + sub * 256, da, db, idesc, (ks | j | q) != 0);
-                            }
-                        }
-                    }
+                    issue(s, 0, ks);
+                    issue(s, 1, ks);
                     mma_commit(smem_u32(&ctl->empty[s]));
                 }
                 if (ok) mma_commit(smem_u32(&ctl->acc_full));
@@ -297,57 +450,35 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
             ok = epi_all(warp_wait(smem_u32(&ctl->acc_full), (uint32_t)(tl & 1), abort_flag, lane));
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
 #pragma unroll 1
-            for (int q4 = 0; q4 < UN / 128; ++q4) {           // 4 groups of 32 columns = one 16-byte store of bits
-                if (n0 + q4 * 128 >= N) break;                // uniform over the CTA
-                uint32_t words[4];
-#pragma unroll
-                for (int gq = 0; gq < 4; ++gq) {
-                    const int gi = q4 * 4 + gq;
-                    uint32_t acc[32];
-                    tmem_ld32(taddr + gi * 32, acc);
-                    tmem_ld_wait();
-                    const int nb = n0 + gi * 32;
-                    float y[32];
-                    uint32_t wd = 0u;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float v = fmaf(ctl->sc[gi * 32 + j], __uint_as_float(acc[j]), ctl->sh[gi * 32 + j]);
-                        if (g.act == BNN_ACT_HARDTANH) v = fminf(fmaxf(v, -1.0f), 1.0f);
-                        if (g.act == BNN_ACT_SIGMOID) v = 1.0f / (1.0f + expf(-v));
-                        y[j] = v;
-                        wd |= (uint32_t)(nb + j < N && sign_is_pos(v, g.sign_mode)) << j;
-                    }
-                    words[gq] = wd;
-                    if (g.Y && m < M && nb < N) {
-                        float* dst = g.Y + (size_t)m * g.ldy + nb;
-                        if (vy && nb + 31 < N) {
-#pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                reinterpret_cast<float4*>(dst)[q] = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (nb + j < N) dst[j] = y[j];
-                        }
-                    }
-                }
-                if (pack && m < M) {
-                    const int w0 = (n0 >> 5) + q4 * 4;
-                    uint32_t* dst = g.out_bits + (size_t)m * g.ldob + w0;
-                    if (w0 + 4 <= nw) {
-                        *reinterpret_cast<uint4*>(dst) = make_uint4(words[0], words[1], words[2], words[3]);
+            for (int sub = 0; sub < 2; ++sub) {
+                const int c0 = sub * 256, left = N - (n0 + c0);        // columns of this accumulator that exist
+                if (left > 0) {                                        // uniform over the CTA
+                    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
+                    const int w0 = (n0 + c0) >> 5;
+                    uint32_t* bits = g.out_bits ? g.out_bits + (size_t)(m < M ? m : 0) * g.ldob + w0 : nullptr;
+                    float* y = g.Y ? g.Y + (size_t)(m < M ? m : 0) * g.ldy + n0 + c0 : nullptr;
+                    const float* sc = &ctl->sc[c0];
+                    const float* sh = &ctl->sh[c0];
+                    if (pack && !g.Y) {
+                        if (g.sign_mode == kSignZeroNeg) epilogue_bits<true>(taddr, sc, sh, left, bits, nw - w0, m < M);
+                        else epilogue_bits<false>(taddr, sc, sh, left, bits, nw - w0, m < M);
+                    } else if (pack) {
+                        epilogue_real<BNN_ACT_SIGN_PACK>(taddr, sc, sh, left, y, vy, bits, nw - w0, m < M, g.sign_mode);
+                    } else if (g.act == BNN_ACT_HARDTANH) {
+                        epilogue_real<BNN_ACT_HARDTANH>(taddr, sc, sh, left, y, vy, nullptr, 0, m < M, g.sign_mode);
+                    } else if (g.act == BNN_ACT_SIGMOID) {
+                        epilogue_real<BNN_ACT_SIGMOID>(taddr, sc, sh, left, y, vy, nullptr, 0, m < M, g.sign_mode);
                     } else {
-#pragma unroll
-                        for (int gq = 0; gq < 4; ++gq)
-                            if (w0 + gq < nw) dst[gq] = words[gq];
+                        epilogue_real<BNN_ACT_NONE>(taddr, sc, sh, left, y, vy, nullptr, 0, m < M, g.sign_mode);
                     }
                 }
+                // accumulator `sub` is free again: the MMA thread starts the next tile on accumulator 0
+                // while accumulator 1 is still being read
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[sub]));
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty));
         }
     }
 
@@ -381,7 +512,8 @@ int launch_nt(const RealGemmArgs& r, void* workspace, cudaStream_t st) {
            tc_status_ptr()};
     if (!a.status) return BNN_ERR_CUDA;
     const int tiles = mt * ceil_div(r.N, UN);
-    signw_img_kernel<NT><<<tiles < sms ? tiles : sms, THREADS, SMEM, st>>>(a);
+    if (launch_pdl(signw_img_kernel<NT>, dim3(tiles < sms ? tiles : sms), dim3(THREADS), SMEM, st, a) != cudaSuccess)
+        return BNN_ERR_CUDA;
     return launch_status();
 }
 
