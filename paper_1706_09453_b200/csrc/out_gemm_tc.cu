@@ -38,7 +38,7 @@ constexpr int THREADS = (PROD_WARP0 + PROD_WARPS) * 32;
 constexpr uint32_t TMEM_COLS = 512;
 
 struct Control {
-    uint64_t full[STAGES], empty[STAGES], acc_full, acc_empty;
+    uint64_t full[STAGES], empty[STAGES], acc_full, acc_empty[2];
     uint32_t tmem_base;
     int abort;
 };
@@ -127,7 +127,8 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         mbar_init(smem_u32(&ctl->acc_full), 1);
-        mbar_init(smem_u32(&ctl->acc_empty), EPI_WARPS);
+        mbar_init(smem_u32(&ctl->acc_empty[0]), EPI_WARPS);
+        mbar_init(smem_u32(&ctl->acc_empty[1]), EPI_WARPS);
         ctl->abort = 0;
         mbar_init_fence();
     }
@@ -158,7 +159,7 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 const int f = f0 + p + 256 * q;
-                if (f < M) o[q] = __ldg(reinterpret_cast<const uint4*>(Hp + (size_t)f * ldhp) + pf_g);
+                if (f < M) o[q] = ldg_nc_u4(reinterpret_cast<const uint4*>(Hp + (size_t)f * ldhp) + pf_g);
             }
             if (++pf_g == ngroups) { pf_g = 0; pf_tile += gridDim.x; --pf_left; }
         };
@@ -209,32 +210,55 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
     } else if (warp == MMA_WARP) {
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc(kAccF32, kFmtF16, kFmtF16, BC, 256);
+            // MMAs of one stage into accumulator `sub` (frames [256 sub, 256 sub + 256) of the tile)
+            auto issue = [&](int s, int sub, int ks) {
+                const uint32_t a0 = smem_u32(smem + s * STAGE_BYTES);
+                const uint32_t b0 = a0 + A_BYTES;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (FN * 16) + sub * 256 * 16, FN * 16, 128);
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const uint64_t da = smem_desc_kmajor(a0 + q * A_PLANE + 2 * j * (BC * 16), BC * 16, 128);
+                        mma_f16(tmem + sub * 256, da, db, idesc, (ks | j | q) != 0);
+                    }
+                }
+            };
             int it = 0, tl = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
-                ok = mbar_wait(smem_u32(&ctl->acc_empty), (uint32_t)((tl & 1) ^ 1), abort_flag);
+                const uint32_t par = (uint32_t)((tl & 1) ^ 1);
+                // The epilogue hands accumulator 0 back first.  The first stages go into it alone
+                // (their slots stay occupied) until accumulator 1 is free as well; then accumulator 1
+                // catches up and the stages are released.
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[0]), par, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
-                for (int ks = 0; ks < nks; ++ks, ++it) {
+                const int lead = nks < STAGES ? nks : STAGES;
+                for (int ks = 0; ks < lead && ok; ++ks) {
+                    const int s = (it + ks) % STAGES;
+                    ok = mbar_wait(smem_u32(&ctl->full[s]), (uint32_t)(((it + ks) / STAGES) & 1), abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue(s, 0, ks);
+                }
+                if (!ok) break;
+                ok = mbar_wait(smem_u32(&ctl->acc_empty[1]), par, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                for (int ks = 0; ks < lead; ++ks) {
+                    const int s = (it + ks) % STAGES;
+                    issue(s, 1, ks);
+                    mma_commit(smem_u32(&ctl->empty[s]));
+                }
+                it += lead;
+                for (int ks = lead; ks < nks; ++ks, ++it) {
                     const int s = it % STAGES;
                     ok = mbar_wait(smem_u32(&ctl->full[s]), (uint32_t)((it / STAGES) & 1), abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t a0 = smem_u32(smem + s * STAGE_BYTES);
-                    const uint32_t b0 = a0 + A_BYTES;
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-#pragma unroll
-                        for (int sub = 0; sub < 2; ++sub) {
-                            // rows [256 sub, 256 sub + 256) of the frame tile
-                            const uint64_t db = smem_desc_kmajor(b0 + 2 * j * (FN * 16) + sub * 256 * 16, FN * 16, 128);
-#pragma unroll
-                            for (int q = 0; q < 2; ++q) {
-                                const uint64_t da = smem_desc_kmajor(a0 + q * A_PLANE + 2 * j * (BC * 16), BC * 16, 128);
-                                mma_f16(tmem + sub * 256, da, db, idesc, (ks | j | q) != 0);
-                            }
-                        }
-                    }
+                    issue(s, 0, ks);
+                    issue(s, 1, ks);
                     mma_commit(smem_u32(&ctl->empty[s]));
                 }
                 if (ok) mma_commit(smem_u32(&ctl->acc_full));
@@ -244,6 +268,8 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
     } else {
         // ---------------- epilogue: thread = one class (TMEM lane), columns = frames
         const int row_in_tile = warp * 32 + lane;
+        uint64_t pol;
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
         int tl = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
@@ -265,12 +291,23 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
                     float* dst = Z + (size_t)(f0 + gi * 32) * ldz + c;
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (f0 + gi * 32 + j < M) dst[(size_t)j * ldz] = fmaf(__uint_as_float(acc[j]), scl, bia);
+                        if (f0 + gi * 32 + j < M) {
+                            const float zv = fmaf(__uint_as_float(acc[j]), scl, bia);
+                            asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(dst + (size_t)j * ldz), "f"(zv), "l"(pol) : "memory");
+                        }
+                }
+                if (gi == FN / 64 - 1) {   // accumulator 0 has been read: the next tile may start on it
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[0]));
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty));
+            if (lane == 0) {
+                if (f0 + (FN / 64 - 1) * 32 >= M) mbar_arrive(smem_u32(&ctl->acc_empty[0]));   // the loop ended before it got there
+                mbar_arrive(smem_u32(&ctl->acc_empty[1]));
+            }
         }
     }
 

@@ -259,7 +259,10 @@ log_softmax_rows_reg_kernel(float* __restrict__ Z, int ldz, int M, int C, const 
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
     int par = 0;   // the two halves of the scratch alternate, which saves a barrier per row
-    for (int row = blockIdx.x; row < M; row += gridDim.x, par ^= 1) {
+    // Rows are taken from the last one down: the kernel that wrote the logits just before this one
+    // produced the last frames last, and those are the rows the L2 cache still holds.
+    for (int r = blockIdx.x; r < M; r += gridDim.x, par ^= 1) {
+        const int row = M - 1 - r;
         float4* z = reinterpret_cast<float4*>(Z + (size_t)row * ldz);
         float4 v[V];
         float mx = -FLT_MAX;
