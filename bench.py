@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--splice", action="store_true",
                     help="feed one 40-dim frame per row and let the first layer form the context window "
                          "(11 or 15 frames) instead of reading an already spliced input")
+    ap.add_argument("--no-stack", action="store_true",
+                    help="one launch per binary hidden layer instead of one launch for the run of equal layers")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every step's kernels from the host instead of replaying a captured CUDA graph")
     ap.add_argument("--sweep", action="store_true",
@@ -343,6 +345,8 @@ def run_ours(args):
     B.bnn_set_xnor_path(B.XNOR_POPC if args.xnor_path == "popc" else B.XNOR_TENSOR)
     B.bnn_set_option(B.OPT_REAL_PATH, B.PATH_TENSOR if args.real_path == "tensor" else B.PATH_CUDA_CORE)
     B.bnn_set_option(B.OPT_XNOR_PREPARED, {"auto": 0, "stream": 1, "resident": 2}[args.xnor_prepared])
+    if args.no_stack:
+        B.bnn_set_option(B.OPT_XNOR_STACK, 0)
     dn = model.DeviceNet(net, device=dev, prepare_xnor=args.xnor_path == "tensor",
                          act_values=B.VALUES_01 if args.act_values == "01" else B.VALUES_PM1,
                          splice=((cfg.in_dim // 40) // 2, (cfg.in_dim // 40) // 2) if args.splice else (0, 0))
@@ -495,6 +499,24 @@ def run_ours(args):
     assert len(rows) == len(layer_ms)
     for r, t in zip(rows, layer_ms):
         r["ms"] = t
+    # A run of equal binary hidden layers is ONE launch (its events are recorded before the run):
+    # the run is reported as one row, time and work summed.
+    if not args.no_stack and frames > 16:
+        merged = []
+        for r in rows:
+            if (merged and r["kernel"] == "xnor_res_kernel" and merged[-1]["kernel"] == "xnor_res_kernel"
+                    and r["work"] == merged[-1]["work_per_layer"]):
+                m = merged[-1]
+                m["ms"] += r["ms"]; m["work"] += r["work"]; m["layers"] += 1
+                m["name"] = m["first_name"] + ".." + r["name"].split("_")[1]
+                if "smem_bytes" in m:
+                    m["smem_bytes"] += r["smem_bytes"]
+            else:
+                r = dict(r, work_per_layer=r["work"], first_name=r["name"], layers=1)
+                merged.append(r)
+        rows = merged
+    for r in rows:
+        t = r["ms"]
         r["achieved"] = r["work"] / (t * 1e-3) / r.get("scale", 1e12)
         r["frac"] = r["achieved"] / r["peak"]
         if "peak_nominal_ratio" in r:
@@ -565,11 +587,11 @@ def run_ours(args):
                 "overlap": "copy-in, forward and copy-out of consecutive steps on three streams"},
         # per step: the kernels named in the layer table (one per binary hidden layer, two per
         # sign-weight layer: split + GEMM, top-layer GEMM, log-softmax)
-        "gpu_launches": K * sum(r["kernel"].count("+") + 1 for r in rows),
+        "gpu_launches": K * (sum(r["kernel"].count("+") + 1 for r in rows)),
         "paths": {"xnor": args.xnor_path, "real": args.real_path},
         "roofline": roofline,
         "forward_roofline": forward_roofline,
-        "layers": [{k: r[k] for k in ("name", "kernel", "bound", "ms", "achieved", "peak", "unit", "frac", "frac_nominal_ratio", "pipe_util", "smem_pipe_util") if k in r}
+        "layers": [{k: r[k] for k in ("name", "kernel", "layers", "bound", "ms", "achieved", "peak", "unit", "frac", "frac_nominal_ratio", "pipe_util", "smem_pipe_util") if k in r}
                    for r in rows],
         "xnor_tbops": (xnor_work / (xnor_ms * 1e-3) / 1e12) if xnor_ms else None,
         "hbm": {"algorithmic_bytes_per_step": hbm, "achieved_gbs": hbm / (total_ms / K * 1e-3) / 1e9,

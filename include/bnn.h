@@ -380,9 +380,13 @@ BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, 
  *                        (Section 1) -- on kernels that spread each layer's weights over all SMs,
  *                        one warp per output unit, on the integer / FP32 pipes, instead of the
  *                        tiled tensor-core kernels (about 4x lower latency); 0 turns that off.
- *                        Integers and bits are identical; the fp32 sums differ by rounding order. */
+ *                        Integers and bits are identical; the fp32 sums differ by rounding order.
+ *   BNN_OPT_XNOR_STACK : 1 (default) lets bnn_forward run consecutive binary hidden layers of one
+ *                        shape with prepared weights (the loop over l of Algorithm 2's forward pass)
+ *                        as ONE launch, in which a layer's frame tiles start as soon as the layer
+ *                        before has stored them; 0 launches one kernel per layer.  Same bits. */
 typedef enum { BNN_OPT_XNOR_PATH = 0, BNN_OPT_REAL_PATH = 1, BNN_OPT_SIGNW_TERMS = 2,
-               BNN_OPT_XNOR_PREPARED = 3, BNN_OPT_SMALL_BATCH = 4 } bnn_option;
+               BNN_OPT_XNOR_PREPARED = 3, BNN_OPT_SMALL_BATCH = 4, BNN_OPT_XNOR_STACK = 5 } bnn_option;
 typedef enum { BNN_PATH_AUTO = 0, BNN_PATH_CUDA_CORE = 1, BNN_PATH_TENSOR = 2 } bnn_path;
 typedef enum { BNN_PREPARED_AUTO = 0, BNN_PREPARED_STREAM = 1, BNN_PREPARED_RESIDENT = 2 } bnn_prepared_kernel;
 BNN_API int bnn_set_option(int option, int value);

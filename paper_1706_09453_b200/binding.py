@@ -134,7 +134,7 @@ def packed_pitch(k: int) -> int:
     return int(lib().bnn_packed_pitch(int(k)))
 
 
-OPT_XNOR_PATH, OPT_REAL_PATH, OPT_SIGNW_TERMS, OPT_XNOR_PREPARED, OPT_SMALL_BATCH = 0, 1, 2, 3, 4
+OPT_XNOR_PATH, OPT_REAL_PATH, OPT_SIGNW_TERMS, OPT_XNOR_PREPARED, OPT_SMALL_BATCH, OPT_XNOR_STACK = 0, 1, 2, 3, 4, 5
 PREPARED_AUTO, PREPARED_STREAM, PREPARED_RESIDENT = 0, 1, 2
 PATH_AUTO, PATH_CUDA_CORE, PATH_TENSOR = 0, 1, 2
 XNOR_AUTO, XNOR_POPC, XNOR_TENSOR = PATH_AUTO, PATH_CUDA_CORE, PATH_TENSOR

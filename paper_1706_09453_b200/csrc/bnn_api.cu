@@ -13,6 +13,7 @@ int g_real_path = BNN_PATH_AUTO;
 int g_xnor_prepared = BNN_PREPARED_AUTO;
 int g_small_batch = 1;  // batches of up to kSmallBatchMax frames take the matrix-vector kernels
 int g_signw_terms = 2;  // |dot| <= K stays exact in every accumulator type used
+int g_xnor_stack = 1;   // runs of equal binary hidden layers go out as one launch
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -96,6 +97,17 @@ int validate_model(const bnn_model* model) {
     return BNN_OK;
 }
 
+// Whether hidden layer l can be part of a run launched as one kernel: a fused Sign layer on packed
+// input with prepared weights, of a shape the resident-weights kernel takes on its fast tiles.
+bool stackable(const bnn_model* model, int l) {
+    const bnn_layer& y = model->layers[l];
+    if (y.kind != BNN_LAYER_XNOR || y.act != BNN_ACT_SIGN_PACK || !y.W_prepared) return false;
+    if (g_xnor_path == BNN_PATH_CUDA_CORE || g_xnor_prepared == BNN_PREPARED_STREAM || y.K > kMaxKTensor) return false;
+    if (reinterpret_cast<uintptr_t>(y.W_prepared) & 255u) return false;
+    if (!xnor_res_applicable(y.N, y.K)) return false;
+    return y.K <= 2048 || g_xnor_prepared == BNN_PREPARED_RESIDENT;
+}
+
 }  // namespace
 
 extern "C" {
@@ -116,11 +128,12 @@ int bnn_set_option(int option, int value) {
         case BNN_OPT_SIGNW_TERMS: slot = &g_signw_terms; break;
         case BNN_OPT_XNOR_PREPARED: slot = &g_xnor_prepared; break;
         case BNN_OPT_SMALL_BATCH: slot = &g_small_batch; break;
+        case BNN_OPT_XNOR_STACK: slot = &g_xnor_stack; break;
         default: return -1;
     }
     if (option == BNN_OPT_SIGNW_TERMS) {
         if (value != 2 && value != 3) return -1;
-    } else if (option == BNN_OPT_SMALL_BATCH) {
+    } else if (option == BNN_OPT_SMALL_BATCH || option == BNN_OPT_XNOR_STACK) {
         if (value != 0 && value != 1) return -1;
     } else if (option == BNN_OPT_XNOR_PREPARED) {
         if (value != BNN_PREPARED_AUTO && value != BNN_PREPARED_STREAM && value != BNN_PREPARED_RESIDENT) return -1;
@@ -407,14 +420,27 @@ int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw,
                              log_softmax, 1, nullptr, 0, nullptr, BNN_ACT_NONE, nullptr, stream);
 }
 
-size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M) {
-    if (validate_model(model) != BNN_OK || M < 1) return 0;
+// Layout of the forward workspace: two activation buffers of `half` bytes each, then the arrival
+// counters of the stacked binary layers (`sync` bytes), then whatever the caller gave beyond that
+// (split-activation images).
+struct WorkspaceLayout {
+    size_t half, sync;
+    size_t need() const { return 2 * half + sync; }
+};
+static WorkspaceLayout workspace_layout(const bnn_model* model, int M) {
     size_t mx = 0;
+    int xnor_layers = 0;
     for (int l = 0; l + 1 < model->n_layers; ++l) {
         size_t b = layer_out_bytes(model->layers[l], M);
         if (b > mx) mx = b;
+        if (model->layers[l].kind == BNN_LAYER_XNOR) ++xnor_layers;
     }
-    return 2 * round256(mx) + 256;
+    return WorkspaceLayout{round256(mx), round256(xnor_stack_sync_bytes(M, xnor_layers))};
+}
+
+size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M) {
+    if (validate_model(model) != BNN_OK || M < 1) return 0;
+    return workspace_layout(model, M).need();
 }
 
 size_t bnn_forward_workspace_bytes(const bnn_model* model, int M) {
@@ -454,16 +480,21 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
     if (M < 1 || ldx < (ctx > 1 ? splice_dim : model->layers[0].K)) return BNN_ERR_SHAPE;
     const int L = model->n_layers;
     if (ldo < model->layers[L - 1].N) return BNN_ERR_SHAPE;
-    const size_t need = bnn_forward_min_workspace_bytes(model, M);
+    const WorkspaceLayout lay = workspace_layout(model, M);
+    const size_t need = lay.need();
     if (L > 1) {
         if (!workspace || workspace_bytes < need) return BNN_ERR_WORKSPACE;
         if (reinterpret_cast<uintptr_t>(workspace) & 255u) return BNN_ERR_ALIGN;
     }
-    char* buf[2] = {static_cast<char*>(workspace),
-                    static_cast<char*>(workspace) + (need - 256) / 2};
-    // whatever lies beyond the two activation buffers serves the sign-weight layers' image
-    char* img = static_cast<char*>(workspace) + (need - 256);
-    const size_t img_bytes = workspace_bytes > need - 256 ? workspace_bytes - (need - 256) : 0;
+    // everything that can be refused is checked before the first launch
+    for (int l = 0; l + 1 < L; ++l)
+        if (layer_out && layer_out[l] && model->layers[l].act == BNN_ACT_SIGN_PACK && !aligned16(layer_out[l]))
+            return BNN_ERR_ALIGN;
+    char* buf[2] = {static_cast<char*>(workspace), static_cast<char*>(workspace) + lay.half};
+    int* sync = reinterpret_cast<int*>(static_cast<char*>(workspace) + 2 * lay.half);
+    // whatever lies beyond the two activation buffers and the counters serves the split-activation images
+    char* img = static_cast<char*>(workspace) + need;
+    const size_t img_bytes = workspace_bytes > need ? workspace_bytes - need : 0;
     const void* in = X;
     int in_ld = ldx;
     bool in_bits = false;
@@ -471,6 +502,8 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
     // spread the weights over all SMs instead of tiling the frames (small_batch.cu).
     const bool small = g_small_batch && M <= kSmallBatchMax;
     const int zo01 = model->act_values == BNN_VALUES_01;
+    bool sync_cleared = false;
+    int sync_used = 0;   // counters handed to earlier runs of this call
     for (int l = 0; l < L; ++l) {
         const bnn_layer& y = model->layers[l];
         if (events && events[l] &&
@@ -501,8 +534,41 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                 return BNN_ERR_CUDA;
             return BNN_OK;
         }
+        // A run of binary hidden layers of one shape whose weights are prepared goes out as ONE launch
+        // of the kernel that keeps a unit tile's weights in shared memory (xnor_gemm_res.cu).
+        if (g_xnor_stack && !small && stackable(model, l)) {
+            int n = 1;
+            while (n < kXnorStackMax && l + n < L && stackable(model, l + n) && model->layers[l + n].N == y.N &&
+                   model->layers[l + n].K == y.K && y.N == y.K)
+                ++n;
+            if (n > 1) {
+                XnorStackLayer sl[kXnorStackMax];
+                for (int i = 0; i < n; ++i) {
+                    const bnn_layer& z = model->layers[l + i];
+                    void* o = (layer_out && layer_out[l + i]) ? layer_out[l + i] : buf[(l + i) & 1];
+                    sl[i] = XnorStackLayer{z.W_prepared, z.thr, z.flip, static_cast<uint32_t*>(o)};
+                    if (i > 0 && events && events[l + i] &&
+                        cudaEventRecord((cudaEvent_t)events[l + i], (cudaStream_t)stream) != cudaSuccess)
+                        return BNN_ERR_CUDA;
+                }
+                if (int rc = check_packed(in, in_ld, y.K)) return rc;
+                if (!sync_cleared) {
+                    if (cudaMemsetAsync(sync, 0, lay.sync, (cudaStream_t)stream) != cudaSuccess) return BNN_ERR_CUDA;
+                    sync_cleared = true;
+                }
+                const int ldob = bnn_packed_pitch(y.N);
+                if (int rc = launch_xnor_stack(static_cast<const uint32_t*>(in), in_ld, sl, n, M, y.N, y.K, ldob, zo01,
+                                               sync + sync_used, (cudaStream_t)stream))
+                    return rc;
+                sync_used += (int)(xnor_stack_sync_bytes(M, n) / sizeof(int));
+                in = sl[n - 1].out_bits;
+                in_ld = ldob;
+                in_bits = true;
+                l += n - 1;
+                continue;
+            }
+        }
         void* out = (layer_out && layer_out[l]) ? layer_out[l] : buf[l & 1];
-        if (y.act == BNN_ACT_SIGN_PACK && !aligned16(out)) return BNN_ERR_ALIGN;
         bnn_epilogue e{};
         e.act = y.act;
         e.sign_mode = model->sign_mode;

@@ -104,6 +104,20 @@ __host__ __device__ __forceinline__ int xnor_image_npad(int N) { return ceil_div
 bool xnor_res_applicable(int N, int K);
 int launch_xnor_res(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
                     const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int zo, cudaStream_t st);
+// A run of consecutive fused Sign layers of one shape (N == K beyond the first) in ONE launch of that
+// kernel: layer l reads the bits layer l - 1 wrote (pitch ldob), layer 0 reads Ap.  `progress` points
+// to xnor_stack_sync_bytes(M, n_layers) bytes of ZEROED device memory (per frame tile and layer
+// boundary a counter of the unit tiles that have stored their bits).
+constexpr int kXnorStackMax = 8;
+struct XnorStackLayer {
+    const void* image;
+    const int32_t* thr;
+    const uint32_t* flip;
+    uint32_t* out_bits;
+};
+size_t xnor_stack_sync_bytes(int M, int n_layers);
+int launch_xnor_stack(const uint32_t* Ap, int ldap, const XnorStackLayer* layers, int n_layers, int M, int N, int K,
+                      int ldob, int zo, int* progress, cudaStream_t st);
 int launch_xnor_prepare(const uint32_t* Wp, int ldwp, int N, int K, void* image, cudaStream_t st);
 int launch_xnor_img(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
                     int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,

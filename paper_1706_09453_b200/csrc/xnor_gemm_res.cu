@@ -28,6 +28,17 @@
 //                tensor memory, so it overlaps the next tile's MMAs
 // Every wait is bounded; a wait that runs out sets the CTA's abort flag, all roles fall
 // through to the common teardown and the device status word is set.
+//
+// A run of consecutive hidden layers of the same shape (the forward loop of Algorithm 2 over
+// l = 2 .. L-1) is ONE launch: the roles above loop over the layers.  Between layers nothing is
+// torn down; a CTA keeps its unit tile index and its frame tiles.  What a layer needs from the
+// one before it is tracked per frame tile: a counter in global memory that every CTA increments
+// (release) once its bits of that frame tile and layer are stored, and the thread that loads a
+// frame tile waits (acquire, bounded) until all unit tiles have arrived.  The weight slice of the
+// next layer replaces the current one stage by stage, each stage as soon as the last frame tile's
+// MMAs of that stage have completed, so the reload overlaps the tail of the layer.  (Measured on
+// B200: five launches of one layer each spent 6 us per layer between the end of one kernel and
+// the first MMA of the next.)
 #include "bnn_common.cuh"
 #include "tcgen05.cuh"
 #include "xnor_widen.cuh"
@@ -60,10 +71,12 @@ template <int BN> struct Cfg {
     static_assert(NKS <= MAX_NKS && A_STAGES >= 3 && TMEM_SF_COL + SF_COLS <= TMEM_COLS, "tile configuration");
 };
 
+constexpr int MAX_STACK = kXnorStackMax;
+
 struct Control {
     int T[192];              // per unit: threshold + kMagicBits
     uint32_t flipw[8];
-    uint64_t full_a[6], empty_a[6], full_b[MAX_NKS], acc_full[2], acc_empty[2];
+    uint64_t full_a[6], empty_a[6], full_b[MAX_NKS], b_free[MAX_NKS], acc_full[2], acc_empty[2];
     uint64_t group_full[GROUPS], group_empty[GROUPS];
     uint32_t tmem_base;
     int abort;
@@ -172,12 +185,46 @@ __device__ __forceinline__ void produce_a(const ProducerArgs& a, int r, int team
     }
 }
 
+// One layer of the run: its prepared weight image, folded thresholds and output.
+struct StackLayer {
+    const uint8_t* img;
+    const int32_t* thr;
+    const uint32_t* flip;
+    uint32_t* out_bits;
+};
+struct StackArgs {
+    StackLayer layer[MAX_STACK];
+    int n_layers;
+    int M, N, K, ldob, zo;
+    int* status;
+    int* progress;           // [n_layers - 1][frame tiles] arrival counters, zero at launch (unused for one layer)
+};
+struct StackMaps {
+    CUtensorMap m[MAX_STACK];   // packed input of each layer
+};
+
+// Wait until `*p` has reached `target` (acquire at GPU scope); bounded like the mbarrier waits.
+__device__ __forceinline__ bool wait_counter(const int* p, int target, volatile int* abort_flag) {
+    const long long t0 = clock64();
+#pragma unroll 1
+    while (true) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        if (v >= target) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            return false;
+        }
+        __nanosleep(64);
+    }
+}
+
 template <int BN>
 __global__ void __launch_bounds__(THREADS, 1)
-xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restrict__ img,
-                int M, int N, int K, const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
-                uint32_t* __restrict__ out_bits, int ldob, int zo, int* __restrict__ status) {
+xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ StackArgs g) {
     using C = Cfg<BN>;
+    const int M = g.M, N = g.N, K = g.K, ldob = g.ldob, zo = g.zo, L = g.n_layers;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(smem + B_REGION + GROUPS * GROUP_BYTES);
@@ -200,7 +247,10 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
             mbar_init(smem_u32(&ctl->full_a[s]), A_WARPS);
             mbar_init(smem_u32(&ctl->empty_a[s]), 1);
         }
-        for (int s = 0; s < MAX_NKS; ++s) mbar_init(smem_u32(&ctl->full_b[s]), 1);   // the copying thread (+ bytes)
+        for (int s = 0; s < MAX_NKS; ++s) {
+            mbar_init(smem_u32(&ctl->full_b[s]), 1);   // the copying thread (+ bytes)
+            mbar_init(smem_u32(&ctl->b_free[s]), 1);   // the MMA thread's commit
+        }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
@@ -228,58 +278,69 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
         for (int j = 0; j < 32; ++j) ones[j] = 0x7F7F7F7Fu;
         tmem_st32(tmem + ((uint32_t)(warp * 32) << 16) + C::TMEM_SF_COL, ones);
         tmem_st_wait();
-        // thresholds of this CTA's units: the unit tile never changes
-        const int t = warp * 32 + lane;
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int nl = t + h * 128, n = n0 + nl;
-            if (nl < BN) ctl->T[nl] = kMagicBits + (n < N ? thr[n] : 0);
-        }
-        if (t < BN / 32) {
-            const int wi = (n0 >> 5) + t;
-            ctl->flipw[t] = wi < words_for(N) ? flip[wi] : 0u;
-        }
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
 
     if (warp == TMA_WARP) {
-        // ---------------- one thread: the weight slice once, then the staging ring of frame rows
+        // ---------------- one thread: per layer the weight slice, then the staging ring of frame rows
         if (lane == 0 && share.count > 0) {
             const uint32_t stg = smem_u32(smem) + B_REGION;
             const int ng = ceil_div(nks, 2);
-            const int total_groups = share.count * ng;
-            int gc = 0;
-            auto load_group = [&](int g) {   // g: index in this CTA's sequence of groups, < GROUPS ahead of its consumers
-                const int slot = g % GROUPS;
-                const int m0 = (share.first + (g / ng) * share.step) * BM;
+            const size_t run = (size_t)xnor_image_npad(N) * 16;   // bytes between chunks of the image
+            int gc = 0;   // groups issued so far, over all layers: slot gc % GROUPS, < GROUPS ahead of its consumers
+            int gl = 0, gt = 0, gi = 0;   // the next group to issue: layer, index of the frame tile, group inside the tile
+            bool ok = true;
+            auto issue_group = [&]() {
+                const int mt = share.first + gt * share.step;
+                if (gi == 0 && gl > 0) {
+                    // the frame tile's bits of the layer before: every unit tile's CTA has stored them
+                    ok = wait_counter(g.progress + (size_t)(gl - 1) * m_tiles + mt, n_tiles, abort_flag);
+                    if (!ok) return;
+                    asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes of other CTAs -> this thread's TMA reads
+                }
+                const int slot = gc % GROUPS;
+                if (gc >= GROUPS) {
+                    ok = mbar_wait_relaxed(smem_u32(&ctl->group_empty[slot]), (uint32_t)(((gc / GROUPS) - 1) & 1), abort_flag);
+                    if (!ok) return;
+                }
                 const uint32_t bar = smem_u32(&ctl->group_full[slot]);
                 mbar_arrive_expect_tx(bar, GROUP_BYTES);
-                tma_load_2d(stg + slot * GROUP_BYTES, &mapA, (g % ng) * 16, m0, bar);
+                tma_load_2d(stg + slot * GROUP_BYTES, &maps.m[gl], gi * 16, mt * BM, bar);
+                ++gc;
+                if (++gi == ng) { gi = 0; if (++gt == share.count) { gt = 0; ++gl; } }
             };
-            // the weights first: they do not depend on the kernel before this one in the stream
-            const uint8_t* src = img + (size_t)n0 * 16;
-            const size_t run = (size_t)xnor_image_npad(N) * 16;   // bytes between chunks of the image
-            for (int ks = 0; ks < nks; ++ks) {
-                const uint32_t bar = smem_u32(&ctl->full_b[ks]);
-                mbar_arrive_expect_tx(bar, C::B_BYTES);
+            for (int l = 0; l < L && ok; ++l) {
+                // A later layer's first frame rows go into the staging ring before its weights: the
+                // producers widen them into tensor memory while the weight stages arrive.
+                if (l > 0)
+                    for (int i = 0; i < GROUPS && gl == l && ok; ++i) issue_group();
+                if (!ok) break;
+                // The weights do not depend on the kernel before this one in the stream (layer 0) nor on
+                // other CTAs (later layers).  A stage of the previous layer's slice is overwritten once
+                // the MMAs of this CTA's last frame tile that read it have completed.
+                const uint8_t* src = g.layer[l].img + (size_t)n0 * 16;
+                for (int ks = 0; ks < nks && ok; ++ks) {
+                    if (l > 0) ok = mbar_wait(smem_u32(&ctl->b_free[ks]), (uint32_t)((l - 1) & 1), abort_flag);
+                    if (!ok) break;
+                    const uint32_t bar = smem_u32(&ctl->full_b[ks]);
+                    mbar_arrive_expect_tx(bar, C::B_BYTES);
 #pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    bulk_g2s(smem_u32(smem + ks * C::B_BYTES + c * (BN * 16)), src + (size_t)(ks * 8 + c) * run, BN * 16, bar);
-            }
-            // the frames are the previous kernel's output: wait until that kernel has completed
-            // and its writes are visible (returns at once when there is no such dependency)
-            pdl_wait();
-            for (; gc < GROUPS && gc < total_groups; ++gc) load_group(gc);
-            for (; gc < total_groups; ++gc) {
-                if (!mbar_wait_relaxed(smem_u32(&ctl->group_empty[gc % GROUPS]), (uint32_t)(((gc / GROUPS) - 1) & 1), abort_flag)) break;
-                load_group(gc);
+                    for (int c = 0; c < 8; ++c)
+                        bulk_g2s(smem_u32(smem + ks * C::B_BYTES + c * (BN * 16)), src + (size_t)(ks * 8 + c) * run, BN * 16, bar);
+                }
+                if (!ok) break;
+                // the frames of layer 0 are the previous kernel's output: wait until that kernel has
+                // completed and its writes are visible (returns at once when there is no such dependency)
+                if (l == 0) pdl_wait();
+                while (gl == l && ok) issue_group();
             }
         }
         __syncwarp();
     } else if (warp >= PROD_WARP0) {
-        ProducerArgs pa{smem_u32(smem) + B_REGION, tmem + C::TMEM_A_COL, ctl, abort_flag, share.count, nks, kw, tail_mask(K), lane, zo};
+        // the layers follow one another in the producers' sequence of (tile, stage) pairs
+        ProducerArgs pa{smem_u32(smem) + B_REGION, tmem + C::TMEM_A_COL, ctl, abort_flag, L * share.count, nks, kw, tail_mask(K), lane, zo};
         produce_a<C::A_STAGES>(pa, (warp & 3) * 32 + lane, (warp - PROD_WARP0) / A_WARPS);
     } else if (warp == MMA_WARP) {
         // ---------------- MMA issue: one thread
@@ -298,51 +359,59 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
             int sa = 0;          // slot of the A ring and the parity its `full` barrier shows next
             uint32_t pa = 0;
             bool ok = true;
-            for (int tl = 0; tl < share.count && ok; ++tl) {
-                const int b = tl & 1;
-                ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), (uint32_t)(((tl >> 1) & 1) ^ 1), abort_flag);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t d = tmem + (uint32_t)(b * BN);
-                uint64_t db = desc0;
-                int ks = 0;
-                for (; ks + 1 < nks; ks += 2) {
-                    const int sa2 = sa + 1 == C::A_STAGES ? 0 : sa + 1;
-                    const uint32_t pa2 = sa + 1 == C::A_STAGES ? pa ^ 1u : pa;
-                    // a weight stage arrives once (phase 0) and then stays
-                    ok = (tl > 0 || (mbar_wait(smem_u32(&ctl->full_b[ks]), 0u, abort_flag) &&
-                                     mbar_wait(smem_u32(&ctl->full_b[ks + 1]), 0u, abort_flag))) &&
-                         mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag) &&
-                         mbar_wait(smem_u32(&ctl->full_a[sa2]), pa2, abort_flag);
+            int tl = 0;          // tiles so far, over all layers
+            for (int l = 0; l < L && ok; ++l) {
+                const uint32_t pb = (uint32_t)(l & 1);   // a layer's weight stages arrive once and then stay
+                for (int t = 0; t < share.count && ok; ++t, ++tl) {
+                    const bool first = t == 0;
+                    const bool hand_over = t == share.count - 1 && l + 1 < L;   // the next layer's slice follows
+                    const int b = tl & 1;
+                    ok = mbar_wait(smem_u32(&ctl->acc_empty[b]), (uint32_t)(((tl >> 1) & 1) ^ 1), abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t ta = tmem_a + sa * A_COLS, ta2 = tmem_a + sa2 * A_COLS;
-#pragma unroll
-                    for (int j = 0; j < BK / 64; ++j)   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
-                        mma_mxf4_ts(d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
-                    mma_commit(smem_u32(&ctl->empty_a[sa]));
-#pragma unroll
-                    for (int j = 0; j < BK / 64; ++j)
-                        mma_mxf4_ts(d, ta2 + 8 * j, db + kStepS + j * kStepJ, idesc, sfa, sfb, 1u);
-                    mma_commit(smem_u32(&ctl->empty_a[sa2]));
-                    db += 2 * kStepS;
-                    sa = sa2; pa = pa2;
-                    if (++sa == C::A_STAGES) { sa = 0; pa ^= 1u; }
-                }
-                if (ok && ks < nks) {   // odd number of stages: the last one alone
-                    ok = (tl > 0 || mbar_wait(smem_u32(&ctl->full_b[ks]), 0u, abort_flag)) &&
-                         mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag);
-                    if (ok) {
+                    const uint32_t d = tmem + (uint32_t)(b * BN);
+                    uint64_t db = desc0;
+                    int ks = 0;
+                    for (; ks + 1 < nks; ks += 2) {
+                        const int sa2 = sa + 1 == C::A_STAGES ? 0 : sa + 1;
+                        const uint32_t pa2 = sa + 1 == C::A_STAGES ? pa ^ 1u : pa;
+                        ok = (!first || (mbar_wait(smem_u32(&ctl->full_b[ks]), pb, abort_flag) &&
+                                         mbar_wait(smem_u32(&ctl->full_b[ks + 1]), pb, abort_flag))) &&
+                             mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag) &&
+                             mbar_wait(smem_u32(&ctl->full_a[sa2]), pa2, abort_flag);
+                        if (!ok) break;
                         tc_fence_after_sync();
-                        const uint32_t ta = tmem_a + sa * A_COLS;
+                        const uint32_t ta = tmem_a + sa * A_COLS, ta2 = tmem_a + sa2 * A_COLS;
 #pragma unroll
-                        for (int j = 0; j < BK / 64; ++j)
+                        for (int j = 0; j < BK / 64; ++j)   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
                             mma_mxf4_ts(d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
                         mma_commit(smem_u32(&ctl->empty_a[sa]));
+                        if (hand_over) mma_commit(smem_u32(&ctl->b_free[ks]));
+#pragma unroll
+                        for (int j = 0; j < BK / 64; ++j)
+                            mma_mxf4_ts(d, ta2 + 8 * j, db + kStepS + j * kStepJ, idesc, sfa, sfb, 1u);
+                        mma_commit(smem_u32(&ctl->empty_a[sa2]));
+                        if (hand_over) mma_commit(smem_u32(&ctl->b_free[ks + 1]));
+                        db += 2 * kStepS;
+                        sa = sa2; pa = pa2;
                         if (++sa == C::A_STAGES) { sa = 0; pa ^= 1u; }
                     }
+                    if (ok && ks < nks) {   // odd number of stages: the last one alone
+                        ok = (!first || mbar_wait(smem_u32(&ctl->full_b[ks]), pb, abort_flag)) &&
+                             mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag);
+                        if (ok) {
+                            tc_fence_after_sync();
+                            const uint32_t ta = tmem_a + sa * A_COLS;
+#pragma unroll
+                            for (int j = 0; j < BK / 64; ++j)
+                                mma_mxf4_ts(d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
+                            mma_commit(smem_u32(&ctl->empty_a[sa]));
+                            if (hand_over) mma_commit(smem_u32(&ctl->b_free[ks]));
+                            if (++sa == C::A_STAGES) { sa = 0; pa ^= 1u; }
+                        }
+                    }
+                    if (ok) mma_commit(smem_u32(&ctl->acc_full[b]));
                 }
-                if (ok) mma_commit(smem_u32(&ctl->acc_full[b]));
             }
         }
         __syncwarp();
@@ -351,47 +420,78 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
         const int row_in_tile = warp * 32 + lane;
         const float magic = __int_as_float(kMagicBits);
         bool ok = true;
-        for (int tl = 0; tl < share.count && ok; ++tl) {
-            const int m0 = (share.first + tl * share.step) * BM;
-            const int m = m0 + row_in_tile;
-            const int b = tl & 1;
-            // all four epilogue warps take the same decision, so none is left at a barrier
-            ok = epi_all(warp_wait_relaxed(smem_u32(&ctl->acc_full[b]), (uint32_t)((tl >> 1) & 1), abort_flag, lane));
-            if (!ok) break;
-            tc_fence_after_sync();
-            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * BN);
-            uint32_t words[BN / 32];
+        int tl = 0;              // tiles so far, over all layers
+        for (int l = 0; l < L && ok; ++l) {
+            // thresholds of this CTA's units for this layer (the unit tile never changes); the
+            // barriers keep them apart from the previous layer's last readers
+            const int32_t* __restrict__ thr = g.layer[l].thr;
+            const uint32_t* __restrict__ flip = g.layer[l].flip;
+            uint32_t* __restrict__ out_bits = g.layer[l].out_bits;
+            if (l > 0) epi_bar_sync();
 #pragma unroll
-            for (int g = 0; g < BN / 32; ++g) {
-                uint32_t acc[32];
-                tmem_ld32(taddr + g * 32, acc);
-                tmem_ld_wait();
-                // The accumulator holds the integer dot product as a float; adding 1.5 * 2^23
-                // leaves that integer, offset by kMagicBits, in the bit pattern of the sum.
-                // bit = (dot - thr >= 0); the sign bits are shifted in from the top, element 31
-                // first, so element j ends up in bit j, inverted.
-                uint32_t wd = 0u;
-#pragma unroll
-                for (int j = 31; j >= 0; --j)
-                    wd = __funnelshift_l((uint32_t)(__float_as_int(__uint_as_float(acc[j]) + magic) - ctl->T[g * 32 + j]), wd, 1);
-                words[g] = ~wd ^ ctl->flipw[g];
-                const int valid = N - (n0 + g * 32);  // columns of this word that exist
-                if (valid < 32) words[g] = valid > 0 ? (words[g] & ((1u << valid) - 1u)) : 0u;
+            for (int h = 0; h < 2; ++h) {
+                const int nl = row_in_tile + h * 128, n = n0 + nl;
+                if (nl < BN) ctl->T[nl] = kMagicBits + (n < N ? thr[n] : 0);
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
-            if (m < M) {
+            if (row_in_tile < BN / 32) {
+                const int wi = (n0 >> 5) + row_in_tile;
+                ctl->flipw[row_in_tile] = wi < words_for(N) ? flip[wi] : 0u;
+            }
+            epi_bar_sync();
+            for (int t = 0; t < share.count && ok; ++t, ++tl) {
+                const int mt = share.first + t * share.step;
+                const int m = mt * BM + row_in_tile;
+                const int b = tl & 1;
+                // all four epilogue warps take the same decision, so none is left at a barrier
+                ok = epi_all(warp_wait_relaxed(smem_u32(&ctl->acc_full[b]), (uint32_t)((tl >> 1) & 1), abort_flag, lane));
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * BN);
                 const int nw = words_for(N), w0 = n0 >> 5;
-                uint32_t* dst = out_bits + (size_t)m * ldob + w0;
-                if (w0 + BN / 32 <= nw) {   // rows are 16-byte aligned and BN/32 is even: 8-byte stores
+                uint32_t* dst = out_bits + (size_t)(m < M ? m : 0) * ldob + w0;
+                const bool whole = w0 + BN / 32 <= nw;   // rows are 16-byte aligned and BN/32 is even: 8-byte stores
 #pragma unroll
-                    for (int i = 0; i < BN / 64; ++i)
-                        reinterpret_cast<uint2*>(dst)[i] = make_uint2(words[2 * i], words[2 * i + 1]);
-                } else {
+                for (int gp = 0; gp < BN / 64; ++gp) {
+                    uint32_t pair[2];
 #pragma unroll
-                    for (int g = 0; g < BN / 32; ++g)
-                        if (w0 + g < nw) dst[g] = words[g];
+                    for (int h = 0; h < 2; ++h) {
+                        const int gq = 2 * gp + h;
+                        uint32_t acc[32];
+                        tmem_ld32(taddr + gq * 32, acc);
+                        tmem_ld_wait();
+                        // The accumulator holds the integer dot product as a float; adding 1.5 * 2^23
+                        // leaves that integer, offset by kMagicBits, in the bit pattern of the sum.
+                        // bit = (dot - thr >= 0); the sign bits are shifted in from the top, element 31
+                        // first, so element j ends up in bit j, inverted.
+                        uint32_t wd = 0u;
+#pragma unroll
+                        for (int j = 31; j >= 0; --j)
+                            wd = __funnelshift_l((uint32_t)(__float_as_int(__uint_as_float(acc[j]) + magic) - ctl->T[gq * 32 + j]), wd, 1);
+                        wd = ~wd ^ ctl->flipw[gq];
+                        const int valid = N - (n0 + gq * 32);  // columns of this word that exist
+                        if (valid < 32) wd = valid > 0 ? (wd & ((1u << valid) - 1u)) : 0u;
+                        pair[h] = wd;
+                    }
+                    if (m < M) {
+                        if (whole) {
+                            reinterpret_cast<uint2*>(dst)[gp] = make_uint2(pair[0], pair[1]);
+                        } else {
+                            if (w0 + 2 * gp < nw) dst[2 * gp] = pair[0];
+                            if (w0 + 2 * gp + 1 < nw) dst[2 * gp + 1] = pair[1];
+                        }
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[b]));
+                if (l + 1 < L) {
+                    // this CTA's share of frame tile mt is stored: tell the CTAs that read it in the next layer
+                    __threadfence();
+                    epi_bar_sync();
+                    if (threadIdx.x == 0) {
+                        asm volatile("fence.proxy.async;" ::: "memory");
+                        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(g.progress + (size_t)l * m_tiles + mt) : "memory");
+                    }
                 }
             }
         }
@@ -404,12 +504,12 @@ xnor_res_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (threadIdx.x == 0 && ctl->abort) atomicExch(status, 1);
+    if (threadIdx.x == 0 && ctl->abort) atomicExch(g.status, 1);
 }
 
 template <int BN>
-int launch_bn(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
-              const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int zo, int sm_count, cudaStream_t st) {
+int launch_bn(const uint32_t* Ap, int ldap, const XnorStackLayer* layers, int n_layers, int M, int N, int K, int ldob,
+              int zo, int* progress, int sm_count, cudaStream_t st) {
     auto kern = xnor_res_kernel<BN>;
     static bool configured = false;
     if (!configured) {
@@ -418,12 +518,19 @@ int launch_bn(const uint32_t* Ap, int ldap, const void* image, int M, int N, int
     }
     const long long tiles = (long long)ceil_div(M, BM) * ceil_div(N, BN);
     const int grid = tiles < sm_count ? (int)tiles : sm_count;
-    int* status = tc_status_ptr();
-    if (!status) return BNN_ERR_CUDA;
-    CUtensorMap mapA;
-    if (!encode_packed_map(&mapA, Ap, ldap, M, K, BM)) return BNN_ERR_CUDA;
-    if (launch_pdl(kern, dim3(grid), dim3(THREADS), SMEM_BYTES, st, mapA, static_cast<const uint8_t*>(image), M, N, K,
-                   thr, flip, out_bits, ldob, zo, status) != cudaSuccess)
+    StackArgs a{};
+    StackMaps maps{};
+    a.n_layers = n_layers; a.M = M; a.N = N; a.K = K; a.ldob = ldob; a.zo = zo;
+    a.status = tc_status_ptr();
+    a.progress = progress;
+    if (!a.status) return BNN_ERR_CUDA;
+    for (int l = 0; l < n_layers; ++l) {
+        a.layer[l] = StackLayer{static_cast<const uint8_t*>(layers[l].image), layers[l].thr, layers[l].flip, layers[l].out_bits};
+        // a layer reads what the layer before it wrote
+        const uint32_t* in = l == 0 ? Ap : layers[l - 1].out_bits;
+        if (!encode_packed_map(&maps.m[l], in, l == 0 ? ldap : ldob, M, K, BM)) return BNN_ERR_CUDA;
+    }
+    if (launch_pdl(kern, dim3(grid), dim3(THREADS), SMEM_BYTES, st, maps, a) != cudaSuccess)
         return BNN_ERR_CUDA;
     return launch_status();
 }
@@ -455,14 +562,25 @@ bool xnor_res_applicable(int N, int K) {
     return sms > 0 && tile_units(N, K, sms) != 0;
 }
 
-int launch_xnor_res(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
-                    const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
+size_t xnor_stack_sync_bytes(int M, int n_layers) {
+    return n_layers > 1 ? (size_t)(n_layers - 1) * ceil_div(M, BM) * sizeof(int) : 0;
+}
+
+int launch_xnor_stack(const uint32_t* Ap, int ldap, const XnorStackLayer* layers, int n_layers, int M, int N, int K,
+                      int ldob, int zo, int* progress, cudaStream_t st) {
     const int sms = sm_count_of_device();
     if (sms <= 0) return BNN_ERR_CUDA;
+    if (n_layers < 1 || n_layers > kXnorStackMax || (n_layers > 1 && (N != K || !progress))) return BNN_ERR_UNSUPPORTED;
     const int bn = tile_units(N, K, sms);
-    if (bn == 192) return launch_bn<192>(Ap, ldap, image, M, N, K, thr, flip, out_bits, ldob, zo, sms, st);
-    if (bn == 128) return launch_bn<128>(Ap, ldap, image, M, N, K, thr, flip, out_bits, ldob, zo, sms, st);
+    if (bn == 192) return launch_bn<192>(Ap, ldap, layers, n_layers, M, N, K, ldob, zo, progress, sms, st);
+    if (bn == 128) return launch_bn<128>(Ap, ldap, layers, n_layers, M, N, K, ldob, zo, progress, sms, st);
     return BNN_ERR_UNSUPPORTED;
+}
+
+int launch_xnor_res(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
+                    const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
+    const XnorStackLayer one{image, thr, flip, out_bits};
+    return launch_xnor_stack(Ap, ldap, &one, 1, M, N, K, ldob, zo, nullptr, st);
 }
 
 }  // namespace bnn
