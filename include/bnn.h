@@ -3,8 +3,10 @@
  * with binary (+-1) weights and activations (Lu, arXiv 1706.09453).
  *
  * Every step of the forward pass runs in this library's own CUDA kernels; there is no CPU
- * path.  The library never allocates, frees or synchronises: the caller owns every buffer
- * and work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ * path.  The library never allocates or frees, and only bnn_device_status synchronises: the
+ * caller owns every buffer and work is enqueued on `stream` (a cudaStream_t passed as void*;
+ * NULL = default stream).  A process may drive several devices; each call works on the device
+ * that is current when it is made.
  *
  * Unless an argument is marked HOST, every pointer is a DEVICE pointer.
  *
@@ -44,7 +46,8 @@ typedef enum {
     BNN_ERR_ALIGN = 3,       /* base pointer or pitch breaks the alignment rules above */
     BNN_ERR_UNSUPPORTED = 4, /* a combination of options this library does not implement */
     BNN_ERR_WORKSPACE = 5,   /* workspace missing or too small */
-    BNN_ERR_CUDA = 6         /* the CUDA runtime reported an error at launch */
+    BNN_ERR_CUDA = 6,        /* the CUDA runtime reported an error at launch */
+    BNN_ERR_TIMEOUT = 7      /* a bounded wait inside a kernel ran out: see bnn_device_status */
 } bnn_status;
 
 /* Value of Sign at zero.  Eq. 3 of the paper gives +1 for x > 0 and -1 for everything else, i.e.
@@ -337,11 +340,14 @@ BNN_API int bnn_forward(const bnn_model* model, const float* X, int ldx, int M,
  * counterpart.
  *   - Inputs and outputs (model, X, logp) are still the caller's.
  *   - Limit: bnn_forward_min_workspace_bytes(model, M) must not exceed the array; otherwise the
- *     call launches nothing and returns BNN_ERR_WORKSPACE.  (8 MiB holds 16384 frames of a
- *     2048-wide binary-activation network, or 512 frames with fp32 hardtanh activations.)
+ *     call launches nothing and returns BNN_ERR_WORKSPACE.  (For a 2048-wide network 8 MiB holds
+ *     16376 frames of binary activations -- the activation buffers plus the counters of the stacked
+ *     binary layers -- or 512 frames of fp32 hardtanh activations.)
  *   - This call makes no cudaMalloc/cudaFree and uses no allocating library routine.
  *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call outside of any stream capture.
+ *     current), and the CUDA runtime may load this library's device code -- the array with it --
+ *     only then; make that first call at start-up, outside of any stream capture.  From then on a
+ *     call leaves the device's free memory exactly as it found it.
  *   - All calls share the one array, which keeps whatever the last call left in it (nothing
  *     needs clearing: each layer only reads what the previous layer wrote in the same call).
  *     Two calls whose kernels can overlap on the GPU -- different streams, or several host
@@ -384,18 +390,35 @@ BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, 
  *   BNN_OPT_XNOR_STACK : 1 (default) lets bnn_forward run consecutive binary hidden layers of one
  *                        shape with prepared weights (the loop over l of Algorithm 2's forward pass)
  *                        as ONE launch, in which a layer's frame tiles start as soon as the layer
- *                        before has stored them; 0 launches one kernel per layer.  Same bits. */
+ *                        before has stored them; 0 launches one kernel per layer.  Same bits.
+ *   BNN_OPT_WAIT_LIMIT_US: how long a kernel may wait on one of its internal barriers or counters before
+ *                        it gives up (see bnn_device_status), in microseconds at a nominal 2 GHz SM
+ *                        clock; default 1 000 000, minimum 1.  Applies to launches made after the call. */
 typedef enum { BNN_OPT_XNOR_PATH = 0, BNN_OPT_REAL_PATH = 1, BNN_OPT_SIGNW_TERMS = 2,
-               BNN_OPT_XNOR_PREPARED = 3, BNN_OPT_SMALL_BATCH = 4, BNN_OPT_XNOR_STACK = 5 } bnn_option;
+               BNN_OPT_XNOR_PREPARED = 3, BNN_OPT_SMALL_BATCH = 4, BNN_OPT_XNOR_STACK = 5,
+               BNN_OPT_WAIT_LIMIT_US = 6 } bnn_option;
 typedef enum { BNN_PATH_AUTO = 0, BNN_PATH_CUDA_CORE = 1, BNN_PATH_TENSOR = 2 } bnn_path;
 typedef enum { BNN_PREPARED_AUTO = 0, BNN_PREPARED_STREAM = 1, BNN_PREPARED_RESIDENT = 2 } bnn_prepared_kernel;
 BNN_API int bnn_set_option(int option, int value);
 
-/* Tensor-core kernels bound every wait they perform; a CTA whose wait runs out stops, frees
- * its tensor memory and sets a status word.  This call SYNCHRONISES the device and stores
- * that word in *status (HOST pointer): 0 = no kernel gave up, 1 = one did (results of the
- * affected launch are invalid).  The paper has no counterpart. */
+/* Give-up path (the paper has no counterpart).  The tensor-core kernels bound every wait they
+ * perform -- on a pipeline barrier, on another CTA's progress counter -- by BNN_OPT_WAIT_LIMIT_US.
+ * A CTA whose wait runs out stops, frees its tensor memory, returns normally and sets a status
+ * word on its device: 0 = no kernel gave up, 1 = one did (the results of that launch are
+ * invalid; the context stays usable).
+ *   bnn_device_status : SYNCHRONISES the current device, stores the word in *status (HOST
+ *                       pointer) and returns BNN_ERR_TIMEOUT when it is set, BNN_OK otherwise.
+ *   bnn_query_status  : the same read in stream order and without a synchronisation: enqueues
+ *                       a 4-byte copy of the word into `dst` (DEVICE or pinned HOST memory) on
+ *                       `stream`; the caller reads it once the stream has got there.
+ *   bnn_reset_status  : enqueues the reset of the word to 0 on `stream`.
+ *   bnn_wait_probe    : enqueues a one-warp launch that waits on a barrier on which nothing
+ *                       arrives, so that its wait runs out after the limit and the word is set:
+ *                       lets a caller (or a test) exercise the path above without a fault. */
 BNN_API int bnn_device_status(int* status);
+BNN_API int bnn_query_status(int* dst, void* stream);
+BNN_API int bnn_reset_status(void* stream);
+BNN_API int bnn_wait_probe(void* stream);
 
 /* Micro-benchmarks of the pipes that bound the kernels above (measurement support; the paper
  * has no counterpart: its Section 3 reports accuracy only).  bnn_pipe_rate enqueues ONE launch

@@ -86,6 +86,12 @@ def lib():
         L.bnn_pipe_rate.restype = C.c_int
         L.bnn_device_status.argtypes = [C.POINTER(C.c_int)]
         L.bnn_device_status.restype = C.c_int
+        L.bnn_query_status.argtypes = [C.c_void_p, C.c_void_p]
+        L.bnn_query_status.restype = C.c_int
+        L.bnn_reset_status.argtypes = [C.c_void_p]
+        L.bnn_reset_status.restype = C.c_int
+        L.bnn_wait_probe.argtypes = [C.c_void_p]
+        L.bnn_wait_probe.restype = C.c_int
         L.bnn_forward_workspace_bytes.restype = C.c_size_t
         L.bnn_forward_workspace_bytes.argtypes = [C.POINTER(Model), C.c_int]
         L.bnn_forward_min_workspace_bytes.restype = C.c_size_t
@@ -134,7 +140,8 @@ def packed_pitch(k: int) -> int:
     return int(lib().bnn_packed_pitch(int(k)))
 
 
-OPT_XNOR_PATH, OPT_REAL_PATH, OPT_SIGNW_TERMS, OPT_XNOR_PREPARED, OPT_SMALL_BATCH, OPT_XNOR_STACK = 0, 1, 2, 3, 4, 5
+OPT_XNOR_PATH, OPT_REAL_PATH, OPT_SIGNW_TERMS, OPT_XNOR_PREPARED, OPT_SMALL_BATCH, OPT_XNOR_STACK, OPT_WAIT_LIMIT_US = 0, 1, 2, 3, 4, 5, 6
+ERR_TIMEOUT = 7
 PREPARED_AUTO, PREPARED_STREAM, PREPARED_RESIDENT = 0, 1, 2
 PATH_AUTO, PATH_CUDA_CORE, PATH_TENSOR = 0, 1, 2
 XNOR_AUTO, XNOR_POPC, XNOR_TENSOR = PATH_AUTO, PATH_CUDA_CORE, PATH_TENSOR
@@ -170,8 +177,24 @@ def bnn_pipe_rate(which: int, repeat: int, scratch) -> float:
 def bnn_device_status() -> int:
     """Synchronises the device; 0 unless a tensor-core kernel gave up on a bounded wait."""
     st = C.c_int(-1)
-    _check(lib().bnn_device_status(C.byref(st)), "bnn_device_status")
+    rc = lib().bnn_device_status(C.byref(st))
+    if rc not in (0, ERR_TIMEOUT):
+        _check(rc, "bnn_device_status")
     return st.value
+
+
+def bnn_query_status(dst):
+    """Enqueues a copy of the status word into ``dst`` (int32 CUDA or pinned tensor) on the current stream."""
+    _check(lib().bnn_query_status(C.c_void_p(dst.data_ptr()), _stream()), "bnn_query_status")
+
+
+def bnn_reset_status():
+    _check(lib().bnn_reset_status(_stream()), "bnn_reset_status")
+
+
+def bnn_wait_probe():
+    """Enqueues the launch whose wait runs out (sets the status word after the wait limit)."""
+    _check(lib().bnn_wait_probe(_stream()), "bnn_wait_probe")
 
 
 def _ptr(t, dtype=None):

@@ -129,6 +129,12 @@ int bnn_set_option(int option, int value) {
         case BNN_OPT_XNOR_PREPARED: slot = &g_xnor_prepared; break;
         case BNN_OPT_SMALL_BATCH: slot = &g_small_batch; break;
         case BNN_OPT_XNOR_STACK: slot = &g_xnor_stack; break;
+        case BNN_OPT_WAIT_LIMIT_US: {
+            // microseconds -> SM clocks at a nominal 2 GHz
+            if (value < 1) return -1;
+            const long long prev = set_wait_limit_clocks((long long)value * 2000);
+            return (int)(prev / 2000 > 0x7FFFFFFF ? 0x7FFFFFFF : prev / 2000);
+        }
         default: return -1;
     }
     if (option == BNN_OPT_SIGNW_TERMS) {
@@ -147,8 +153,18 @@ int bnn_set_option(int option, int value) {
 
 int bnn_device_status(int* status) {
     if (!status) return BNN_ERR_NULL;
-    return read_tc_status(status);
+    if (int rc = read_tc_status(status)) return rc;
+    return *status ? BNN_ERR_TIMEOUT : BNN_OK;
 }
+
+int bnn_query_status(int* dst, void* stream) {
+    if (!dst) return BNN_ERR_NULL;
+    return copy_tc_status_async(dst, (cudaStream_t)stream);
+}
+
+int bnn_reset_status(void* stream) { return reset_tc_status_async((cudaStream_t)stream); }
+
+int bnn_wait_probe(void* stream) { return launch_wait_probe((cudaStream_t)stream); }
 
 const char* bnn_status_string(int status) {
     switch (status) {
@@ -159,6 +175,7 @@ const char* bnn_status_string(int status) {
         case BNN_ERR_UNSUPPORTED: return "unsupported combination of options";
         case BNN_ERR_WORKSPACE: return "workspace missing or too small";
         case BNN_ERR_CUDA: return "CUDA runtime error at launch";
+        case BNN_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out (device status word set)";
         default: return "unknown status";
     }
 }
@@ -558,7 +575,7 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                 }
                 const int ldob = bnn_packed_pitch(y.N);
                 if (int rc = launch_xnor_stack(static_cast<const uint32_t*>(in), in_ld, sl, n, M, y.N, y.K, ldob, zo01,
-                                               sync + sync_used, (cudaStream_t)stream))
+                                               sync + sync_used, true, (cudaStream_t)stream))
                     return rc;
                 sync_used += (int)(xnor_stack_sync_bytes(M, n) / sizeof(int));
                 in = sl[n - 1].out_bits;

@@ -107,7 +107,8 @@ int launch_xnor_res(const uint32_t* Ap, int ldap, const void* image, int M, int 
 // A run of consecutive fused Sign layers of one shape (N == K beyond the first) in ONE launch of that
 // kernel: layer l reads the bits layer l - 1 wrote (pitch ldob), layer 0 reads Ap.  `progress` points
 // to xnor_stack_sync_bytes(M, n_layers) bytes of ZEROED device memory (per frame tile and layer
-// boundary a counter of the unit tiles that have stored their bits).
+// boundary a counter of the unit tiles that have stored their bits).  `chained`: the launch is part of a
+// forward pass (programmatic dependent launch on the layer kernel before it).
 constexpr int kXnorStackMax = 8;
 struct XnorStackLayer {
     const void* image;
@@ -117,7 +118,7 @@ struct XnorStackLayer {
 };
 size_t xnor_stack_sync_bytes(int M, int n_layers);
 int launch_xnor_stack(const uint32_t* Ap, int ldap, const XnorStackLayer* layers, int n_layers, int M, int N, int K,
-                      int ldob, int zo, int* progress, cudaStream_t st);
+                      int ldob, int zo, int* progress, bool chained, cudaStream_t st);
 int launch_xnor_prepare(const uint32_t* Wp, int ldwp, int N, int K, void* image, cudaStream_t st);
 int launch_xnor_img(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
                     int32_t* C, int ldc, const int32_t* thr, const uint32_t* flip,
@@ -125,11 +126,13 @@ int launch_xnor_img(const uint32_t* Ap, int ldap, const void* image, int M, int 
 // Small batches (small_batch.cu): plain kernels that spread a layer's weights over all SMs, one
 // warp per output unit, for M <= kSmallBatchMax frames.
 constexpr int kSmallBatchMax = 16;
-// Whether a layer of fan-in K fits those kernels (they stage the batch's operand in 48 KB of
-// shared memory: 16 x K floats for real input, 16 x K bits for packed input).
-inline bool small_fits_real(int K) { return (size_t)kSmallBatchMax * K * sizeof(float) <= 48 * 1024; }
-inline bool small_fits_bits(int K) { return (size_t)kSmallBatchMax * words_for(K) * sizeof(uint32_t) <= 48 * 1024; }
-inline bool small_fits_out(int H) { return (size_t)words_for(H) * 32 * sizeof(uint16_t) <= 48 * 1024; }
+// Whether a layer of fan-in K fits those kernels: they stage the batch's operand in dynamic shared
+// memory (16 x K floats for real input, 16 x K bits for packed input) next to up to 1 KB of static
+// arrays, and the two together must stay within the 48 KB a kernel gets without opting in.
+constexpr size_t kSmallSmemMax = 47 * 1024;
+inline bool small_fits_real(int K) { return (size_t)kSmallBatchMax * K * sizeof(float) <= kSmallSmemMax; }
+inline bool small_fits_bits(int K) { return (size_t)kSmallBatchMax * words_for(K) * sizeof(uint32_t) <= kSmallSmemMax; }
+inline bool small_fits_out(int H) { return (size_t)words_for(H) * 32 * sizeof(uint16_t) <= kSmallSmemMax; }
 int launch_small_signw(const float* X, int ldx, const uint32_t* Wp, int ldwp, int M, int N, int K,
                        const float* scale, const float* shift, int sign_mode,
                        uint32_t* out_bits, int ldob, cudaStream_t st);
@@ -146,8 +149,17 @@ int launch_pipe_rate(int which, int repeat, void* scratch, size_t scratch_bytes,
 bool encode_packed_map(CUtensorMap* map, const uint32_t* base, int ld, int rows, int K, int box_rows);
 // Reads (synchronously) the word that a tensor-core kernel sets when a bounded wait ran out.
 int read_tc_status(int* out);
-// Device address of that word, passed to every tensor-core kernel (nullptr on failure).
-int* tc_status_ptr();
+// The same as a copy enqueued on `st` (dst: device or pinned host memory), and the reset of the word.
+int copy_tc_status_async(int* dst, cudaStream_t st);
+int reset_tc_status_async(cudaStream_t st);
+// Limit of every bounded wait in SM clocks; returns the previous value.
+long long set_wait_limit_clocks(long long clocks);
+// A one-warp launch whose wait runs out (see tc_support.cu).
+int launch_wait_probe(cudaStream_t st);
+// Per-device bookkeeping of the launchers: SM count of the current device (0 on failure), and
+// cudaFuncAttributeMaxDynamicSharedMemorySize raised once per device and kernel.
+int device_sm_count();
+bool ensure_dynamic_smem(const void* kernel, int bytes);
 
 // Real-valued GEMM on the FP32 pipe: D[m][n] = sum_k A[m][k]*B[n][k], where each operand is
 // either fp32 or packed +-1 bits.

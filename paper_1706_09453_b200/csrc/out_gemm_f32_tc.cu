@@ -50,7 +50,7 @@ constexpr uint32_t TMEM_COLS = 512;
 struct Control {
     uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
-    int abort;
+    WaitState wait;
 };
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + (int)sizeof(Control) + 128;
 static_assert(SMEM_BYTES <= 232448, "shared memory of one CTA");
@@ -98,11 +98,11 @@ h_split_kernel(const float* __restrict__ Hf, int ldh, int M, int H, int nks, uin
 __global__ void __launch_bounds__(THREADS, 1)
 outf_tc_kernel(const uint8_t* __restrict__ himg, const uint8_t* __restrict__ wimg,
                const float* __restrict__ rs, const float* __restrict__ bias,
-               int M, int C, int H, float* __restrict__ Z, int ldz, int act, int* __restrict__ status) {
+               int M, int C, int H, float* __restrict__ Z, int ldz, int act, TcStatus status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES);
-    volatile int* abort_flag = &ctl->abort;
+    volatile int* abort_flag = &ctl->wait.abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nks = ceil_div(H, BK);
@@ -118,7 +118,7 @@ outf_tc_kernel(const uint8_t* __restrict__ himg, const uint8_t* __restrict__ wim
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
         }
-        ctl->abort = 0;
+        wait_state_init(&ctl->wait, status);
         mbar_init_fence();
     }
     if (warp == MMA_WARP) {
@@ -233,7 +233,7 @@ outf_tc_kernel(const uint8_t* __restrict__ himg, const uint8_t* __restrict__ wim
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (threadIdx.x == 0 && ctl->abort) atomicExch(status, 1);
+    if (threadIdx.x == 0 && ctl->wait.abort) atomicExch(status.word, 1);
 }
 
 }  // namespace
@@ -244,23 +244,15 @@ size_t outf_image_bytes(int M, int H) {
 
 int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float* bias,
                    int M, int C, int H, float* Z, int ldz, int act, void* workspace, cudaStream_t st) {
-    static bool configured = false;
-    static int sms = 0;
-    if (!configured) {
-        int dev = 0;
-        if (cudaFuncSetAttribute(outf_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-            cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return BNN_ERR_CUDA;
-        configured = true;
-    }
+    const int sms = device_sm_count();
+    if (sms <= 0 || !ensure_dynamic_smem(reinterpret_cast<const void*>(outf_tc_kernel), SMEM_BYTES)) return BNN_ERR_CUDA;
     const int ct = ceil_div(C, BC), hs = ceil_div(H, BK), ft = ceil_div(M, FN);
     // the prepared weight image: ct * hs blocks of both terms, then the per-class factors 2^-e
     const uint8_t* wimg = static_cast<const uint8_t*>(prepared);
     const float* rs = reinterpret_cast<const float*>(wimg + (size_t)ct * hs * A_BYTES);
     uint8_t* himg = static_cast<uint8_t*>(workspace);
-    int* status = tc_status_ptr();
-    if (!status) return BNN_ERR_CUDA;
+    const TcStatus status = tc_status();
+    if (!status.word) return BNN_ERR_CUDA;
     h_split_kernel<<<ft * hs, FN, 0, st>>>(Hf, ldhf, M, H, hs, himg);
     const int tiles = ct * ft;
     outf_tc_kernel<<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(himg, wimg, rs, bias, M, C, H, Z, ldz, act, status);

@@ -40,7 +40,7 @@ constexpr uint32_t TMEM_COLS = 512;
 struct Control {
     uint64_t full[STAGES], empty[STAGES], acc_full, acc_empty[2];
     uint32_t tmem_base;
-    int abort;
+    WaitState wait;
 };
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + (int)sizeof(Control) + 128;
 
@@ -110,11 +110,11 @@ template <bool ZO>
 __global__ void __launch_bounds__(THREADS, 1)
 out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restrict__ img,
               const float* __restrict__ rs, const float* __restrict__ bias,
-              int M, int C, int H, float* __restrict__ Z, int ldz, int* __restrict__ status) {
+              int M, int C, int H, float* __restrict__ Z, int ldz, TcStatus status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     Control* ctl = reinterpret_cast<Control*>(smem + STAGES * STAGE_BYTES);
-    volatile int* abort_flag = &ctl->abort;
+    volatile int* abort_flag = &ctl->wait.abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nks = ceil_div(H, BK);
@@ -129,7 +129,7 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
         mbar_init(smem_u32(&ctl->acc_full), 1);
         mbar_init(smem_u32(&ctl->acc_empty[0]), EPI_WARPS);
         mbar_init(smem_u32(&ctl->acc_empty[1]), EPI_WARPS);
-        ctl->abort = 0;
+        wait_state_init(&ctl->wait, status);
         mbar_init_fence();
     }
     if (warp == MMA_WARP) {
@@ -317,7 +317,7 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (threadIdx.x == 0 && ctl->abort) atomicExch(status, 1);
+    if (threadIdx.x == 0 && ctl->wait.abort) atomicExch(status.word, 1);
 }
 
 }  // namespace
@@ -339,23 +339,16 @@ int launch_out_prepare(const float* W, int ldw, int C, int H, void* prepared, cu
 
 int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const float* bias,
                   int M, int C, int H, float* Z, int ldz, int zo, cudaStream_t st) {
-    static bool configured = false;
-    static int sms = 0;
-    if (!configured) {
-        int dev = 0;
-        if (cudaFuncSetAttribute(out_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-            cudaFuncSetAttribute(out_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-            cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return BNN_ERR_CUDA;
-        configured = true;
-    }
+    const int sms = device_sm_count();
+    if (sms <= 0 || !ensure_dynamic_smem(reinterpret_cast<const void*>(out_tc_kernel<false>), SMEM_BYTES) ||
+        !ensure_dynamic_smem(reinterpret_cast<const void*>(out_tc_kernel<true>), SMEM_BYTES))
+        return BNN_ERR_CUDA;
     const int ct = ceil_div(C, BC), hs = ceil_div(H, BK);
     const uint8_t* img = static_cast<const uint8_t*>(prepared);
     const float* rs = reinterpret_cast<const float*>(img + (size_t)ct * hs * A_BYTES);
     const int tiles = ct * ceil_div(M, FN);
-    int* status = tc_status_ptr();
-    if (!status) return BNN_ERR_CUDA;
+    const TcStatus status = tc_status();
+    if (!status.word) return BNN_ERR_CUDA;
     if (zo)
         out_tc_kernel<true><<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(Hp, ldhp, img, rs, bias, M, C, H, Z, ldz, status);
     else

@@ -65,17 +65,17 @@ l2_read_kernel(const uint4* __restrict__ src, size_t vecs, int trips, uint32_t* 
 constexpr int MMA_SMEM = 128 * 32 + 256 * 32 + 1024;   // one K step of A and of B, K-major 16-byte chunks
 template <bool MXF4, bool A_TMEM, int N>
 __global__ void __launch_bounds__(128, 1)
-mma_rate_kernel(int n_mma, int* __restrict__ status) {
+mma_rate_kernel(int n_mma, TcStatus status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     __shared__ uint64_t bar;
     __shared__ uint32_t tmem_slot;
-    __shared__ int abort_word;
+    __shared__ WaitState wait;
     const int warp = threadIdx.x >> 5;
     for (int i = threadIdx.x; i < (128 * 32 + 256 * 32) / 4; i += 128) reinterpret_cast<uint32_t*>(smem)[i] = 0x22222222u;
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bar), 1);
-        abort_word = 0;
+        wait_state_init(&wait, status);
         mbar_init_fence();
     }
     fence_proxy_async_smem();
@@ -114,10 +114,10 @@ mma_rate_kernel(int n_mma, int* __restrict__ status) {
                 else mma_f16(d, da, db, idesc, 1u);
             }
             mma_commit(smem_u32(&bar));
-            ok = mbar_wait(smem_u32(&bar), phase, &abort_word);
+            ok = mbar_wait(smem_u32(&bar), phase, &wait.abort);
             phase ^= 1u;
         }
-        if (!ok) atomicExch(status, 1);
+        if (!ok) atomicExch(status.word, 1);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -137,8 +137,8 @@ int launch_alu(int repeat, uint32_t* sink, int sms, double* work, cudaStream_t s
 
 template <bool MXF4, bool A_TMEM, int N>
 int launch_mma(int repeat, int sms, double* work, cudaStream_t st) {
-    int* status = tc_status_ptr();
-    if (!status) return BNN_ERR_CUDA;
+    const TcStatus status = tc_status();
+    if (!status.word) return BNN_ERR_CUDA;
     const int n_mma = repeat * 64;
     mma_rate_kernel<MXF4, A_TMEM, N><<<sms, 128, MMA_SMEM, st>>>(n_mma, status);
     *work = (double)sms * n_mma * 2.0 * 128.0 * N * (MXF4 ? 64.0 : 16.0);

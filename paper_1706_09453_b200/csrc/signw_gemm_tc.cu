@@ -39,7 +39,7 @@ struct Control {
     float sc[BN], sh[BN];
     uint64_t full[8], empty[8], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
-    int abort;
+    WaitState wait;
 };
 
 
@@ -58,7 +58,7 @@ struct Args {
     int act, sign_mode;
     float* Y; int ldy;
     uint32_t* out_bits; int ldob;
-    int* status;
+    TcStatus status;
 };
 
 template <int NT>
@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(THREADS, 1) signw_tc_kernel(Args g) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     Control* ctl = reinterpret_cast<Control*>(smem + C::STAGES * C::STAGE_BYTES);
-    volatile int* abort_flag = &ctl->abort;
+    volatile int* abort_flag = &ctl->wait.abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int M = g.M, N = g.N, K = g.K;
@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(THREADS, 1) signw_tc_kernel(Args g) {
             mbar_init(smem_u32(&ctl->acc_full[b]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
         }
-        ctl->abort = 0;
+        wait_state_init(&ctl->wait, g.status);
         mbar_init_fence();
     }
     if (warp == MMA_WARP) {
@@ -292,23 +292,15 @@ __global__ void __launch_bounds__(THREADS, 1) signw_tc_kernel(Args g) {
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (threadIdx.x == 0 && ctl->abort) atomicExch(g.status, 1);
+    if (threadIdx.x == 0 && ctl->wait.abort) atomicExch(g.status.word, 1);
 }
 
 template <int NT>
 int launch_nt(const Args& a, cudaStream_t st) {
     using C = Cfg<NT>;
     constexpr int SMEM = C::STAGES * C::STAGE_BYTES + (int)sizeof(Control) + 128;
-    static bool configured = false;
-    static int sms = 0;
-    if (!configured) {
-        int dev = 0;
-        if (cudaFuncSetAttribute(signw_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess ||
-            cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return BNN_ERR_CUDA;
-        configured = true;
-    }
+    const int sms = device_sm_count();
+    if (sms <= 0 || !ensure_dynamic_smem(reinterpret_cast<const void*>(signw_tc_kernel<NT>), SMEM)) return BNN_ERR_CUDA;
     const int tiles = ceil_div(a.M, BM) * ceil_div(a.N, BN);
     signw_tc_kernel<NT><<<tiles < sms ? tiles : sms, THREADS, SMEM, st>>>(a);
     return launch_status();
@@ -318,8 +310,8 @@ int launch_nt(const Args& a, cudaStream_t st) {
 
 int launch_signw_tc(const RealGemmArgs& r, int terms, cudaStream_t st) {
     Args a{r.Af, r.lda, r.Bb, r.ldb, r.M, r.N, r.K, r.scale, r.shift, r.act, r.sign_mode,
-           r.Y, r.ldy, r.out_bits, r.ldob, tc_status_ptr()};
-    if (!a.status) return BNN_ERR_CUDA;
+           r.Y, r.ldy, r.out_bits, r.ldob, tc_status()};
+    if (!a.status.word) return BNN_ERR_CUDA;
     return terms == 3 ? launch_nt<3>(a, st) : launch_nt<2>(a, st);
 }
 

@@ -46,7 +46,7 @@ struct Control {
     float sc[UN], sh[UN];
     uint64_t full[4], empty[4], acc_full, acc_empty[2];
     uint32_t tmem_base;
-    int abort;
+    WaitState wait;
 };
 
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
@@ -269,7 +269,7 @@ struct Args {
     int act, sign_mode;
     float* Y; int ldy;
     uint32_t* out_bits; int ldob;
-    int* status;
+    TcStatus status;
 };
 
 template <int NT>
@@ -278,7 +278,7 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     Control* ctl = reinterpret_cast<Control*>(smem + C::STAGES * C::STAGE_BYTES);
-    volatile int* abort_flag = &ctl->abort;
+    volatile int* abort_flag = &ctl->wait.abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int M = g.M, N = g.N;
@@ -294,7 +294,7 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
         mbar_init(smem_u32(&ctl->acc_full), 1);
         mbar_init(smem_u32(&ctl->acc_empty[0]), EPI_WARPS);
         mbar_init(smem_u32(&ctl->acc_empty[1]), EPI_WARPS);
-        ctl->abort = 0;
+        wait_state_init(&ctl->wait, g.status);
         mbar_init_fence();
     }
     if (warp == MMA_WARP) {
@@ -488,29 +488,21 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (threadIdx.x == 0 && ctl->abort) atomicExch(g.status, 1);
+    if (threadIdx.x == 0 && ctl->wait.abort) atomicExch(g.status.word, 1);
 }
 
 template <int NT>
 int launch_nt(const RealGemmArgs& r, void* workspace, cudaStream_t st) {
     using C = Cfg<NT>;
     constexpr int SMEM = C::STAGES * C::STAGE_BYTES + (int)sizeof(Control) + 128;
-    static bool configured = false;
-    static int sms = 0;
-    if (!configured) {
-        int dev = 0;
-        if (cudaFuncSetAttribute(signw_img_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess ||
-            cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return BNN_ERR_CUDA;
-        configured = true;
-    }
+    const int sms = device_sm_count();
+    if (sms <= 0 || !ensure_dynamic_smem(reinterpret_cast<const void*>(signw_img_kernel<NT>), SMEM)) return BNN_ERR_CUDA;
     const int nks = ceil_div(r.K, BK), mt = ceil_div(r.M, BM);
     uint8_t* img = static_cast<uint8_t*>(workspace);
     x_split_kernel<NT><<<mt * nks, 256, 0, st>>>(r.Af, r.lda, r.M, r.K, nks, img, r.splice_dim, r.splice_left);
     Args a{img, r.Bb, r.ldb, r.M, r.N, r.K, r.scale, r.shift, r.act, r.sign_mode, r.Y, r.ldy, r.out_bits, r.ldob,
-           tc_status_ptr()};
-    if (!a.status) return BNN_ERR_CUDA;
+           tc_status()};
+    if (!a.status.word) return BNN_ERR_CUDA;
     const int tiles = mt * ceil_div(r.N, UN);
     if (launch_pdl(signw_img_kernel<NT>, dim3(tiles < sms ? tiles : sms), dim3(THREADS), SMEM, st, a) != cudaSuccess)
         return BNN_ERR_CUDA;

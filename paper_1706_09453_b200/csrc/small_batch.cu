@@ -21,7 +21,6 @@ namespace bnn {
 namespace {
 
 constexpr int MAXM = kSmallBatchMax;   // frames per launch
-constexpr size_t kSmallSmemMax = 48 * 1024;   // the batch's operand is staged in (default-size) shared memory
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -35,21 +35,40 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Every wait is bounded: after kWaitCycles SM clocks (about a second) the waiter raises the
-// CTA-wide abort flag and returns false; all roles then leave their loops, the CTA frees
-// its tensor memory and exits, and the host finds the error in the status word.
-constexpr long long kWaitCycles = 2000000000LL;
+// Every wait is bounded: after `limit` SM clocks (about a second unless the host asked for
+// another limit) the waiter raises the CTA-wide abort flag and returns false; all roles then
+// leave their loops, the CTA frees its tensor memory and exits, and the host finds the error in
+// the status word.  The flag and the limit sit side by side in shared memory; the waits are
+// handed the address of the flag.
+struct WaitState {
+    int abort;
+    int reserved;
+    long long limit;         // SM clocks a wait may take
+};
+__device__ __forceinline__ long long wait_limit_of(volatile int* abort_flag) {
+    return reinterpret_cast<volatile WaitState*>(abort_flag)->limit;
+}
+// What the host hands every tensor-core kernel: the device status word and the wait limit.
+struct TcStatus {
+    int* word;
+    long long limit;
+};
+__device__ __forceinline__ void wait_state_init(WaitState* w, const TcStatus& st) {
+    w->abort = 0;
+    w->reserved = 0;
+    w->limit = st.limit;
+}
 
 // One immediate poll, then polls spaced by the abort and clock checks.  (Measured on B200 on
 // a 4-stage pipeline: this form runs the XNOR layer in 0.052 ms; starting with the clock
 // read, or with a burst of several immediate polls, takes 0.081 ms.)
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = wait_limit_of(abort_flag);
 #pragma unroll 1
     while (!mbar_try_wait(bar, parity)) {
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
@@ -63,7 +82,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // few hundred nanoseconds late, which these roles can afford.
 __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = wait_limit_of(abort_flag);
 #pragma unroll 1
     while (true) {
         uint32_t ok;
@@ -74,7 +93,7 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
             : "=r"(ok) : "r"(bar), "r"(parity), "r"(2000u) : "memory");
         if (ok) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
@@ -252,4 +271,8 @@ __device__ __forceinline__ void tmem_ld_wait() {
 }
 
 }  // namespace tc
+
+// Status word of the current device and the wait limit in force (word == nullptr on failure).
+tc::TcStatus tc_status();
+
 }  // namespace bnn

@@ -67,7 +67,7 @@ struct Control {
     uint64_t full_a[A_STAGES], empty_a[A_STAGES], full_b[B_STAGES], empty_b[B_STAGES], acc_full[2], acc_empty[2];
     uint64_t group_full[GROUPS], group_empty[GROUPS];
     uint32_t tmem_base;
-    int abort;
+    WaitState wait;
 };
 template <bool STORE_C> constexpr int smem_bytes() {
     return B_STAGES * B_BYTES + GROUPS * GROUP_BYTES + (int)sizeof(Control) + Cfg<STORE_C>::CSTAGE_BYTES + 1024;
@@ -185,12 +185,12 @@ __global__ void __launch_bounds__(THREADS, 1)
 xnor_img_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restrict__ img,
                 int M, int N, int K, int32_t* __restrict__ C, int ldc,
                 const int32_t* __restrict__ thr, const uint32_t* __restrict__ flip,
-                uint32_t* __restrict__ out_bits, int ldob, int zo, int* __restrict__ status) {
+                uint32_t* __restrict__ out_bits, int ldob, int zo, TcStatus status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(smem + B_STAGES * B_BYTES + GROUPS * GROUP_BYTES);
     int (*cstage)[2][32][36] = reinterpret_cast<int (*)[2][32][36]>(reinterpret_cast<uint8_t*>(ctl) + sizeof(Control));
-    volatile int* abort_flag = &ctl->abort;
+    volatile int* abort_flag = &ctl->wait.abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kw = words_for(K);
@@ -215,7 +215,7 @@ xnor_img_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
             mbar_init(smem_u32(&ctl->group_full[b]), 1);         // the issuing thread (+ bytes)
             mbar_init(smem_u32(&ctl->group_empty[b]), A_WARPS);  // every producer warp has read it
         }
-        ctl->abort = 0;
+        wait_state_init(&ctl->wait, status);
         mbar_init_fence();
     }
     if (warp == MMA_WARP) {
@@ -431,7 +431,7 @@ xnor_img_kernel(const __grid_constant__ CUtensorMap mapA, const uint8_t* __restr
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (threadIdx.x == 0 && ctl->abort) atomicExch(status, 1);
+    if (threadIdx.x == 0 && ctl->wait.abort) atomicExch(status.word, 1);
 }
 
 template <bool STORE_C, bool SIGN_PACK>
@@ -440,20 +440,12 @@ int launch_variant(const uint32_t* Ap, int ldap, const void* image, int M, int N
                    uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
     auto kern = xnor_img_kernel<STORE_C, SIGN_PACK>;
     constexpr int SMEM = smem_bytes<STORE_C>();
-    static bool configured = false;
-    static int sm_count = 0;
-    if (!configured) {
-        int dev = 0;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess ||
-            cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return BNN_ERR_CUDA;
-        configured = true;
-    }
+    const int sm_count = device_sm_count();
+    if (sm_count <= 0 || !ensure_dynamic_smem(reinterpret_cast<const void*>(kern), SMEM)) return BNN_ERR_CUDA;
     const int tiles = ceil_div(M, BM) * ceil_div(N, BN);
     const int grid = tiles < sm_count ? tiles : sm_count;
-    int* status = tc_status_ptr();
-    if (!status) return BNN_ERR_CUDA;
+    const TcStatus status = tc_status();
+    if (!status.word) return BNN_ERR_CUDA;
     CUtensorMap mapA;
     if (!encode_packed_map(&mapA, Ap, ldap, M, K, BM)) return BNN_ERR_CUDA;
     kern<<<grid, THREADS, SMEM, st>>>(mapA, static_cast<const uint8_t*>(image), M, N, K, C, ldc, thr, flip,

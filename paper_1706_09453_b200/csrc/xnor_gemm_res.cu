@@ -79,7 +79,7 @@ struct Control {
     uint64_t full_a[6], empty_a[6], full_b[MAX_NKS], b_free[MAX_NKS], acc_full[2], acc_empty[2];
     uint64_t group_full[GROUPS], group_empty[GROUPS];
     uint32_t tmem_base;
-    int abort;
+    WaitState wait;
 };
 constexpr int SMEM_BYTES = B_REGION + GROUPS * GROUP_BYTES + (int)sizeof(Control) + 1024;
 static_assert(SMEM_BYTES <= 232448, "shared memory of one CTA");
@@ -196,7 +196,7 @@ struct StackArgs {
     StackLayer layer[MAX_STACK];
     int n_layers;
     int M, N, K, ldob, zo;
-    int* status;
+    TcStatus status;
     int* progress;           // [n_layers - 1][frame tiles] arrival counters, zero at launch (unused for one layer)
 };
 struct StackMaps {
@@ -205,14 +205,14 @@ struct StackMaps {
 
 // Wait until `*p` has reached `target` (acquire at GPU scope); bounded like the mbarrier waits.
 __device__ __forceinline__ bool wait_counter(const int* p, int target, volatile int* abort_flag) {
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = wait_limit_of(abort_flag);
 #pragma unroll 1
     while (true) {
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
         if (v >= target) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
@@ -228,7 +228,7 @@ xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Control* ctl = reinterpret_cast<Control*>(smem + B_REGION + GROUPS * GROUP_BYTES);
-    volatile int* abort_flag = &ctl->abort;
+    volatile int* abort_flag = &ctl->wait.abort;
 
     // The kernel that follows in the stream may be scheduled as soon as this one's CTAs leave
     // their SMs.  This kernel's own set-up and the copy of its weight slice need nothing the
@@ -259,7 +259,7 @@ xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ 
             mbar_init(smem_u32(&ctl->group_full[b]), 1);              // the issuing thread (+ bytes)
             mbar_init(smem_u32(&ctl->group_empty[b]), 2 * A_WARPS);   // per stage of the group, every warp of its team
         }
-        ctl->abort = 0;
+        wait_state_init(&ctl->wait, g.status);
         mbar_init_fence();
     }
     if (warp == MMA_WARP) {
@@ -504,34 +504,37 @@ xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ 
         tc_fence_after_sync();
         tmem_dealloc(tmem, TMEM_COLS);
     }
-    if (threadIdx.x == 0 && ctl->abort) atomicExch(g.status, 1);
+    if (threadIdx.x == 0 && ctl->wait.abort) atomicExch(g.status.word, 1);
 }
 
 template <int BN>
 int launch_bn(const uint32_t* Ap, int ldap, const XnorStackLayer* layers, int n_layers, int M, int N, int K, int ldob,
-              int zo, int* progress, int sm_count, cudaStream_t st) {
+              int zo, int* progress, bool chained, int sm_count, cudaStream_t st) {
     auto kern = xnor_res_kernel<BN>;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return BNN_ERR_CUDA;
-        configured = true;
-    }
+    if (!ensure_dynamic_smem(reinterpret_cast<const void*>(kern), SMEM_BYTES)) return BNN_ERR_CUDA;
     const long long tiles = (long long)ceil_div(M, BM) * ceil_div(N, BN);
     const int grid = tiles < sm_count ? (int)tiles : sm_count;
     StackArgs a{};
     StackMaps maps{};
     a.n_layers = n_layers; a.M = M; a.N = N; a.K = K; a.ldob = ldob; a.zo = zo;
-    a.status = tc_status_ptr();
+    a.status = tc_status();
     a.progress = progress;
-    if (!a.status) return BNN_ERR_CUDA;
+    if (!a.status.word) return BNN_ERR_CUDA;
     for (int l = 0; l < n_layers; ++l) {
         a.layer[l] = StackLayer{static_cast<const uint8_t*>(layers[l].image), layers[l].thr, layers[l].flip, layers[l].out_bits};
         // a layer reads what the layer before it wrote
         const uint32_t* in = l == 0 ? Ap : layers[l - 1].out_bits;
         if (!encode_packed_map(&maps.m[l], in, l == 0 ? ldap : ldob, M, K, BM)) return BNN_ERR_CUDA;
     }
-    if (launch_pdl(kern, dim3(grid), dim3(THREADS), SMEM_BYTES, st, maps, a) != cudaSuccess)
-        return BNN_ERR_CUDA;
+    // Programmatic dependent launch only inside a forward pass: there the kernel before this one is a
+    // layer's kernel and everything read before the wait (weights, thresholds) was complete before the
+    // forward pass started.  A stand-alone call may follow the kernel that wrote its thresholds or its
+    // weight image on the same stream, so it is launched the ordinary way.
+    if (chained) {
+        if (launch_pdl(kern, dim3(grid), dim3(THREADS), SMEM_BYTES, st, maps, a) != cudaSuccess) return BNN_ERR_CUDA;
+    } else {
+        kern<<<grid, THREADS, SMEM_BYTES, st>>>(maps, a);
+    }
     return launch_status();
 }
 
@@ -546,16 +549,7 @@ static int tile_units(int N, int K, int sm_count) {
     return bn;
 }
 
-static int sm_count_of_device() {
-    static int sm_count = 0;
-    if (!sm_count) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            sm_count = 0;
-    }
-    return sm_count;
-}
+static int sm_count_of_device() { return device_sm_count(); }
 
 bool xnor_res_applicable(int N, int K) {
     const int sms = sm_count_of_device();
@@ -567,20 +561,20 @@ size_t xnor_stack_sync_bytes(int M, int n_layers) {
 }
 
 int launch_xnor_stack(const uint32_t* Ap, int ldap, const XnorStackLayer* layers, int n_layers, int M, int N, int K,
-                      int ldob, int zo, int* progress, cudaStream_t st) {
+                      int ldob, int zo, int* progress, bool chained, cudaStream_t st) {
     const int sms = sm_count_of_device();
     if (sms <= 0) return BNN_ERR_CUDA;
     if (n_layers < 1 || n_layers > kXnorStackMax || (n_layers > 1 && (N != K || !progress))) return BNN_ERR_UNSUPPORTED;
     const int bn = tile_units(N, K, sms);
-    if (bn == 192) return launch_bn<192>(Ap, ldap, layers, n_layers, M, N, K, ldob, zo, progress, sms, st);
-    if (bn == 128) return launch_bn<128>(Ap, ldap, layers, n_layers, M, N, K, ldob, zo, progress, sms, st);
+    if (bn == 192) return launch_bn<192>(Ap, ldap, layers, n_layers, M, N, K, ldob, zo, progress, chained, sms, st);
+    if (bn == 128) return launch_bn<128>(Ap, ldap, layers, n_layers, M, N, K, ldob, zo, progress, chained, sms, st);
     return BNN_ERR_UNSUPPORTED;
 }
 
 int launch_xnor_res(const uint32_t* Ap, int ldap, const void* image, int M, int N, int K,
                     const int32_t* thr, const uint32_t* flip, uint32_t* out_bits, int ldob, int zo, cudaStream_t st) {
     const XnorStackLayer one{image, thr, flip, out_bits};
-    return launch_xnor_stack(Ap, ldap, &one, 1, M, N, K, ldob, zo, nullptr, st);
+    return launch_xnor_stack(Ap, ldap, &one, 1, M, N, K, ldob, zo, nullptr, false, st);
 }
 
 }  // namespace bnn

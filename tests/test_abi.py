@@ -36,7 +36,7 @@ def test_every_declared_symbol_is_exported(lib):
 def test_status_strings_and_pitch(lib):
     from paper_1706_09453_b200 import binding as B
     assert B.status_string(0) == "ok"
-    assert len({B.status_string(i) for i in range(7)}) == 7
+    assert len({B.status_string(i) for i in range(8)}) == 8
     assert [B.packed_pitch(k) for k in (1, 32, 33, 128, 129, 440, 2048)] == [4, 4, 4, 4, 8, 16, 64]
 
 

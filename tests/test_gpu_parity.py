@@ -173,6 +173,44 @@ def test_xnor_gemm_int32_bit_exact(B, torch_, xnor_path, shape, p):
     np.testing.assert_array_equal(got[:, n:], -77)
 
 
+@pytest.mark.parametrize("shape", [(96, 40, 8192), (65536, 24, 1024)])
+def test_xnor_gemm_int32_longest_fan_in_and_largest_batch(B, torch_, xnor_path, shape):
+    """The corner sizes of the GEMM sweep (fan-in 8192; 65536 frames) with few units, so that the
+    oracle checks every output: all three kernels, every element."""
+    m, n, k = shape
+    ap = wl.make_bit_planes(m, k, 0.5, [5, m, n, k], B.packed_pitch(k))
+    wp = wl.make_bit_planes(n, k, 0.1, [6, m, n, k], B.packed_pitch(k))
+    c = torch_.full((m, n), -77, dtype=torch_.int32, device="cuda:0")
+    run_xnor(B, xnor_path, dev(ap), dev(wp), k, C_out=c)
+    np.testing.assert_array_equal(c.cpu().numpy(), o.xnor_gemm(ap, wp, k))
+    assert B.bnn_device_status() == 0
+
+
+def test_xnor_prepared_right_after_its_setup_on_one_stream(B, torch_):
+    """Thresholds folded, weights prepared and the fused layer launched back to back on one stream,
+    several times over with changing parameters: the layer must see each set-up's results (plain
+    stream order is all the header promises)."""
+    m, n, k = 1000, 384, 2048
+    rng = np.random.default_rng(5)
+    ap = wl.make_bit_planes(m, k, 0.5, [7, m, n, k], B.packed_pitch(k))
+    a_dev = dev(ap)
+    thr = torch_.zeros(n, dtype=torch_.int32, device="cuda:0")
+    flip = torch_.zeros((n + 31) // 32, dtype=torch_.int32, device="cuda:0")
+    image = torch_.empty(B.bnn_xnor_prepared_bytes(n, k), dtype=torch_.uint8, device="cuda:0")
+    out = torch_.zeros((m, B.packed_pitch(n)), dtype=torch_.int32, device="cuda:0")
+    for rep in range(4):
+        wp = wl.make_bit_planes(n, k, 0.5, [8, rep, n, k], B.packed_pitch(k))
+        scale = rng.uniform(0.5, 1.5, n).astype(np.float32) * (1 if rep % 2 else -1)
+        shift = rng.normal(0, 3.0, n).astype(np.float32)
+        w_dev, sc, sh = dev(wp), dev(scale), dev(shift)
+        B.bnn_fold_thresholds(sc, sh, n, k, thr, flip, 0)
+        B.bnn_xnor_prepare(w_dev, k, image)
+        B.bnn_xnor_gemm_prepared(a_dev, image, n, k, thr=thr, flip=flip, out_bits=out)
+        want = o.affine_sign_pack_i32(o.xnor_gemm(ap, wp, k), scale, shift, 0)
+        np.testing.assert_array_equal(out.cpu().numpy().view(np.uint32)[:, :(n + 31) // 32], want)
+    assert B.bnn_device_status() == 0
+
+
 def test_xnor_gemm_ignores_garbage_in_pad_bits(B, torch_, xnor_path):
     m, n, k = 70, 90, 1000 - 13
     pitch = B.packed_pitch(k) + 4
