@@ -295,9 +295,10 @@ int bnn_signw_gemm(const float* X, int ldx, const uint32_t* Wp, int ldwp,
 static int signw_impl(const float* X, int ldx, const uint32_t* Wp, int ldwp,
                       int M, int N, int K, float* Y, int ldy,
                       const bnn_epilogue* epi, void* workspace, size_t workspace_bytes,
-                      int splice_dim, int splice_left, void* stream) {
+                      int splice_dim, int splice_left, void* stream,
+                      bool image_ready = false, void* out_image = nullptr, int out_kind = 0) {
     if (int rc = check_dims(M, N, K)) return rc;
-    if (!X) return BNN_ERR_NULL;
+    if (!X && !image_ready) return BNN_ERR_NULL;
     if (ldx < (splice_dim > 0 ? splice_dim : K)) return BNN_ERR_SHAPE;
     if (int rc = check_packed(Wp, ldwp, K)) return rc;
     if (Y && ldy < N) return BNN_ERR_SHAPE;
@@ -319,12 +320,12 @@ static int signw_impl(const float* X, int ldx, const uint32_t* Wp, int ldwp,
             a.out_bits = epi->out_bits; a.ldob = epi->ldob;
         }
     }
-    if (!a.Y && !a.out_bits) return BNN_ERR_NULL;
+    if (!a.Y && !a.out_bits && !out_image) return BNN_ERR_NULL;
     if (g_real_path != BNN_PATH_CUDA_CORE) {
         if (workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255u) &&
             workspace_bytes >= signw_image_bytes(M, K, g_signw_terms))
-            return launch_signw_img(a, g_signw_terms, workspace, (cudaStream_t)stream);
-        if (splice_dim > 0) return BNN_ERR_WORKSPACE;
+            return launch_signw_img(a, g_signw_terms, workspace, image_ready, out_image, out_kind, (cudaStream_t)stream);
+        if (splice_dim > 0 || image_ready || out_image) return BNN_ERR_WORKSPACE;
         return launch_signw_tc(a, g_signw_terms, (cudaStream_t)stream);
     }
     if (splice_dim > 0) return BNN_ERR_UNSUPPORTED;
@@ -356,7 +357,7 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
                              const float* Wout, int ldw, const float* b, const void* prepared,
                              int M, int C, int H, float* logp, int ldo, int log_softmax,
                              int zo, void* workspace, size_t workspace_bytes, const float* log_prior,
-                             int act, void* mid_event, void* stream) {
+                             int act, void* mid_event, void* stream, bool image_ready = false) {
     if (int rc = check_dims(M, C, H)) return rc;
     if (act != BNN_ACT_NONE && (Hp || log_softmax || (act != BNN_ACT_SIGMOID && act != BNN_ACT_HARDTANH)))
         return BNN_ERR_UNSUPPORTED;
@@ -382,7 +383,9 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
         rc = launch_out_tc(Hp, ldhp, prepared, b, M, C, H, logp, ldo, zo, (cudaStream_t)stream);
     else if (Hf && prepared && g_real_path != BNN_PATH_CUDA_CORE && workspace &&
              !(reinterpret_cast<uintptr_t>(workspace) & 255u) && workspace_bytes >= outf_image_bytes(M, H))
-        rc = launch_outf_tc(Hf, ldhf, prepared, b, M, C, H, logp, ldo, act, workspace, (cudaStream_t)stream);
+        rc = launch_outf_tc(Hf, ldhf, prepared, b, M, C, H, logp, ldo, act, workspace, image_ready, (cudaStream_t)stream);
+    else if (image_ready)
+        return BNN_ERR_WORKSPACE;
     else
         rc = launch_real_gemm(a, (cudaStream_t)stream);
     if (rc) return rc;
@@ -467,11 +470,15 @@ size_t bnn_forward_workspace_bytes(const bnn_model* model, int M) {
     for (int l = 0; l < model->n_layers; ++l) {
         const bnn_layer& y = model->layers[l];
         size_t b = 0;
-        if (y.kind == BNN_LAYER_SIGNW)
+        if (y.kind == BNN_LAYER_SIGNW) {
             b = signw_image_bytes(M, y.K, 3);  // room for either term count
-        else if (y.kind == BNN_LAYER_REAL ||
-                 (y.kind == BNN_LAYER_REAL_OUT && l > 0 && model->layers[l - 1].act != BNN_ACT_SIGN_PACK))
+            // a layer of this kind that feeds another one writes that layer's image while it reads its own
+            if (y.act != BNN_ACT_SIGN_PACK && l + 1 < model->n_layers && model->layers[l + 1].kind != BNN_LAYER_XNOR)
+                b = 2 * round256(signw_image_bytes(M, y.N > y.K ? y.N : y.K, 3));
+        } else if (y.kind == BNN_LAYER_REAL ||
+                   (y.kind == BNN_LAYER_REAL_OUT && l > 0 && model->layers[l - 1].act != BNN_ACT_SIGN_PACK)) {
             b = outf_image_bytes(M, y.K);      // fp32 activations into a real-valued layer
+        }
         if (b > img) img = b;
     }
     return base + round256(img);
@@ -520,6 +527,19 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
     const bool small = g_small_batch && M <= kSmallBatchMax;
     const int zo01 = model->act_values == BNN_VALUES_01;
     bool sync_cleared = false;
+    bool chain_in = false;   // the layer before wrote this layer's split-activation image (slot chain_slot)
+    int chain_slot = 0;
+    size_t img_half = 0;     // bytes of one of the two alternating images: the largest any sign-weight layer reads
+    for (int l = 0; l < L; ++l)
+        if (model->layers[l].kind == BNN_LAYER_SIGNW) {
+            size_t b = round256(signw_image_bytes(M, model->layers[l].K, g_signw_terms));
+            if (b > img_half) img_half = b;
+            // the real-valued layer it may feed reads an image of its own format
+            if (l + 1 < L && (model->layers[l + 1].kind == BNN_LAYER_REAL_OUT || model->layers[l + 1].kind == BNN_LAYER_REAL)) {
+                b = round256(outf_image_bytes(M, model->layers[l].N));
+                if (b > img_half) img_half = b;
+            }
+        }
     int sync_used = 0;   // counters handed to earlier runs of this call
     for (int l = 0; l < L; ++l) {
         const bnn_layer& y = model->layers[l];
@@ -543,8 +563,9 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
             int rc = output_layer_impl(in_bits ? static_cast<const uint32_t*>(in) : nullptr, in_ld,
                                        in_bits ? nullptr : static_cast<const float*>(in), in_ld,
                                        y.W, y.ldw, y.shift, y.W_prepared, M, y.N, y.K, logp, ldo, 1,
-                                       in_bits && model->act_values == BNN_VALUES_01, img, img_bytes,
-                                       model->log_prior, BNN_ACT_NONE, events ? events[L + 1] : nullptr, stream);
+                                       in_bits && model->act_values == BNN_VALUES_01,
+                                       chain_in ? img + (size_t)chain_slot * img_half : img, chain_in ? img_half : img_bytes,
+                                       model->log_prior, BNN_ACT_NONE, events ? events[L + 1] : nullptr, stream, chain_in);
             if (rc) return rc;
             if (events && events[L] &&
                 cudaEventRecord((cudaEvent_t)events[L], (cudaStream_t)stream) != cudaSuccess)
@@ -605,22 +626,37 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
             e.scale = y.scale; e.shift = y.shift;
             float* yf = nullptr;
             int out_ld;
+            // A layer of this kind that feeds another one writes its outputs straight into that layer's
+            // split-activation image (two images alternate in the scratch beyond the activation buffers),
+            // and as fp32 only where the caller asked to see them.
+            const bnn_layer* nx = l + 1 < L ? &model->layers[l + 1] : nullptr;
+            const bool to_signw = nx && nx->kind == BNN_LAYER_SIGNW && !(small && nx->act == BNN_ACT_SIGN_PACK);
+            const bool to_real = nx && (nx->kind == BNN_LAYER_REAL_OUT || nx->kind == BNN_LAYER_REAL) && nx->W_prepared;
+            const bool chain_out = y.act != BNN_ACT_SIGN_PACK && (to_signw || to_real) &&
+                                   g_real_path != BNN_PATH_CUDA_CORE && img_bytes >= 2 * img_half;
+            char* img_in = img + (chain_in ? (size_t)chain_slot * img_half : 0);
+            char* img_out = chain_out ? img + (size_t)((chain_in ? chain_slot : 0) ^ 1) * img_half : nullptr;
             if (y.act == BNN_ACT_SIGN_PACK) {
                 e.out_bits = static_cast<uint32_t*>(out); e.ldob = bnn_packed_pitch(y.N);
                 out_ld = e.ldob;
             } else {
-                yf = static_cast<float*>(out);
+                if (!chain_out || (layer_out && layer_out[l])) yf = static_cast<float*>(out);
                 out_ld = y.N;
             }
             rc = signw_impl(static_cast<const float*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
-                            yf, y.N, &e, img, img_bytes, l == 0 ? splice_dim : 0, model->splice_left, stream);
+                            yf, y.N, &e, img_in, chain_in ? img_half : (chain_out ? img_half : img_bytes),
+                            l == 0 ? splice_dim : 0, model->splice_left, stream, chain_in, img_out, to_real ? 1 : 0);
             in_ld = out_ld;
+            if (chain_out) chain_slot = (chain_in ? chain_slot : 0) ^ 1;
+            chain_in = chain_out;
         } else if (y.kind == BNN_LAYER_REAL) {
             if (l == 0 && splice_dim > 0) return BNN_ERR_UNSUPPORTED;
             rc = output_layer_impl(nullptr, 0, static_cast<const float*>(in), in_ld, y.W, y.ldw, y.shift,
                                    y.W_prepared, M, y.N, y.K, static_cast<float*>(out), y.N, 0, 0,
-                                   img, img_bytes, nullptr, y.act, nullptr, stream);
+                                   chain_in ? img + (size_t)chain_slot * img_half : img, chain_in ? img_half : img_bytes,
+                                   nullptr, y.act, nullptr, stream, chain_in);
             in_ld = y.N;
+            chain_in = false;
         } else if (y.act == BNN_ACT_SIGMOID) {
             // binary layer with Sigmoid units: the integer dot products go to the output buffer
             // and are turned into fp32 activations in place

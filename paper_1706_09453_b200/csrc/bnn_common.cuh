@@ -190,7 +190,13 @@ int launch_signw_tc(const RealGemmArgs& a, int terms, cudaStream_t st);
 // Same product with the activations split once into a scratch image (see signw_img_tc.cu):
 // `workspace` must hold signw_image_bytes(M, K, terms) bytes, 256-byte aligned.
 size_t signw_image_bytes(int M, int K, int terms);
-int launch_signw_img(const RealGemmArgs& a, int terms, void* workspace, cudaStream_t st);
+// image_ready: `workspace` already holds the image of a.Af's values (a.Af is not read then);
+// out_image (256-byte aligned, signw_image_bytes(M, N, terms) bytes) or nullptr: the outputs are also
+// written as the image of a following layer of this kind with fan-in N.
+// out_kind 0: that layer's own image (bf16 terms, blocks of 128 frames); 1: the image the real-valued
+// layer on fp32 activations reads (two fp16 terms, blocks of 256 frames, outf_image_bytes(M, N) bytes).
+int launch_signw_img(const RealGemmArgs& a, int terms, void* workspace, bool image_ready, void* out_image, int out_kind,
+                     cudaStream_t st);
 size_t out_prepared_bytes(int C, int H);
 int launch_out_prepare(const float* W, int ldw, int C, int H, void* prepared, cudaStream_t st);
 int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const float* bias,
@@ -198,9 +204,10 @@ int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const floa
 // The top layer on fp32 activations (finite, |a| < 65504) with both operands split into fp16
 // terms (out_gemm_f32_tc.cu): `workspace` holds outf_image_bytes(M, H) bytes, 256-byte aligned.
 size_t outf_image_bytes(int M, int H);
-// `act`: bnn_act applied after the bias (NONE, SIGMOID, HARDTANH).
+// `act`: bnn_act applied after the bias (NONE, SIGMOID, HARDTANH).  image_ready: `workspace` already
+// holds the fp16 image of the activations (written by launch_signw_img with out_kind 1); Hf is not read.
 int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float* bias,
-                   int M, int C, int H, float* Z, int ldz, int act, void* workspace, cudaStream_t st);
+                   int M, int C, int H, float* Z, int ldz, int act, void* workspace, bool image_ready, cudaStream_t st);
 // Y = Sigmoid(fma(scale, D, shift)) element by element (Y may alias D when the pitches agree).
 int launch_affine_sigmoid_i32(const int32_t* D, int ldd, const float* scale, const float* shift,
                               int M, int N, float* Y, int ldy, cudaStream_t st);

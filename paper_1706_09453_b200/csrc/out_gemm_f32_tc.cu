@@ -243,7 +243,7 @@ size_t outf_image_bytes(int M, int H) {
 }
 
 int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float* bias,
-                   int M, int C, int H, float* Z, int ldz, int act, void* workspace, cudaStream_t st) {
+                   int M, int C, int H, float* Z, int ldz, int act, void* workspace, bool image_ready, cudaStream_t st) {
     const int sms = device_sm_count();
     if (sms <= 0 || !ensure_dynamic_smem(reinterpret_cast<const void*>(outf_tc_kernel), SMEM_BYTES)) return BNN_ERR_CUDA;
     const int ct = ceil_div(C, BC), hs = ceil_div(H, BK), ft = ceil_div(M, FN);
@@ -253,7 +253,8 @@ int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float*
     uint8_t* himg = static_cast<uint8_t*>(workspace);
     const TcStatus status = tc_status();
     if (!status.word) return BNN_ERR_CUDA;
-    h_split_kernel<<<ft * hs, FN, 0, st>>>(Hf, ldhf, M, H, hs, himg);
+    if (!image_ready)   // (else the layer that produced the activations wrote the image itself)
+        h_split_kernel<<<ft * hs, FN, 0, st>>>(Hf, ldhf, M, H, hs, himg);
     const int tiles = ct * ft;
     outf_tc_kernel<<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(himg, wimg, rs, bias, M, C, H, Z, ldz, act, status);
     return launch_status();

@@ -11,12 +11,16 @@
 // Frames are on the M side (TMEM lane = frame), units on the N side.  A CTA tile is 128 frames
 // x 512 units (two 256-column accumulators fed by the same activation stage).  The epilogue
 // thread owns a frame: per-unit affine (one fma), then Sign + pack (16 words per row and
-// tile) and/or fp32 stores of 128 contiguous bytes.
+// tile) and/or fp32 stores of 128 contiguous bytes.  When the layer that consumes the outputs is
+// again of this kind (a network with binary weights and real activations, Algorithm 1), the
+// epilogue can also write them as that layer's image (step 1 above), which saves the split pass
+// and one round trip of the fp32 activations.
 //
 // |result - exact| <= 2^-17 * sum_k |x[m][k]| with 2 terms (products exact with 3), plus fp32
 // accumulation rounding.  The contraction index is permuted inside each group of 32 exactly
 // as in the other sign-weight kernel: word t of a K step holds k = t and k = t + 16.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "bnn_common.cuh"
 #include "tcgen05.cuh"
@@ -213,12 +217,22 @@ __device__ __forceinline__ void epilogue_bits(uint32_t taddr, const float* sc, c
     tmem_ld_wait();
 }
 
-// Epilogue of one 256-column accumulator with an fp32 output (and packed bits as well when the
-// activation is Sign).
-template <int ACT>
+// Epilogue of one 256-column accumulator with real-valued outputs: fp32 rows in `y`, packed bits as
+// well when the activation is Sign, and / or the outputs as the split-activation image of the layer
+// that consumes them (`img`: the block of this frame tile and of the first K stage these columns
+// belong to; 32 columns are one stage of the consumer, stored exactly as x_split_kernel stores them).
+// Where an epilogue thread writes its row of a consumer's image: address of its 16 bytes in chunk 0 of
+// term 0 of the first stage, and the distances between stages, terms and chunks.
+struct ImageOut {
+    uint8_t* base;
+    uint32_t stage_stride, plane_stride, chunk_stride;
+    bool fp16;
+};
+
+template <int ACT, int NT>
 __device__ __forceinline__ void epilogue_real(uint32_t taddr, const float* sc, const float* sh, int cols_left,
                                               float* y, bool vec, uint32_t* bits, int words_left, bool row_ok,
-                                              int sign_mode) {
+                                              int sign_mode, const ImageOut& img) {
     uint32_t a0[16], a1[16];
     tmem_ld16(taddr, a0);
     auto emit = [&](uint32_t (&a)[16], int c) -> uint32_t {   // columns c .. c+15 of the accumulator
@@ -244,24 +258,61 @@ __device__ __forceinline__ void epilogue_real(uint32_t taddr, const float* sc, c
         return wd;
     };
 #pragma unroll 1
-    for (int gi = 0; gi < 8; ++gi) {              // one packed word per iteration
+    for (int gi = 0; gi < 8; ++gi) {              // one packed word / one K stage of the consumer per iteration
         const int c = gi * 32;
         if (c >= cols_left) break;                // uniform over the CTA
         tmem_ld_wait();
         tmem_ld16(taddr + c + 16, a1);
         uint32_t wd = emit(a0, c);
         tmem_ld_wait();
-        if (c + 32 < 256) tmem_ld16(taddr + c + 32, a0);
         wd |= emit(a1, c + 16) << 16;
         if (ACT == BNN_ACT_SIGN_PACK && bits && row_ok && gi < words_left) {
             const int valid = cols_left - c;
             bits[gi] = valid >= 32 ? wd : (wd & ((1u << valid) - 1u));
         }
+        if (img.base) {
+            // word e of 16-byte chunk jc pairs column 4 jc + e (low half) with column 4 jc + e + 16;
+            // columns beyond the layer's last unit and rows beyond the batch are stored as zeros
+            uint8_t* blk = img.base + (size_t)gi * img.stage_stride;
+#pragma unroll
+            for (int jc = 0; jc < 4; ++jc) {
+                uint32_t w[3][4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int i = 4 * jc + e;
+                    float lo = (row_ok && c + i < cols_left) ? __uint_as_float(a0[i]) : 0.f;
+                    float hi = (row_ok && c + 16 + i < cols_left) ? __uint_as_float(a1[i]) : 0.f;
+                    if (img.fp16) {     // two fp16 terms
+                        const __half l1 = __float2half_rn(lo), h1 = __float2half_rn(hi);
+                        const __half l2 = __float2half_rn(lo - __half2float(l1)), h2 = __float2half_rn(hi - __half2float(h1));
+                        w[0][e] = (uint32_t)__half_as_ushort(l1) | ((uint32_t)__half_as_ushort(h1) << 16);
+                        w[1][e] = (uint32_t)__half_as_ushort(l2) | ((uint32_t)__half_as_ushort(h2) << 16);
+                    } else {            // NT bf16 terms
+#pragma unroll
+                        for (int q = 0; q < NT; ++q) {
+                            const uint32_t pk = pack_bf16x2(lo, hi);
+                            w[q][e] = pk;
+                            if (q + 1 < NT) { lo -= bf16_lo_as_float(pk); hi -= bf16_hi_as_float(pk); }
+                        }
+                    }
+                }
+                const int planes = img.fp16 ? 2 : NT;
+#pragma unroll
+                for (int q = 0; q < 3; ++q)
+                    if (q < planes)
+                        *reinterpret_cast<uint4*>(blk + q * img.plane_stride + jc * img.chunk_stride) = make_uint4(w[q][0], w[q][1], w[q][2], w[q][3]);
+            }
+        }
+        if (c + 32 < 256) tmem_ld16(taddr + c + 32, a0);
     }
     tmem_ld_wait();
 }
 
 struct Args {
+    uint8_t* img_out;        // split-activation image of the layer that consumes this one's outputs, or nullptr
+    int nks_out;             //   its K stages per block of frames
+    int img_out_kind;        //   0: bf16 terms, blocks of 128 frames (this kernel's own input format);
+                             //   1: two fp16 terms, blocks of 256 frames (the real-valued layer on fp32 activations)
     const uint8_t* img;
     const uint32_t* Wp; int ldwp;
     int M, N, K;
@@ -460,17 +511,29 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
                     float* y = g.Y ? g.Y + (size_t)(m < M ? m : 0) * g.ldy + n0 + c0 : nullptr;
                     const float* sc = &ctl->sc[c0];
                     const float* sh = &ctl->sh[c0];
+                    ImageOut io{nullptr, 0u, 0u, 0u, false};
+                    if (g.img_out) {
+                        const int ks0 = (n0 + c0) >> 5;   // first K stage of the consumer these columns belong to
+                        if (g.img_out_kind == 1) {
+                            const int mrow = m0 + row_in_tile;   // blocks of 256 frames, 32 KB per stage: [term][chunk][row][16 B]
+                            io = ImageOut{g.img_out + ((size_t)(mrow >> 8) * g.nks_out + ks0) * 32768u + (size_t)(mrow & 255) * 16,
+                                          32768u, 16384u, 4096u, true};
+                        } else {
+                            io = ImageOut{g.img_out + ((size_t)(m0 / BM) * g.nks_out + ks0) * (NT * A_PLANE) + (size_t)row_in_tile * 16,
+                                          (uint32_t)(NT * A_PLANE), (uint32_t)A_PLANE, (uint32_t)(BM * 16), false};
+                        }
+                    }
                     if (pack && !g.Y) {
                         if (g.sign_mode == kSignZeroNeg) epilogue_bits<true>(taddr, sc, sh, left, bits, nw - w0, m < M);
                         else epilogue_bits<false>(taddr, sc, sh, left, bits, nw - w0, m < M);
                     } else if (pack) {
-                        epilogue_real<BNN_ACT_SIGN_PACK>(taddr, sc, sh, left, y, vy, bits, nw - w0, m < M, g.sign_mode);
+                        epilogue_real<BNN_ACT_SIGN_PACK, NT>(taddr, sc, sh, left, y, vy, bits, nw - w0, m < M, g.sign_mode, ImageOut{nullptr, 0u, 0u, 0u, false});
                     } else if (g.act == BNN_ACT_HARDTANH) {
-                        epilogue_real<BNN_ACT_HARDTANH>(taddr, sc, sh, left, y, vy, nullptr, 0, m < M, g.sign_mode);
+                        epilogue_real<BNN_ACT_HARDTANH, NT>(taddr, sc, sh, left, y, vy, nullptr, 0, m < M, g.sign_mode, io);
                     } else if (g.act == BNN_ACT_SIGMOID) {
-                        epilogue_real<BNN_ACT_SIGMOID>(taddr, sc, sh, left, y, vy, nullptr, 0, m < M, g.sign_mode);
+                        epilogue_real<BNN_ACT_SIGMOID, NT>(taddr, sc, sh, left, y, vy, nullptr, 0, m < M, g.sign_mode, io);
                     } else {
-                        epilogue_real<BNN_ACT_NONE>(taddr, sc, sh, left, y, vy, nullptr, 0, m < M, g.sign_mode);
+                        epilogue_real<BNN_ACT_NONE, NT>(taddr, sc, sh, left, y, vy, nullptr, 0, m < M, g.sign_mode, io);
                     }
                 }
                 // accumulator `sub` is free again: the MMA thread starts the next tile on accumulator 0
@@ -492,15 +555,18 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
 }
 
 template <int NT>
-int launch_nt(const RealGemmArgs& r, void* workspace, cudaStream_t st) {
+int launch_nt(const RealGemmArgs& r, void* workspace, bool image_ready, void* out_image, int out_kind, cudaStream_t st) {
     using C = Cfg<NT>;
     constexpr int SMEM = C::STAGES * C::STAGE_BYTES + (int)sizeof(Control) + 128;
     const int sms = device_sm_count();
     if (sms <= 0 || !ensure_dynamic_smem(reinterpret_cast<const void*>(signw_img_kernel<NT>), SMEM)) return BNN_ERR_CUDA;
     const int nks = ceil_div(r.K, BK), mt = ceil_div(r.M, BM);
     uint8_t* img = static_cast<uint8_t*>(workspace);
-    x_split_kernel<NT><<<mt * nks, 256, 0, st>>>(r.Af, r.lda, r.M, r.K, nks, img, r.splice_dim, r.splice_left);
-    Args a{img, r.Bb, r.ldb, r.M, r.N, r.K, r.scale, r.shift, r.act, r.sign_mode, r.Y, r.ldy, r.out_bits, r.ldob,
+    // (when the kernel before this one in the stream already wrote the image -- the layer that produced
+    // these activations -- there is nothing to split)
+    if (!image_ready)
+        x_split_kernel<NT><<<mt * nks, 256, 0, st>>>(r.Af, r.lda, r.M, r.K, nks, img, r.splice_dim, r.splice_left);
+    Args a{static_cast<uint8_t*>(out_image), ceil_div(r.N, BK), out_kind, img, r.Bb, r.ldb, r.M, r.N, r.K, r.scale, r.shift, r.act, r.sign_mode, r.Y, r.ldy, r.out_bits, r.ldob,
            tc_status()};
     if (!a.status.word) return BNN_ERR_CUDA;
     const int tiles = mt * ceil_div(r.N, UN);
@@ -515,8 +581,10 @@ size_t signw_image_bytes(int M, int K, int terms) {
     return (size_t)ceil_div(M, BM) * ceil_div(K, BK) * (terms == 3 ? 3 : 2) * A_PLANE;
 }
 
-int launch_signw_img(const RealGemmArgs& r, int terms, void* workspace, cudaStream_t st) {
-    return terms == 3 ? launch_nt<3>(r, workspace, st) : launch_nt<2>(r, workspace, st);
+int launch_signw_img(const RealGemmArgs& r, int terms, void* workspace, bool image_ready, void* out_image, int out_kind,
+                     cudaStream_t st) {
+    return terms == 3 ? launch_nt<3>(r, workspace, image_ready, out_image, out_kind, st)
+                      : launch_nt<2>(r, workspace, image_ready, out_image, out_kind, st);
 }
 
 }  // namespace bnn

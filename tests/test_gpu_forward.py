@@ -195,6 +195,26 @@ def test_forward_unwritten_workspace_path_equals_layer_out_path(env):
     assert torch.equal(a, b)
 
 
+def test_forward_binary_weights_only_chained_images_equal_fp32_hand_over(env):
+    """Binary weights, real activations: without layer_out every hidden layer writes the next layer's
+    split-activation image directly; with layer_out it also stores fp32 rows.  Both, and the minimal
+    scratch (fp32 rows, split again by every layer), give the same log-probabilities bit for bit: the
+    bf16 terms are the same numbers however they get into the image."""
+    torch, B, model = env
+    cfg = wl.CONFIGS["wsj_bw"]
+    frames = 300
+    dn = model.DeviceNet(wl.make_model(cfg))
+    X = model.to_dev(wl.make_frames(cfg, frames))
+    a = dn.forward(X).clone()
+    b = dn.forward(X, layer_out=dn.layer_out_buffers(frames)).clone()
+    assert torch.equal(a, b)
+    small = torch.empty(dn.desc.min_workspace_bytes(frames), dtype=torch.uint8, device="cuda:0")
+    c = torch.empty_like(a)
+    B.bnn_forward(dn.desc, X, c, small)
+    assert (a - c).abs().max().item() <= LOGP_TOL
+    assert B.bnn_device_status() == 0
+
+
 def run_bw_net(env, cfg, frames, sample=None):
     torch, B, model = env
     net = wl.make_model(cfg)
