@@ -664,9 +664,21 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
             rc = xnor_gemm_impl(static_cast<const uint32_t*>(in), in_ld, y.Wp, y.ldwp,
                                 image ? y.W_prepared : nullptr, M, y.N, y.K, static_cast<int32_t*>(out), y.N,
                                 nullptr, model->act_values == BNN_VALUES_01, stream);
-            if (!rc)
+            // The real-valued layer that consumes these units reads its activations as an image of fp16
+            // terms: when there is room for it the Sigmoid goes straight into that image, else into fp32.
+            const bnn_layer* nx = l + 1 < L ? &model->layers[l + 1] : nullptr;
+            const size_t need_img = round256(outf_image_bytes(M, y.N));
+            const bool to_image = nx && (nx->kind == BNN_LAYER_REAL_OUT || nx->kind == BNN_LAYER_REAL) && nx->W_prepared &&
+                                  g_real_path != BNN_PATH_CUDA_CORE && img_bytes >= need_img && !(layer_out && layer_out[l]);
+            if (!rc && to_image) {
+                rc = launch_outf_image_from_i32(static_cast<const int32_t*>(out), y.N, y.scale, y.shift, M, y.N, img,
+                                                (cudaStream_t)stream);
+                chain_in = true; chain_slot = 0;
+                if (img_half < need_img) img_half = need_img;
+            } else if (!rc) {
                 rc = launch_affine_sigmoid_i32(static_cast<const int32_t*>(out), y.N, y.scale, y.shift, M, y.N,
                                                static_cast<float*>(out), y.N, (cudaStream_t)stream);
+            }
             in_ld = y.N;
         } else {
             e.thr = y.thr; e.flip = y.flip;

@@ -208,6 +208,10 @@ size_t outf_image_bytes(int M, int H);
 // holds the fp16 image of the activations (written by launch_signw_img with out_kind 1); Hf is not read.
 int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float* bias,
                    int M, int C, int H, float* Z, int ldz, int act, void* workspace, bool image_ready, cudaStream_t st);
+// The image launch_outf_tc reads (image_ready), made from integer dot products D [M][ldd]: the activations
+// are Sigmoid(fma(scale[h], d, shift[h])).  image: outf_image_bytes(M, H) bytes, 256-byte aligned.
+int launch_outf_image_from_i32(const int32_t* D, int ldd, const float* scale, const float* shift, int M, int H,
+                               void* image, cudaStream_t st);
 // Y = Sigmoid(fma(scale, D, shift)) element by element (Y may alias D when the pitches agree).
 int launch_affine_sigmoid_i32(const int32_t* D, int ldd, const float* scale, const float* shift,
                               int M, int N, float* Y, int ldy, cudaStream_t st);

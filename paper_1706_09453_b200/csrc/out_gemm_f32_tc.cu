@@ -64,15 +64,43 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 // Block (ft, ks) of the image: [term 0..1][chunk c = 2 j + cc][row 0..255][16 bytes], where
 // chunk (j, cc) holds, in element e, position k = 32 ks + 8 j + (pos >> 1) + 16 (pos & 1),
 // pos = 8 cc + e: the order of the prepared weight image, so both operands agree on k.
+// FROM_I32: the activations are Sigmoid(fma(scale[h], d, shift[h])) of integer dot products d (a binary
+// layer with Sigmoid units, Section 3.2 / Table 2), evaluated here instead of in a pass of their own.
+template <bool FROM_I32>
 __global__ void __launch_bounds__(FN)
-h_split_kernel(const float* __restrict__ Hf, int ldh, int M, int H, int nks, uint8_t* __restrict__ img) {
+h_split_kernel(const void* __restrict__ src, int ldh, int M, int H, int nks, uint8_t* __restrict__ img,
+               const float* __restrict__ scale, const float* __restrict__ shift) {
     const int ft = blockIdx.x / nks, ks = blockIdx.x % nks;
     const int row = threadIdx.x, m = ft * FN + row;
     float v[BK];
+    const bool vec = (ldh % 4 == 0) && ((reinterpret_cast<uintptr_t>(src) & 15) == 0) && ks * BK + BK <= H;
+    if (m < M && vec) {
+        const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint32_t*>(src) + (size_t)m * ldh + ks * BK);
 #pragma unroll
-    for (int k = 0; k < BK; ++k) {
-        const int kk = ks * BK + k;
-        v[k] = (m < M && kk < H) ? __ldg(Hf + (size_t)m * ldh + kk) : 0.f;
+        for (int q = 0; q < BK / 4; ++q) {
+            const uint4 t = __ldg(p + q);
+            v[4 * q] = __uint_as_float(t.x); v[4 * q + 1] = __uint_as_float(t.y);
+            v[4 * q + 2] = __uint_as_float(t.z); v[4 * q + 3] = __uint_as_float(t.w);
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < BK; ++k) {
+            const int kk = ks * BK + k;
+            v[k] = (m < M && kk < H) ? __uint_as_float(__ldg(static_cast<const uint32_t*>(src) + (size_t)m * ldh + kk)) : 0.f;
+        }
+    }
+    if (FROM_I32) {
+#pragma unroll
+        for (int k = 0; k < BK; ++k) {
+            const int kk = ks * BK + k;
+            if (m < M && kk < H) {
+                const float d = (float)__float_as_int(v[k]);
+                const float y = fmaf(scale ? __ldg(scale + kk) : 1.0f, d, shift ? __ldg(shift + kk) : 0.0f);
+                v[k] = 1.0f / (1.0f + expf(-y));
+            } else {
+                v[k] = 0.f;
+            }
+        }
     }
     uint8_t* blk = img + ((size_t)ft * nks + ks) * B_BYTES;
 #pragma unroll
@@ -254,9 +282,17 @@ int launch_outf_tc(const float* Hf, int ldhf, const void* prepared, const float*
     const TcStatus status = tc_status();
     if (!status.word) return BNN_ERR_CUDA;
     if (!image_ready)   // (else the layer that produced the activations wrote the image itself)
-        h_split_kernel<<<ft * hs, FN, 0, st>>>(Hf, ldhf, M, H, hs, himg);
+        h_split_kernel<false><<<ft * hs, FN, 0, st>>>(Hf, ldhf, M, H, hs, himg, nullptr, nullptr);
     const int tiles = ct * ft;
     outf_tc_kernel<<<tiles < sms ? tiles : sms, THREADS, SMEM_BYTES, st>>>(himg, wimg, rs, bias, M, C, H, Z, ldz, act, status);
+    return launch_status();
+}
+
+
+int launch_outf_image_from_i32(const int32_t* D, int ldd, const float* scale, const float* shift, int M, int H,
+                               void* image, cudaStream_t st) {
+    const int hs = ceil_div(H, BK), ft = ceil_div(M, FN);
+    h_split_kernel<true><<<ft * hs, FN, 0, st>>>(D, ldd, M, H, hs, static_cast<uint8_t*>(image), scale, shift);
     return launch_status();
 }
 

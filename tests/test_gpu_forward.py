@@ -215,6 +215,21 @@ def test_forward_binary_weights_only_chained_images_equal_fp32_hand_over(env):
     assert B.bnn_device_status() == 0
 
 
+def test_forward_mixed_topology_sigmoid_units_into_the_top_layers_image(env):
+    """The binary layer with Sigmoid units feeds the real-valued top layer: without layer_out its
+    Sigmoid outputs go straight into the top layer's image of fp16 terms, with layer_out through fp32
+    rows that are split afterwards.  The terms are the same numbers, so the log-probabilities are equal."""
+    torch, B, model = env
+    cfg = wl.CONFIGS["wsj_mixed"]
+    frames = 300
+    dn = model.DeviceNet(wl.make_model(cfg))
+    X = model.to_dev(wl.make_frames(cfg, frames))
+    a = dn.forward(X).clone()
+    b = dn.forward(X, layer_out=dn.layer_out_buffers(frames)).clone()
+    assert torch.equal(a, b)
+    assert B.bnn_device_status() == 0
+
+
 def run_bw_net(env, cfg, frames, sample=None):
     torch, B, model = env
     net = wl.make_model(cfg)
