@@ -486,11 +486,11 @@ def run_ours(args):
     if args.xnor_path != "popc":
         kind = B.RATE_KINDS["mma_mxf4_n192_atmem"]
         scratch = torch.zeros(max(256, B.bnn_pipe_rate_scratch_bytes(kind)), dtype=torch.uint8, device=dev)
-        B.bnn_pipe_rate(kind, 128, scratch)
+        B.bnn_pipe_rate(kind, 512, scratch)
         torch.cuda.synchronize()
         e0.record()
         for _ in range(3):
-            work = B.bnn_pipe_rate(kind, 128, scratch)
+            work = B.bnn_pipe_rate(kind, 512, scratch)
         e1.record()
         torch.cuda.synchronize()
         mxf4_rate = work / (e0.elapsed_time(e1) / 3 * 1e-3) / 1e12
