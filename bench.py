@@ -606,24 +606,29 @@ def run_ours(args):
         # later bit must be equal; those bits come from one more forward on the same input.
         last = (K - 1) % nsets
         g1, outs = None, None
-        binary = cfg.act == 1 and not getattr(cfg, "mixed", False) and args.act_values == "pm1" and not args.splice
-        if binary:
+        mixed = getattr(cfg, "mixed", False)
+        plain = args.act_values == "pm1" and not args.splice
+        binary = cfg.act == 1 and not mixed and plain
+        if (binary or mixed) and plain:
             outs = dn.layer_out_buffers(frames)
             chk = torch.empty_like(Ld[last])
             B.bnn_forward(dn.desc, Xd[last], chk, ws, layer_out=outs)
             torch.cuda.synchronize()
-            g1 = model.words_to_numpy(outs[0][:n], cfg.hidden)
+            # the first layer with Sign units: layer 1, or layer 2 of the mixed topology
+            g1 = model.words_to_numpy(outs[1 if mixed else 0][:n], cfg.hidden)
             same_logp = bool(torch.equal(chk, Ld[last]))
         t0 = time.perf_counter()
         if binary:
             ref = o.forward(Xh[:n], net.W, net.scale, net.shift, net.Wout, net.bout, o.ACT_SIGN, o.SIGN_ZERO_POS,
                             layer1_bits=g1)
+        elif mixed and plain:
+            ref = o.forward_mixed(Xh[:n], net.W, net.scale, net.shift, net.Wout, net.bout, o.SIGN_ZERO_POS, layer2_bits=g1)
         else:
             ref = oracle_step(cfg, net, Xh[:n])
         dt = time.perf_counter() - t0
         out["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": o.num_threads(), "kind": "oracle",
                                "sample": "first %d frames of the batch, one pass (%.1f s)" % (n, dt)}
-        if not args.splice and args.act_values == "pm1":
+        if plain:
             got = Ld[last][:n].cpu().numpy()
             par = {"frames": n, "max_abs_dlogp": float(np.abs(got - ref["logp"]).max()), "tolerance_logp": 1e-4}
             if binary:
@@ -635,8 +640,17 @@ def run_ours(args):
                 par["hidden_bits_equal"] = bool(all(
                     (model.words_to_numpy(outs[l][:n], cfg.hidden) == ref["bits"][l]).all() for l in range(1, cfg.n_hidden)))
                 par["timed_step_logp_equal_to_checked_forward"] = same_logp
+            elif mixed:
+                band = 1e-4 * np.abs(net.scale[1])[None, :] * ref["sumabs2"][:, None]
+                decided = np.abs(ref["pre2"]) > band
+                par["layer2_bits_equal_outside_tolerance_band"] = bool(
+                    (o.unpack_pm1(g1, cfg.hidden)[decided] == o.unpack_pm1(ref["bits_own_layer2"], cfg.hidden)[decided]).all())
+                par["hidden_bits_equal"] = bool(all(
+                    (model.words_to_numpy(outs[l][:n], cfg.hidden) == ref["bits"][l - 1]).all() for l in range(2, cfg.n_hidden - 1)))
+                par["timed_step_logp_equal_to_checked_forward"] = same_logp
             par["ok"] = bool(par["max_abs_dlogp"] <= 1e-4 and par.get("hidden_bits_equal", True)
-                             and par.get("layer1_bits_equal_outside_tolerance_band", True))
+                             and par.get("layer1_bits_equal_outside_tolerance_band", True)
+                             and par.get("layer2_bits_equal_outside_tolerance_band", True))
             out["parity"] = par
     print(json.dumps(out))
     if dist:
