@@ -526,7 +526,16 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
     // spread the weights over all SMs instead of tiling the frames (small_batch.cu).
     const bool small = g_small_batch && M <= kSmallBatchMax;
     const int zo01 = model->act_values == BNN_VALUES_01;
-    bool sync_cleared = false;
+    // The arrival counters of stacked binary layers are cleared before the first layer's kernels, not
+    // in front of the stacked launch itself: a memset between the first layer's kernel and that launch
+    // would take away its programmatic overlap with the first layer's tail.
+    if (g_xnor_stack && !small && lay.sync > 0) {
+        bool any = false;
+        for (int l = 0; l + 1 < L && !any; ++l)
+            any = stackable(model, l) && stackable(model, l + 1) && model->layers[l].N == model->layers[l].K &&
+                  model->layers[l + 1].N == model->layers[l].N && model->layers[l + 1].K == model->layers[l].K;
+        if (any && cudaMemsetAsync(sync, 0, lay.sync, (cudaStream_t)stream) != cudaSuccess) return BNN_ERR_CUDA;
+    }
     bool chain_in = false;   // the layer before wrote this layer's split-activation image (slot chain_slot)
     int chain_slot = 0;
     size_t img_half = 0;     // bytes of one of the two alternating images: the largest any sign-weight layer reads
@@ -590,10 +599,6 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                         return BNN_ERR_CUDA;
                 }
                 if (int rc = check_packed(in, in_ld, y.K)) return rc;
-                if (!sync_cleared) {
-                    if (cudaMemsetAsync(sync, 0, lay.sync, (cudaStream_t)stream) != cudaSuccess) return BNN_ERR_CUDA;
-                    sync_cleared = true;
-                }
                 const int ldob = bnn_packed_pitch(y.N);
                 if (int rc = launch_xnor_stack(static_cast<const uint32_t*>(in), in_ld, sl, n, M, y.N, y.K, ldob, zo01,
                                                sync + sync_used, true, (cudaStream_t)stream))
