@@ -33,8 +33,12 @@ constexpr int A_BYTES = 2 * A_PLANE;        // hi + lo
 constexpr int B_BYTES = FN * BK * 2;        // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int STAGES = 4;
-constexpr int MMA_WARP = 4, PROD_WARP0 = 5, PROD_WARPS = 8, EPI_WARPS = 4;
-constexpr int THREADS = (PROD_WARP0 + PROD_WARPS) * 32;
+constexpr int MMA_WARP = 4, PROD_WARP0 = 5, PROD_WARPS = 8;
+// Epilogue: warps 0-3 and four more after the producers, two per tensor-memory lane quarter.  Of each
+// 256-frame accumulator the first group stores frames [0, 128), the second frames [128, 256): an
+// accumulator is read, and handed back to the MMA thread, in half the time.
+constexpr int EPI2_WARP0 = PROD_WARP0 + PROD_WARPS, EPI_WARPS = 8;
+constexpr int THREADS = (EPI2_WARP0 + 4) * 32;   // 544
 constexpr uint32_t TMEM_COLS = 512;
 
 struct Control {
@@ -141,7 +145,7 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
     tc_fence_after_sync();
     const uint32_t tmem = ctl->tmem_base;
 
-    if (warp >= PROD_WARP0) {
+    if (warp >= PROD_WARP0 && warp < EPI2_WARP0) {
         // ---------------- producers: thread p widens the packed activation rows p and p+256;
         // the first producer thread also starts the bulk copy of the stage's weights.
         const int p = threadIdx.x - PROD_WARP0 * 32;  // 0..255
@@ -267,7 +271,8 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
         __syncwarp();
     } else {
         // ---------------- epilogue: thread = one class (TMEM lane), columns = frames
-        const int row_in_tile = warp * 32 + lane;
+        const int row_in_tile = (warp & 3) * 32 + lane;   // a warp reads the lanes of its quarter: 32 (warp % 4) ..
+        const int half = warp < 4 ? 0 : 1;                // which 128 frames of each accumulator
         uint64_t pol;
         asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
         int tl = 0;
@@ -277,36 +282,36 @@ out_tc_kernel(const uint32_t* __restrict__ Hp, int ldhp, const uint8_t* __restri
             const int f0 = (tile / c_tiles) * FN;
             const float scl = rs[c];                       // rs is padded to whole tiles
             const float bia = (bias && c < C) ? bias[c] : 0.f;
-            ok = epi_all(warp_wait(smem_u32(&ctl->acc_full), (uint32_t)(tl & 1), abort_flag, lane));
+            // the four warps of a group take the same decision, so none is left at a barrier
+            const bool got = warp_wait(smem_u32(&ctl->acc_full), (uint32_t)(tl & 1), abort_flag, lane);
+            ok = half ? epi_all_b(got) : epi_all(got);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+            const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 #pragma unroll 1
-            for (int gi = 0; gi < FN / 32; ++gi) {
-                if (f0 + gi * 32 >= M) break;              // uniform over the CTA
-                uint32_t acc[32];
-                tmem_ld32(taddr + gi * 32, acc);
-                tmem_ld_wait();
-                if (c < C) {
-                    float* dst = Z + (size_t)(f0 + gi * 32) * ldz + c;
+            for (int sub = 0; sub < 2; ++sub) {
+#pragma unroll 1
+                for (int g4 = 0; g4 < 4; ++g4) {
+                    const int gi = sub * 8 + half * 4 + g4;       // group of 32 frames
+                    if (f0 + gi * 32 >= M) break;                  // uniform over the warp
+                    uint32_t acc[32];
+                    tmem_ld32(taddr + gi * 32, acc);
+                    tmem_ld_wait();
+                    if (c < C) {
+                        float* dst = Z + (size_t)(f0 + gi * 32) * ldz + c;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (f0 + gi * 32 + j < M) {
-                            const float zv = fmaf(__uint_as_float(acc[j]), scl, bia);
-                            asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(dst + (size_t)j * ldz), "f"(zv), "l"(pol) : "memory");
-                        }
+                        for (int j = 0; j < 32; ++j)
+                            if (f0 + gi * 32 + j < M) {
+                                const float zv = fmaf(__uint_as_float(acc[j]), scl, bia);
+                                asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(dst + (size_t)j * ldz), "f"(zv), "l"(pol) : "memory");
+                            }
+                    }
                 }
-                if (gi == FN / 64 - 1) {   // accumulator 0 has been read: the next tile may start on it
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[0]));
-                }
-            }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) {
-                if (f0 + (FN / 64 - 1) * 32 >= M) mbar_arrive(smem_u32(&ctl->acc_empty[0]));   // the loop ended before it got there
-                mbar_arrive(smem_u32(&ctl->acc_empty[1]));
+                // this warp's share of accumulator `sub` has been read: once all eight warps are through,
+                // the MMA thread may start the next tile on it
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[sub]));
             }
         }
     }

@@ -125,6 +125,17 @@ __device__ __forceinline__ bool epi_all(bool pred) {
         : "=r"(r) : "r"((uint32_t)pred) : "memory");
     return r != 0;
 }
+// The same vote for a second group of 128 epilogue threads (named barrier 3).
+__device__ __forceinline__ bool epi_all_b(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "barrier.red.and.pred q, 3, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"((uint32_t)pred) : "memory");
+    return r != 0;
+}
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // 16-byte store to a shared-space address (keeps the compiler from using generic stores).
