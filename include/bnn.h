@@ -307,10 +307,13 @@ typedef struct bnn_model {
 } bnn_model;
 
 /* Bytes of scratch for M frames.  bnn_forward_workspace_bytes is what makes bnn_forward
- * fastest: two ping-pong activation buffers plus the split-activation image of the widest
- * sign-weight layer (see bnn_signw_gemm_ws) or of a top layer fed with fp32 activations (see
- * bnn_output_layer_ws).  bnn_forward_min_workspace_bytes is the least it
- * accepts (the two buffers only; sign-weight layers then run without the image). */
+ * fastest: two ping-pong activation buffers, the arrival counters of binary hidden layers that
+ * run as one launch (a few bytes per 128 frames and layer), and room for the split-activation
+ * images: of the widest sign-weight layer (see bnn_signw_gemm_ws; two of them when such layers
+ * follow one another, because each writes the next one's image while it reads its own) or of a
+ * real-valued layer fed with fp32 activations (see bnn_output_layer_ws).
+ * bnn_forward_min_workspace_bytes is the least it accepts (the two buffers and the counters;
+ * sign-weight layers then split their activations inside the GEMM and hand on fp32 rows). */
 BNN_API size_t bnn_forward_workspace_bytes(const bnn_model* model, int M);
 BNN_API size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M);
 
