@@ -139,3 +139,12 @@ def test_model_validation(lib):
     # last layer must be the real-valued one
     bad, keep4 = model(layer(0, 440, 64, 1), layer(1, 64, 64, 1))
     assert B.raw_call("bnn_forward", C.byref(bad), fake, 440, 8, fake, 10, fake, 1 << 20, None, None) == 4
+    # a misaligned layer_out entry of a LATER layer is refused before anything is launched
+    # (0x10000 is not device memory: a launch of the first layer would have failed otherwise)
+    lo = (C.c_void_p * 2)(None, fake + 4)
+    assert B.raw_call("bnn_forward", C.byref(good), fake, 440, 8, fake, 10, fake, 1 << 20, lo, None) == 3
+    # the new status and option entry points
+    assert B.raw_call("bnn_query_status", None, None) == 1
+    assert B.status_string(7) != B.status_string(6)
+    assert B.raw_call("bnn_set_option", 6, 0) == -1      # wait limit: at least one microsecond
+    assert B.raw_call("bnn_set_option", 5, 2) == -1      # stacking: 0 or 1
