@@ -227,8 +227,9 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
                 rows.append(dict(name="real_1", kernel="real_gemm_kernel", work=work, unit="TFLOP/s", bound="alu",
                                  peak=fp32_peak))
         elif xnor and mixed and l == cfg.n_hidden - 1 and xnor_path != "popc":
-            # binary layer with Sigmoid units: int32 dot products, then one pointwise pass
-            rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_tc_kernel+affine_sigmoid_i32_kernel", work=work,
+            # binary layer with Sigmoid units: int32 dot products, then one pass that applies the Sigmoid and
+            # writes the top layer's fp16 activation image
+            rows.append(dict(name="xnor_%d" % (l + 1), kernel="xnor_tc_kernel+h_split_kernel", work=work,
                              unit="Tbop/s", bound="tensor", peak=peaks["mxf4"], peak_nominal_ratio=4.0 * peaks["bf16"]))
         elif xnor and xnor_path in ("tensor", "tensor-unprepared"):
             # 4-bit (e2m1, kind::mxf4) tensor-core MACs, 1 bit-MAC = 2 bop.  Peak: the rate of a bare
@@ -260,8 +261,11 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
         elif real_path == "tensor":
             # bf16 tensor-core MMAs, one pass per bf16 term of the real operand (2 terms);
             # algorithmic flops count the product once
-            rows.append(dict(name="signw_%d" % (l + 1), kernel="x_split_kernel+signw_img_kernel", work=work, unit="TFLOP/s",
-                             bound="tensor", peak=peaks["bf16"], passes=2))
+            # (a sign-weight layer fed by another one finds its split-activation image written by that
+            # layer's epilogue: no split launch of its own)
+            chained = l > 0 and not mixed
+            rows.append(dict(name="signw_%d" % (l + 1), kernel="signw_img_kernel" if chained else "x_split_kernel+signw_img_kernel",
+                             work=work, unit="TFLOP/s", bound="tensor", peak=peaks["bf16"], passes=2))
         else:
             rows.append(dict(name="signw_%d" % (l + 1), kernel="real_gemm_kernel", work=work, unit="TFLOP/s",
                              bound="alu", peak=fp32_peak))
@@ -272,7 +276,8 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
                          peak=peaks["bf16"], passes=2))
     elif real_path == "tensor":
         # fp32 activations: both operands in two fp16 terms, three MMAs per step
-        rows.append(dict(name="output_gemm", kernel="h_split_kernel+outf_tc_kernel", work=owork, unit="TFLOP/s",
+        # (its fp16 activation image comes from the epilogue of the layer before: no split launch)
+        rows.append(dict(name="output_gemm", kernel="outf_tc_kernel", work=owork, unit="TFLOP/s",
                          bound="tensor", peak=peaks["bf16"], passes=3))
     else:
         rows.append(dict(name="output_gemm", kernel="real_gemm_kernel", work=owork, unit="TFLOP/s", bound="alu",
@@ -308,20 +313,24 @@ def hbm_bytes_per_step(cfg, frames):
     return b
 
 
-def ncu_traffic(kernel):
-    """DRAM bytes (read + write) per launch of `kernel` from the committed ncu capture, or
-    None when there is none or the kernel's source has changed since it was taken."""
+def ncu_traffic(kernel, workload):
+    """DRAM bytes (read + write) per launch of `kernel` from the committed ncu capture, or None when
+    there is none for this workload's shapes or the kernel's source has changed since it was taken."""
     import hashlib
     path = os.path.join(ROOT, "profiles", "traffic.json")
     if not os.path.exists(path):
         return None
-    rec = json.load(open(path)).get(kernel)
-    if not rec:
-        return None
-    src = os.path.join(ROOT, "paper_1706_09453_b200", "csrc", rec["source"])
-    if not os.path.exists(src) or hashlib.sha256(open(src, "rb").read()).hexdigest() != rec["source_sha256"]:
-        return None
-    return rec["dram_bytes_per_launch"]
+    table = json.load(open(path))
+    total = 0.0
+    for part in kernel.split("+"):      # a row of two launches (split + GEMM): the sum of both
+        rec = table.get(part)
+        if not rec or workload not in rec.get("workloads", []):
+            return None
+        src = os.path.join(ROOT, "paper_1706_09453_b200", "csrc", rec["source"])
+        if not os.path.exists(src) or hashlib.sha256(open(src, "rb").read()).hexdigest() != rec["source_sha256"]:
+            return None
+        total += rec["dram_bytes_per_launch"]
+    return total
 
 
 # ------------------------------------------------------------------ GPU arm
@@ -546,7 +555,7 @@ def run_ours(args):
         peak_source = "derived from unit counts x max SM clock (%.0f MHz)" % peaks["sm_max_mhz"]
     roofline = {"kernel": dk, "launches_per_step": dg["n"], "bound": dom["bound"],
                 "achieved": achieved, "peak": dom["peak"], "unit": dom["unit"],
-                "frac": achieved / dom["peak"], "traffic": ncu_traffic(dk),
+                "frac": achieved / dom["peak"], "traffic": ncu_traffic(dk, cfg.name if frames == cfg.frames else None),
                 "peak_source": peak_source,
                 "algorithmic_work_per_launch": dg["work"] / dg["n"],
                 "share_of_step": dg["ms"] / sum(layer_ms), "avg_launch_ms": dg["ms"] / dg["n"]}
