@@ -393,7 +393,12 @@ BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, 
  *   BNN_OPT_XNOR_STACK : 1 (default) lets bnn_forward run consecutive binary hidden layers of one
  *                        shape with prepared weights (the loop over l of Algorithm 2's forward pass)
  *                        as ONE launch, in which a layer's frame tiles start as soon as the layer
- *                        before has stored them; 0 launches one kernel per layer.  Same bits.
+ *                        before has stored them; 0 launches one kernel per layer.  Same bits.  The CTAs
+ *                        of such a launch wait for one another, so all of them (one per SM at most)
+ *                        must be resident together: a caller that runs several forward passes on ONE
+ *                        device at the same time (several streams or threads), whose kernels could share
+ *                        the SMs between them, should set 0; otherwise such a launch may give up on a
+ *                        bounded wait (status word set, see bnn_device_status) instead of finishing.
  *   BNN_OPT_WAIT_LIMIT_US: how long a kernel may wait on one of its internal barriers or counters before
  *                        it gives up (see bnn_device_status), in microseconds at a nominal 2 GHz SM
  *                        clock; default 1 000 000, minimum 1.  Applies to launches made after the call. */

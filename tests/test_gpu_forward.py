@@ -131,6 +131,27 @@ def test_forward_small_batch_at_the_edge_of_the_staging_memory(env):
     assert env[1].bnn_device_status() == 0
 
 
+@pytest.mark.parametrize("hidden,n_hidden,frames,values", [
+    (1000, 4, 700, 0),     # units and fan-in not multiples of the tile / stage sizes (ragged last stage)
+    (1280, 3, 1500, 1),    # odd number of K stages; (0,1) activations
+    (96, 5, 300, 0),       # a single, narrow unit tile
+    (512, 11, 400, 0),     # ten binary layers in a row: more than one launch can hold, so two runs
+])
+def test_forward_stacked_hidden_layers_edge_shapes(env, hidden, n_hidden, frames, values):
+    """The run of binary hidden layers as one launch on shapes that exercise its tails, checked against
+    the oracle like every other network (and once more with one launch per layer)."""
+    import dataclasses
+    B = env[1]
+    cfg = dataclasses.replace(wl.CONFIGS["tiny"], hidden=hidden, n_hidden=n_hidden, classes=300)
+    run_binary_net(env, cfg, frames, values=values)
+    prev = B.bnn_set_option(B.OPT_XNOR_STACK, 0)
+    try:
+        run_binary_net(env, cfg, frames, values=values)
+    finally:
+        B.bnn_set_option(B.OPT_XNOR_STACK, prev)
+    assert B.bnn_device_status() == 0
+
+
 def test_forward_wsj_config_full_batch_sampled_frames(env):
     """The benchmark's launch configuration (8192 frames); the oracle checks 600 of them,
     including the first and last tile of frames."""
