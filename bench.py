@@ -48,6 +48,8 @@ def parse_args():
                          "(11 or 15 frames) instead of reading an already spliced input")
     ap.add_argument("--no-stack", action="store_true",
                     help="one launch per binary hidden layer instead of one launch for the run of equal layers")
+    ap.add_argument("--no-follow", action="store_true",
+                    help="run the log-softmax after the top layer's kernel instead of behind it (overlapped)")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every step's kernels from the host instead of replaying a captured CUDA graph")
     ap.add_argument("--sweep", action="store_true",
@@ -356,6 +358,8 @@ def run_ours(args):
     B.bnn_set_option(B.OPT_XNOR_PREPARED, {"auto": 0, "stream": 1, "resident": 2}[args.xnor_prepared])
     if args.no_stack:
         B.bnn_set_option(B.OPT_XNOR_STACK, 0)
+    if args.no_follow:
+        B.bnn_set_option(B.OPT_SOFTMAX_FOLLOW, 0)
     dn = model.DeviceNet(net, device=dev, prepare_xnor=args.xnor_path == "tensor",
                          act_values=B.VALUES_01 if args.act_values == "01" else B.VALUES_PM1,
                          splice=((cfg.in_dim // 40) // 2, (cfg.in_dim // 40) // 2) if args.splice else (0, 0))
@@ -588,6 +592,10 @@ def run_ours(args):
         "config": {"workload": workload_name(cfg, frames), "frames_per_gpu": frames,
                    "launch": "host launches" if args.no_graph else "one captured CUDA graph per step (a single bnn_forward call each)", "l2": "inputs/outputs rotate over %d buffer sets (%.0f MB > 2 x L2); weights stay hot"
                          % (nsets, nsets * set_bytes / 1e6),
+                   "log_softmax": ("after the top layer's kernel" if args.no_follow else
+                                   "launched behind the top layer's tensor-core kernel and overlapped with it where that "
+                                   "kernel has more than one wave of tiles (log_softmax_rows_follow_kernel); the "
+                                   "per-layer rows time the two kernels apart (log_softmax_rows_reg_kernel)"),
                    "sign_zero": "+1", "act_values": "(0,1)" if args.act_values == "01" else "(-1,+1)",
                    "input": "one 40-dim frame per row, context window formed in the first layer" if args.splice else "spliced", "seed": cfg.seed},
         "clocks": ck,

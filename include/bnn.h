@@ -399,12 +399,19 @@ BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, 
  *                        device at the same time (several streams or threads), whose kernels could share
  *                        the SMs between them, should set 0; otherwise such a launch may give up on a
  *                        bounded wait (status word set, see bnn_device_status) instead of finishing.
+ *   BNN_OPT_SOFTMAX_FOLLOW: 1 (default) lets bnn_forward launch the log-softmax of a tensor-core top layer
+ *                        on packed activations BEHIND that layer's kernel instead of after it: the
+ *                        log-softmax kernel shares the SMs with the (tensor-pipe-bound) GEMM and takes every
+ *                        512 frames as soon as all their logits are stored, so that only the last frames are
+ *                        left when the GEMM ends.  Same log-probabilities.  Its waits are bounded like all
+ *                        others (BNN_OPT_WAIT_LIMIT_US).  0 runs the two kernels one after the other; so does
+ *                        bnn_forward_events, whose per-layer events need them apart.
  *   BNN_OPT_WAIT_LIMIT_US: how long a kernel may wait on one of its internal barriers or counters before
  *                        it gives up (see bnn_device_status), in microseconds at a nominal 2 GHz SM
  *                        clock; default 1 000 000, minimum 1.  Applies to launches made after the call. */
 typedef enum { BNN_OPT_XNOR_PATH = 0, BNN_OPT_REAL_PATH = 1, BNN_OPT_SIGNW_TERMS = 2,
                BNN_OPT_XNOR_PREPARED = 3, BNN_OPT_SMALL_BATCH = 4, BNN_OPT_XNOR_STACK = 5,
-               BNN_OPT_WAIT_LIMIT_US = 6 } bnn_option;
+               BNN_OPT_WAIT_LIMIT_US = 6, BNN_OPT_SOFTMAX_FOLLOW = 7 } bnn_option;
 typedef enum { BNN_PATH_AUTO = 0, BNN_PATH_CUDA_CORE = 1, BNN_PATH_TENSOR = 2 } bnn_path;
 typedef enum { BNN_PREPARED_AUTO = 0, BNN_PREPARED_STREAM = 1, BNN_PREPARED_RESIDENT = 2 } bnn_prepared_kernel;
 BNN_API int bnn_set_option(int option, int value);

@@ -141,6 +141,7 @@ def packed_pitch(k: int) -> int:
 
 
 OPT_XNOR_PATH, OPT_REAL_PATH, OPT_SIGNW_TERMS, OPT_XNOR_PREPARED, OPT_SMALL_BATCH, OPT_XNOR_STACK, OPT_WAIT_LIMIT_US = 0, 1, 2, 3, 4, 5, 6
+OPT_SOFTMAX_FOLLOW = 7
 ERR_TIMEOUT = 7
 PREPARED_AUTO, PREPARED_STREAM, PREPARED_RESIDENT = 0, 1, 2
 PATH_AUTO, PATH_CUDA_CORE, PATH_TENSOR = 0, 1, 2

@@ -14,6 +14,7 @@ int g_xnor_prepared = BNN_PREPARED_AUTO;
 int g_small_batch = 1;  // batches of up to kSmallBatchMax frames take the matrix-vector kernels
 int g_signw_terms = 2;  // |dot| <= K stays exact in every accumulator type used
 int g_xnor_stack = 1;   // runs of equal binary hidden layers go out as one launch
+int g_softmax_follow = 1;   // bnn_forward's log-softmax follows the top layer's kernel tile by tile
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -129,6 +130,7 @@ int bnn_set_option(int option, int value) {
         case BNN_OPT_XNOR_PREPARED: slot = &g_xnor_prepared; break;
         case BNN_OPT_SMALL_BATCH: slot = &g_small_batch; break;
         case BNN_OPT_XNOR_STACK: slot = &g_xnor_stack; break;
+        case BNN_OPT_SOFTMAX_FOLLOW: slot = &g_softmax_follow; break;
         case BNN_OPT_WAIT_LIMIT_US: {
             // microseconds -> SM clocks at a nominal 2 GHz
             if (value < 1) return -1;
@@ -139,7 +141,7 @@ int bnn_set_option(int option, int value) {
     }
     if (option == BNN_OPT_SIGNW_TERMS) {
         if (value != 2 && value != 3) return -1;
-    } else if (option == BNN_OPT_SMALL_BATCH || option == BNN_OPT_XNOR_STACK) {
+    } else if (option == BNN_OPT_SMALL_BATCH || option == BNN_OPT_XNOR_STACK || option == BNN_OPT_SOFTMAX_FOLLOW) {
         if (value != 0 && value != 1) return -1;
     } else if (option == BNN_OPT_XNOR_PREPARED) {
         if (value != BNN_PREPARED_AUTO && value != BNN_PREPARED_STREAM && value != BNN_PREPARED_RESIDENT) return -1;
@@ -357,7 +359,8 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
                              const float* Wout, int ldw, const float* b, const void* prepared,
                              int M, int C, int H, float* logp, int ldo, int log_softmax,
                              int zo, void* workspace, size_t workspace_bytes, const float* log_prior,
-                             int act, void* mid_event, void* stream, bool image_ready = false) {
+                             int act, void* mid_event, void* stream, bool image_ready = false,
+                             int* done = nullptr) {
     if (int rc = check_dims(M, C, H)) return rc;
     if (act != BNN_ACT_NONE && (Hp || log_softmax || (act != BNN_ACT_SIGMOID && act != BNN_ACT_HARDTANH)))
         return BNN_ERR_UNSUPPORTED;
@@ -379,8 +382,13 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
     a.Y = logp; a.ldy = ldo;
     if (prepared && (reinterpret_cast<uintptr_t>(prepared) & 255u)) return BNN_ERR_ALIGN;
     int rc;
+    // `done` (zeroed counters in the caller's workspace): the log-softmax kernel is launched right behind
+    // the tensor-core kernel and takes each group of frames as soon as all its logits are stored
+    const bool follow = done && Hp && prepared && g_real_path != BNN_PATH_CUDA_CORE && log_softmax && !mid_event &&
+                        g_softmax_follow && log_softmax_can_follow(logp, ldo, C, log_prior) &&
+                        out_tc_more_than_one_wave(M, C);
     if (Hp && prepared && g_real_path != BNN_PATH_CUDA_CORE)
-        rc = launch_out_tc(Hp, ldhp, prepared, b, M, C, H, logp, ldo, zo, (cudaStream_t)stream);
+        rc = launch_out_tc(Hp, ldhp, prepared, b, M, C, H, logp, ldo, zo, follow ? done : nullptr, (cudaStream_t)stream);
     else if (Hf && prepared && g_real_path != BNN_PATH_CUDA_CORE && workspace &&
              !(reinterpret_cast<uintptr_t>(workspace) & 255u) && workspace_bytes >= outf_image_bytes(M, H))
         rc = launch_outf_tc(Hf, ldhf, prepared, b, M, C, H, logp, ldo, act, workspace, image_ready, (cudaStream_t)stream);
@@ -391,6 +399,9 @@ static int output_layer_impl(const uint32_t* Hp, int ldhp, const float* Hf, int 
     if (rc) return rc;
     if (mid_event && cudaEventRecord((cudaEvent_t)mid_event, (cudaStream_t)stream) != cudaSuccess)
         return BNN_ERR_CUDA;
+    if (follow)
+        return launch_log_softmax_rows_follow(logp, ldo, M, C, log_prior, done, out_tc_group_arrivals(C),
+                                              out_tc_group_rows(), (cudaStream_t)stream);
     if (log_softmax) return launch_log_softmax_rows(logp, ldo, M, C, log_prior, (cudaStream_t)stream);
     return BNN_OK;
 }
@@ -440,11 +451,12 @@ int bnn_output_layer01(const uint32_t* Hp, int ldhp, const float* Wout, int ldw,
                              log_softmax, 1, nullptr, 0, nullptr, BNN_ACT_NONE, nullptr, stream);
 }
 
-// Layout of the forward workspace: two activation buffers of `half` bytes each, then the arrival
-// counters of the stacked binary layers (`sync` bytes), then whatever the caller gave beyond that
+// Layout of the forward workspace: two activation buffers of `half` bytes each, then `sync` bytes of
+// counters (the arrival counters of the stacked binary layers, `stack_sync` bytes, then the top
+// layer's completed-frame-group counters), then whatever the caller gave beyond that
 // (split-activation images).
 struct WorkspaceLayout {
-    size_t half, sync;
+    size_t half, stack_sync, sync;
     size_t need() const { return 2 * half + sync; }
 };
 static WorkspaceLayout workspace_layout(const bnn_model* model, int M) {
@@ -455,7 +467,9 @@ static WorkspaceLayout workspace_layout(const bnn_model* model, int M) {
         if (b > mx) mx = b;
         if (model->layers[l].kind == BNN_LAYER_XNOR) ++xnor_layers;
     }
-    return WorkspaceLayout{round256(mx), round256(xnor_stack_sync_bytes(M, xnor_layers))};
+    const size_t stack = round256(xnor_stack_sync_bytes(M, xnor_layers));
+    const bool top = model->layers[model->n_layers - 1].kind == BNN_LAYER_REAL_OUT && model->n_layers > 1;
+    return WorkspaceLayout{round256(mx), stack, stack + (top ? round256(out_tc_done_bytes(M)) : 0)};
 }
 
 size_t bnn_forward_min_workspace_bytes(const bnn_model* model, int M) {
@@ -529,12 +543,18 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
     // The arrival counters of stacked binary layers are cleared before the first layer's kernels, not
     // in front of the stacked launch itself: a memset between the first layer's kernel and that launch
     // would take away its programmatic overlap with the first layer's tail.
-    if (g_xnor_stack && !small && lay.sync > 0) {
+    // The same goes for the counters on which the log-softmax follows the top layer's kernel.
+    int* top_done = nullptr;
+    if (!small && lay.sync > 0) {
         bool any = false;
-        for (int l = 0; l + 1 < L && !any; ++l)
+        for (int l = 0; g_xnor_stack && l + 1 < L && !any; ++l)
             any = stackable(model, l) && stackable(model, l + 1) && model->layers[l].N == model->layers[l].K &&
                   model->layers[l + 1].N == model->layers[l].N && model->layers[l + 1].K == model->layers[l].K;
-        if (any && cudaMemsetAsync(sync, 0, lay.sync, (cudaStream_t)stream) != cudaSuccess) return BNN_ERR_CUDA;
+        const bnn_layer& top = model->layers[L - 1];
+        if (g_softmax_follow && !events && lay.sync > lay.stack_sync && top.kind == BNN_LAYER_REAL_OUT && top.W_prepared &&
+            L > 1 && model->layers[L - 2].act == BNN_ACT_SIGN_PACK && out_tc_more_than_one_wave(M, top.N))
+            top_done = sync + lay.stack_sync / sizeof(int);
+        if ((any || top_done) && cudaMemsetAsync(sync, 0, lay.sync, (cudaStream_t)stream) != cudaSuccess) return BNN_ERR_CUDA;
     }
     bool chain_in = false;   // the layer before wrote this layer's split-activation image (slot chain_slot)
     int chain_slot = 0;
@@ -574,7 +594,8 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                                        y.W, y.ldw, y.shift, y.W_prepared, M, y.N, y.K, logp, ldo, 1,
                                        in_bits && model->act_values == BNN_VALUES_01,
                                        chain_in ? img + (size_t)chain_slot * img_half : img, chain_in ? img_half : img_bytes,
-                                       model->log_prior, BNN_ACT_NONE, events ? events[L + 1] : nullptr, stream, chain_in);
+                                       model->log_prior, BNN_ACT_NONE, events ? events[L + 1] : nullptr, stream, chain_in,
+                                       in_bits ? top_done : nullptr);
             if (rc) return rc;
             if (events && events[L] &&
                 cudaEventRecord((cudaEvent_t)events[L], (cudaStream_t)stream) != cudaSuccess)

@@ -199,8 +199,19 @@ int launch_signw_img(const RealGemmArgs& a, int terms, void* workspace, bool ima
                      cudaStream_t st);
 size_t out_prepared_bytes(int C, int H);
 int launch_out_prepare(const float* W, int ldw, int C, int H, void* prepared, cudaStream_t st);
+// `done` (optional, out_tc_done_bytes(M) zeroed bytes): one counter per out_tc_group_rows() frames, then
+// the row counter of the kernel that follows; every epilogue warp adds 1 to a group's counter once its
+// share of a tile of that group is stored; out_tc_group_arrivals(C) arrivals complete a group.
+// launch_log_softmax_rows_follow, launched right behind, consumes the groups in order.
+int out_tc_group_rows();
+int out_tc_group_arrivals(int C);
+size_t out_tc_done_bytes(int M);
+bool out_tc_more_than_one_wave(int M, int C);
 int launch_out_tc(const uint32_t* Hp, int ldhp, const void* prepared, const float* bias,
-                  int M, int C, int H, float* Z, int ldz, int zo, cudaStream_t st);
+                  int M, int C, int H, float* Z, int ldz, int zo, int* done, cudaStream_t st);
+bool log_softmax_can_follow(const float* Z, int ldz, int C, const float* prior);
+int launch_log_softmax_rows_follow(float* Z, int ldz, int M, int C, const float* prior, int* done, int need,
+                                   int group_rows, cudaStream_t st);
 // The top layer on fp32 activations (finite, |a| < 65504) with both operands split into fp16
 // terms (out_gemm_f32_tc.cu): `workspace` holds outf_image_bytes(M, H) bytes, 256-byte aligned.
 size_t outf_image_bytes(int M, int H);

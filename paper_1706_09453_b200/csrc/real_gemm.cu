@@ -11,6 +11,7 @@
 #include <float.h>
 
 #include "bnn_common.cuh"
+#include "tcgen05.cuh"
 
 namespace bnn {
 
@@ -247,65 +248,190 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// Same result with the whole row held in registers (C <= 256*4*V, 16-byte aligned rows):
-// every logit is read from memory once and written once.  The maximum is reduced first (warp
-// shuffles, then 8 values through shared memory), so each element costs a subtract, a
-// multiply, one ex2 and one add; the sum is reduced the same way.
+// One row held in registers by the 256 threads of a CTA (C <= 256*4*V, 16-byte aligned rows): every
+// logit is read from memory once and written once.  The maximum is reduced first (warp shuffles, then
+// 8 values through shared memory), so each element costs a subtract, a multiply, one ex2 and one add;
+// the sum is reduced the same way.  sm/ss: 8 floats of shared scratch each; the caller alternates two
+// sets from row to row, which saves a barrier per row.
+template <int V>
+__device__ __forceinline__ void log_softmax_row_reg(float4* __restrict__ z, int c4, const float* __restrict__ prior,
+                                                    float* sm, float* ss) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+    float4 v[V];
+    float mx = -FLT_MAX;
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        const int c = threadIdx.x + i * 256;
+        v[i] = c < c4 ? z[c] : make_float4(-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX);
+        mx = fmaxf(fmaxf(mx, fmaxf(v[i].x, v[i].y)), fmaxf(v[i].z, v[i].w));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    if (lane == 0) sm[w] = mx;
+    __syncthreads();
+    mx = sm[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) mx = fmaxf(mx, sm[i]);
+    // sum of exp(z - max) = sum of 2^((z - max) log2 e); the difference is taken first, so the
+    // rounding error scales with the distance from the maximum, not with the logit itself;
+    // padding (-FLT_MAX) contributes 0
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < V; ++i)
+        s += (ex2_approx((v[i].x - mx) * kLog2e) + ex2_approx((v[i].y - mx) * kLog2e)) +
+             (ex2_approx((v[i].z - mx) * kLog2e) + ex2_approx((v[i].w - mx) * kLog2e));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    if (lane == 0) ss[w] = s;
+    __syncthreads();
+    s = ss[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) s += ss[i];
+    const float lse = mx + kLn2 * log2f(s);
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        const int c = threadIdx.x + i * 256;
+        if (c < c4) {
+            // optional log-prior of each class (16-byte aligned, C % 4 == 0): a hybrid decoder
+            // wants log p(state | frame) - log p(state)
+            const float4 pr = prior ? __ldg(reinterpret_cast<const float4*>(prior) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+            z[c] = make_float4(v[i].x - lse - pr.x, v[i].y - lse - pr.y, v[i].z - lse - pr.z, v[i].w - lse - pr.w);
+        }
+    }
+}
+
+// R rows at once by a CTA of NT threads (z0, z0 + ldz4, ...; rows at or beyond `rows` are left alone):
+// the loads of all of them are in flight together and the reductions share their barriers.
+// sm/ss: R x (NT / 32) floats each.
+template <int V, int R, int NT>
+__device__ __forceinline__ void log_softmax_rows_reg(float4* __restrict__ z0, size_t ldz4, int rows, int c4,
+                                                     const float* __restrict__ prior, float (*sm)[NT / 32],
+                                                     float (*ss)[NT / 32]) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+    float4 v[R][V];
+    float mx[R], s[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const int c = threadIdx.x + i * NT;
+            v[r][i] = (c < c4 && r < rows) ? __ldcs(z0 + r * ldz4 + c) : make_float4(-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX);
+        }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        mx[r] = -FLT_MAX;
+#pragma unroll
+        for (int i = 0; i < V; ++i)
+            mx[r] = fmaxf(fmaxf(mx[r], fmaxf(v[r][i].x, v[r][i].y)), fmaxf(v[r][i].z, v[r][i].w));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xFFFFFFFFu, mx[r], o));
+        if (lane == 0) sm[r][w] = mx[r];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        mx[r] = sm[r][0];
+#pragma unroll
+        for (int i = 1; i < NT / 32; ++i) mx[r] = fmaxf(mx[r], sm[r][i]);
+        // sum of 2^((z - max) log2 e), as in log_softmax_row_reg; padding (-FLT_MAX) contributes 0
+        s[r] = 0.f;
+#pragma unroll
+        for (int i = 0; i < V; ++i)
+            s[r] += (ex2_approx((v[r][i].x - mx[r]) * kLog2e) + ex2_approx((v[r][i].y - mx[r]) * kLog2e)) +
+                    (ex2_approx((v[r][i].z - mx[r]) * kLog2e) + ex2_approx((v[r][i].w - mx[r]) * kLog2e));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s[r] += __shfl_xor_sync(0xFFFFFFFFu, s[r], o);
+        if (lane == 0) ss[r][w] = s[r];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        float t = ss[r][0];
+#pragma unroll
+        for (int i = 1; i < NT / 32; ++i) t += ss[r][i];
+        const float lse = mx[r] + kLn2 * log2f(t);
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const int c = threadIdx.x + i * NT;
+            if (c < c4 && r < rows) {
+                const float4 pr = prior ? __ldg(reinterpret_cast<const float4*>(prior) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+                __stcs(z0 + r * ldz4 + c, make_float4(v[r][i].x - lse - pr.x, v[r][i].y - lse - pr.y, v[r][i].z - lse - pr.z, v[r][i].w - lse - pr.w));
+            }
+        }
+    }
+}
+
+// Same result as log_softmax_rows_kernel, one CTA per row at a time.
 template <int V>
 __global__ void __launch_bounds__(256)
 log_softmax_rows_reg_kernel(float* __restrict__ Z, int ldz, int M, int C, const float* __restrict__ prior) {
     __shared__ float sm[2][8], ss[2][8];
     const int c4 = C >> 2;  // C % 4 == 0
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
-    int par = 0;   // the two halves of the scratch alternate, which saves a barrier per row
+    int par = 0;
     // Rows are taken from the last one down: the kernel that wrote the logits just before this one
     // produced the last frames last, and those are the rows the L2 cache still holds.
-    for (int r = blockIdx.x; r < M; r += gridDim.x, par ^= 1) {
-        const int row = M - 1 - r;
-        float4* z = reinterpret_cast<float4*>(Z + (size_t)row * ldz);
-        float4 v[V];
-        float mx = -FLT_MAX;
-#pragma unroll
-        for (int i = 0; i < V; ++i) {
-            const int c = threadIdx.x + i * 256;
-            v[i] = c < c4 ? z[c] : make_float4(-FLT_MAX, -FLT_MAX, -FLT_MAX, -FLT_MAX);
-            mx = fmaxf(fmaxf(mx, fmaxf(v[i].x, v[i].y)), fmaxf(v[i].z, v[i].w));
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-        if (lane == 0) sm[par][w] = mx;
-        __syncthreads();
-        mx = sm[par][0];
-#pragma unroll
-        for (int i = 1; i < 8; ++i) mx = fmaxf(mx, sm[par][i]);
-        // sum of exp(z - max) = sum of 2^((z - max) log2 e); the difference is taken first, so the
-        // rounding error scales with the distance from the maximum, not with the logit itself;
-        // padding (-FLT_MAX) contributes 0
-        float s = 0.f;
-#pragma unroll
-        for (int i = 0; i < V; ++i)
-            s += (ex2_approx((v[i].x - mx) * kLog2e) + ex2_approx((v[i].y - mx) * kLog2e)) +
-                 (ex2_approx((v[i].z - mx) * kLog2e) + ex2_approx((v[i].w - mx) * kLog2e));
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-        if (lane == 0) ss[par][w] = s;
-        __syncthreads();
-        s = ss[par][0];
-#pragma unroll
-        for (int i = 1; i < 8; ++i) s += ss[par][i];
-        const float lse = mx + kLn2 * log2f(s);
-#pragma unroll
-        for (int i = 0; i < V; ++i) {
-            const int c = threadIdx.x + i * 256;
-            if (c < c4) {
-                // optional log-prior of each class (16-byte aligned, C % 4 == 0): a hybrid decoder
-                // wants log p(state | frame) - log p(state)
-                const float4 pr = prior ? __ldg(reinterpret_cast<const float4*>(prior) + c) : make_float4(0.f, 0.f, 0.f, 0.f);
-                z[c] = make_float4(v[i].x - lse - pr.x, v[i].y - lse - pr.y, v[i].z - lse - pr.z, v[i].w - lse - pr.w);
+    for (int r = blockIdx.x; r < M; r += gridDim.x, par ^= 1)
+        log_softmax_row_reg<V>(reinterpret_cast<float4*>(Z + (size_t)(M - 1 - r) * ldz), c4, prior, sm[par], ss[par]);
+}
+
+// The same rows, taken while the kernel that writes the logits is still running.  That kernel counts, per
+// group of `group_rows` consecutive frames, the arrivals of the warps that have stored their share of the
+// group (release at GPU scope); a group is complete at `need` arrivals.  This kernel is launched behind it
+// with programmatic stream serialisation: its first CTAs move onto the SMs as soon as every CTA of the
+// producer is resident, share them with it (the producer is bound by the tensor pipe, this one by memory)
+// and follow it group by group, reading the logits from the L2 cache that has just received them; the
+// rest of the grid moves in when the producer's CTAs leave and helps with the last groups.  Rows are
+// claimed kFollowRows at a time, in order, from one counter (done[groups], zero at launch), so a CTA that starts
+// late goes straight to the rows that are left.  Every wait is bounded: after status.limit clocks the
+// CTA sets the status word and returns.
+// The CTA is small -- four warps, one per scheduler of an SM -- because that is what fits beside the 17 warps
+// of 72 registers of the kernel it follows: the busiest scheduler's register file has room for one more
+// warp of up to 152 registers.
+constexpr int kFollowRows = 2, kFollowThreads = 128;
+template <int V>
+__global__ void __launch_bounds__(kFollowThreads)
+log_softmax_rows_follow_kernel(float* __restrict__ Z, int ldz, int M, int C, const float* __restrict__ prior,
+                               int* __restrict__ done, int need, int group_rows, tc::TcStatus status) {
+    constexpr int R = kFollowRows, NT = kFollowThreads;
+    __shared__ float sm[2][R][NT / 32], ss[2][R][NT / 32];
+    __shared__ int claim;
+    const int c4 = C >> 2;
+    int* next_row = done + ceil_div(M, group_rows);
+    int pending = 0, ready_group = -1;   // thread 0: the claim in flight; the last group seen complete
+    int par = 0;
+    if (threadIdx.x == 0) pending = atomicAdd(next_row, R);
+    while (true) {
+        if (threadIdx.x == 0) {
+            int r = pending;
+            const int gi = r / group_rows;           // group_rows is a multiple of R: the rows lie in one group
+            if (r < M && gi > ready_group) {
+                const long long t0 = clock64();
+#pragma unroll 1
+                while (true) {
+                    int v;
+                    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(done + gi) : "memory");
+                    if (v >= need) { ready_group = gi; break; }
+                    if (clock64() - t0 > status.limit) { r = -1; break; }
+                    __nanosleep(200);
+                }
             }
+            claim = r;
         }
+        __syncthreads();
+        const int r = claim;
+        if (r < 0 || r >= M) {
+            if (threadIdx.x == 0 && r < 0) atomicExch(status.word, 1);
+            break;
+        }
+        if (threadIdx.x == 0) pending = atomicAdd(next_row, R);   // in flight while these rows are worked on
+        log_softmax_rows_reg<V, R, NT>(reinterpret_cast<float4*>(Z + (size_t)r * ldz), (size_t)(ldz >> 2), M - r, c4, prior,
+                                   sm[par], ss[par]);
+        par ^= 1;   // the scratch alternates; `claim` is rewritten only after the two barriers inside
     }
+    // completion of this kernel implies completion of the one it followed
+    if (threadIdx.x == 0) pdl_wait();
 }
 
 }  // namespace
@@ -321,6 +447,23 @@ int launch_real_gemm(const RealGemmArgs& a, cudaStream_t st) {
     else
         return BNN_ERR_UNSUPPORTED;
     return launch_status();
+}
+
+bool log_softmax_can_follow(const float* Z, int ldz, int C, const float* prior) {
+    return (C % 4 == 0) && (ldz % 4 == 0) && aligned16(Z) && C <= 128 * 4 * 8 && (!prior || aligned16(prior));
+}
+
+int launch_log_softmax_rows_follow(float* Z, int ldz, int M, int C, const float* prior, int* done, int need,
+                                   int group_rows, cudaStream_t st) {
+    const int sms = device_sm_count();
+    const tc::TcStatus status = tc_status();
+    if (sms <= 0 || !status.word || !log_softmax_can_follow(Z, ldz, C, prior)) return BNN_ERR_CUDA;
+    if (group_rows % kFollowRows != 0) return BNN_ERR_UNSUPPORTED;
+    const int blocks = M < sms * 5 * kFollowRows ? ceil_div(M, kFollowRows) : sms * 5;
+    const cudaError_t e = C <= kFollowThreads * 4 * 4
+        ? launch_pdl(log_softmax_rows_follow_kernel<4>, dim3(blocks), dim3(kFollowThreads), 0, st, Z, ldz, M, C, prior, done, need, group_rows, status)
+        : launch_pdl(log_softmax_rows_follow_kernel<8>, dim3(blocks), dim3(kFollowThreads), 0, st, Z, ldz, M, C, prior, done, need, group_rows, status);
+    return e == cudaSuccess ? launch_status() : BNN_ERR_CUDA;
 }
 
 int launch_log_softmax_rows(float* Z, int ldz, int M, int C, const float* prior, cudaStream_t st) {

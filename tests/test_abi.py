@@ -148,3 +148,5 @@ def test_model_validation(lib):
     assert B.status_string(7) != B.status_string(6)
     assert B.raw_call("bnn_set_option", 6, 0) == -1      # wait limit: at least one microsecond
     assert B.raw_call("bnn_set_option", 5, 2) == -1      # stacking: 0 or 1
+    assert B.raw_call("bnn_set_option", 7, 2) == -1      # log-softmax behind the top layer: 0 or 1
+    assert B.bnn_set_option(B.OPT_SOFTMAX_FOLLOW, 0) == 1 and B.bnn_set_option(B.OPT_SOFTMAX_FOLLOW, 1) == 0

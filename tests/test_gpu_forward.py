@@ -152,6 +152,43 @@ def test_forward_stacked_hidden_layers_edge_shapes(env, hidden, n_hidden, frames
     assert B.bnn_device_status() == 0
 
 
+@pytest.mark.parametrize("frames,classes,values,with_prior", [
+    (2100, 4000, 0, False),   # 5 frame groups x 32 class tiles, ragged last group, the wide-row variant
+    (4700, 2000, 1, True),    # 10 groups x 16 class tiles, the narrow-row variant; (0,1) activations; log-prior
+    (2561, 3400, 0, True),    # one frame in the last group
+])
+def test_forward_log_softmax_following_the_top_layer(env, frames, classes, values, with_prior):
+    """The log-softmax launched behind the top layer's kernel, taking each group of 512 frames as soon as
+    its logits are complete (default when the top layer has more than one wave of tiles), against the
+    oracle, against the two kernels run one after the other, and repeated into the same workspace."""
+    import dataclasses
+    torch, B, model = env
+    cfg = dataclasses.replace(wl.CONFIGS["tiny"], hidden=256, n_hidden=2, classes=classes)
+    net = wl.make_model(cfg)
+    X = wl.make_frames(cfg, frames)
+    rng = np.random.default_rng(frames)
+    log_prior = np.log(rng.dirichlet(np.ones(classes) * 5.0)).astype(np.float32) if with_prior else None
+    dn = model.DeviceNet(net, act_values=values, log_prior=log_prior)
+    outs = dn.layer_out_buffers(frames)
+    Xd = model.to_dev(X)
+    a = dn.forward(Xd, layer_out=outs).clone()
+    g1 = model.words_to_numpy(outs[0], cfg.hidden)
+    ref = o.forward(X, net.W, net.scale, net.shift, net.Wout, net.bout, o.ACT_SIGN, 0, layer1_bits=g1,
+                    values=values, log_prior=log_prior)
+    assert np.abs(a.cpu().numpy() - ref["logp"]).max() <= LOGP_TOL
+    prev = B.bnn_set_option(B.OPT_SOFTMAX_FOLLOW, 0)
+    try:
+        b = dn.forward(Xd, layer_out=outs).clone()
+    finally:
+        B.bnn_set_option(B.OPT_SOFTMAX_FOLLOW, prev)
+    assert prev == 1
+    # the same arithmetic per element; only the order of the row reductions differs
+    assert (a - b).abs().max().item() <= 1e-5
+    for _ in range(3):   # the counters are cleared by every call
+        assert torch.equal(dn.forward(Xd), a)
+    assert B.bnn_device_status() == 0
+
+
 def test_forward_wsj_config_full_batch_sampled_frames(env):
     """The benchmark's launch configuration (8192 frames); the oracle checks 600 of them,
     including the first and last tile of frames."""
