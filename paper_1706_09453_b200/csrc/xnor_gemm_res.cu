@@ -348,7 +348,9 @@ xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ 
         // MMAs (polls, commits, loop bookkeeping) is time the tensor pipe idles, so the waits
         // of two stages are taken together and their eight MMAs issued back to back (12 % off
         // the steady state against one stage per iteration).
-        if (lane == 0) {
+        // The whole warp runs the loop (converged); the MMAs and commits are issued by lane 0 alone.
+        {
+            const uint32_t issue = lane == 0;
             constexpr uint32_t idesc = instr_desc_mxf4(BM, BN);
             const uint32_t sfa = tmem + C::TMEM_SF_COL, sfb = tmem + C::TMEM_SF_COL + SF_COLS / 2;
             // descriptor of stage 0, chunk pair 0; the address field (16-byte units) of the others
@@ -384,14 +386,14 @@ xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ 
                         const uint32_t ta = tmem_a + sa * A_COLS, ta2 = tmem_a + sa2 * A_COLS;
 #pragma unroll
                         for (int j = 0; j < BK / 64; ++j)   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
-                            mma_mxf4_ts(d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
-                        mma_commit(smem_u32(&ctl->empty_a[sa]));
-                        if (hand_over) mma_commit(smem_u32(&ctl->b_free[ks]));
+                            mma_mxf4_ts_if(issue, d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
+                        mma_commit_if(issue, smem_u32(&ctl->empty_a[sa]));
+                        if (hand_over) mma_commit_if(issue, smem_u32(&ctl->b_free[ks]));
 #pragma unroll
                         for (int j = 0; j < BK / 64; ++j)
-                            mma_mxf4_ts(d, ta2 + 8 * j, db + kStepS + j * kStepJ, idesc, sfa, sfb, 1u);
-                        mma_commit(smem_u32(&ctl->empty_a[sa2]));
-                        if (hand_over) mma_commit(smem_u32(&ctl->b_free[ks + 1]));
+                            mma_mxf4_ts_if(issue, d, ta2 + 8 * j, db + kStepS + j * kStepJ, idesc, sfa, sfb, 1u);
+                        mma_commit_if(issue, smem_u32(&ctl->empty_a[sa2]));
+                        if (hand_over) mma_commit_if(issue, smem_u32(&ctl->b_free[ks + 1]));
                         db += 2 * kStepS;
                         sa = sa2; pa = pa2;
                         if (++sa == C::A_STAGES) { sa = 0; pa ^= 1u; }
@@ -404,13 +406,13 @@ xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ 
                             const uint32_t ta = tmem_a + sa * A_COLS;
 #pragma unroll
                             for (int j = 0; j < BK / 64; ++j)
-                                mma_mxf4_ts(d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
-                            mma_commit(smem_u32(&ctl->empty_a[sa]));
-                            if (hand_over) mma_commit(smem_u32(&ctl->b_free[ks]));
+                                mma_mxf4_ts_if(issue, d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
+                            mma_commit_if(issue, smem_u32(&ctl->empty_a[sa]));
+                            if (hand_over) mma_commit_if(issue, smem_u32(&ctl->b_free[ks]));
                             if (++sa == C::A_STAGES) { sa = 0; pa ^= 1u; }
                         }
                     }
-                    if (ok) mma_commit(smem_u32(&ctl->acc_full[b]));
+                    if (ok) mma_commit_if(issue, smem_u32(&ctl->acc_full[b]));
                 }
             }
         }
