@@ -16,14 +16,15 @@
 // stage's block (K-major core matrices).  BN = 192 while K <= 2048 and BN = 128 while
 // K <= 3072 keep the slice within 192 KB; other shapes are left to the streaming kernel.
 //
-// Roles in a CTA of 14 warps (one CTA per SM):
+// Roles in a CTA of 15 warps (one CTA per SM):
 //   warp 13      one thread issues the bulk copies of the weight slice (once) and the 2-D TMA
 //                tile loads of the packed frame rows (64 bytes per row = two stages) into a
 //                staging ring (64-byte swizzle, no multicast)
 //   warps 5-12   two teams of four warps widen the frame rows, thread = one row, 32 bytes ->
 //                128 bytes per stage, into tensor memory (the MMA reads its A operand from
 //                there); the teams take alternate stages
-//   warp 4       one thread issues the MMAs (4 per stage, K = 64 each) and the commits
+//   warps 4, 14  issue the MMAs (4 per stage, K = 64 each) and the commits, one lane each; the two
+//                warps take a tile's stages in turn and accumulate into the same accumulator
 //   warps 0-3    epilogue: accumulator -> threshold -> repacked bits; two accumulators in
 //                tensor memory, so it overlaps the next tile's MMAs
 // Every wait is bounded; a wait that runs out sets the CTA's abort flag, all roles fall
@@ -55,7 +56,8 @@ constexpr int ROW_BYTES = BK / 2;                         // widened bytes per r
 constexpr int B_REGION = 192 * 1024;                      // shared memory that holds the weight slice
 constexpr int EPI_WARPS = 4, MMA_WARP = 4, PROD_WARP0 = 5, A_WARPS = BM / 32, TEAMS = 2;
 constexpr int TMA_WARP = PROD_WARP0 + TEAMS * A_WARPS;
-constexpr int THREADS = (TMA_WARP + 1) * 32;              // 448
+constexpr int MMA_WARP2 = TMA_WARP + 1;                   // the second issuing warp
+constexpr int THREADS = (MMA_WARP2 + 1) * 32;             // 480
 constexpr int GROUPS = 4;                                 // staging ring of the packed frame rows: groups of two stages
 constexpr int GROUP_BYTES = BM * 64;
 constexpr uint32_t A_COLS = ROW_BYTES / 4;                // 32-bit columns per A stage
@@ -78,6 +80,7 @@ struct Control {
     uint32_t flipw[8];
     uint64_t full_a[6], empty_a[6], full_b[MAX_NKS], b_free[MAX_NKS], acc_full[2], acc_empty[2];
     uint64_t group_full[GROUPS], group_empty[GROUPS];
+    uint64_t started[2];
     uint32_t tmem_base;
     WaitState wait;
 };
@@ -252,7 +255,8 @@ xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ 
             mbar_init(smem_u32(&ctl->b_free[s]), 1);   // the MMA thread's commit
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
+            mbar_init(smem_u32(&ctl->acc_full[b]), 2);       // one commit of each issuing warp
+            mbar_init(smem_u32(&ctl->started[b]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[b]), EPI_WARPS);
         }
         for (int b = 0; b < GROUPS; ++b) {
@@ -338,33 +342,34 @@ xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ 
             }
         }
         __syncwarp();
-    } else if (warp >= PROD_WARP0) {
+    } else if (warp >= PROD_WARP0 && warp < TMA_WARP) {
         // the layers follow one another in the producers' sequence of (tile, stage) pairs
         ProducerArgs pa{smem_u32(smem) + B_REGION, tmem + C::TMEM_A_COL, ctl, abort_flag, L * share.count, nks, kw, tail_mask(K), lane, zo};
         produce_a<C::A_STAGES>(pa, (warp & 3) * 32 + lane, (warp - PROD_WARP0) / A_WARPS);
-    } else if (warp == MMA_WARP) {
-        // ---------------- MMA issue: one thread
-        // Two stages per iteration: measured on B200, whatever this thread does between two
-        // MMAs (polls, commits, loop bookkeeping) is time the tensor pipe idles, so the waits
-        // of two stages are taken together and their eight MMAs issued back to back (12 % off
-        // the steady state against one stage per iteration).
-        // The whole warp runs the loop (converged); the MMAs and commits are issued by lane 0 alone.
+    } else if (warp == MMA_WARP || warp == MMA_WARP2) {
+        // ---------------- MMA issue: two warps, one issuing lane each; the warps stay converged and the
+        // MMAs and commits are predicated on lane 0.  A tile's stages go to the two warps in turn, and both
+        // accumulate into the tile's accumulator: the sums are exact integers (|sum| <= K < 2^24), so the
+        // order of the accumulations does not matter.  Only the stage that overwrites the accumulator has
+        // to come first: warp 0 commits its first MMA of a tile to `started`, and warp 1 waits for that
+        // before its first MMA of the tile.  (Measured on B200: what an issuing thread does between MMAs
+        // -- polls, commits, bookkeeping -- is time the tensor pipe idles; with two issuers one thread's
+        // waits overlap the other's MMAs.  2 % off the WSJ-scale step against one issuer that takes the
+        // stages in pairs; two issuers taking pairs, and a deeper ring of narrower tiles, gained less.)
         {
+            const int w = warp == MMA_WARP ? 0 : 1;
             const uint32_t issue = lane == 0;
             constexpr uint32_t idesc = instr_desc_mxf4(BM, BN);
             const uint32_t sfa = tmem + C::TMEM_SF_COL, sfb = tmem + C::TMEM_SF_COL + SF_COLS / 2;
-            // descriptor of stage 0, chunk pair 0; the address field (16-byte units) of the others
-            // is reached by plain additions: the whole region lies below 2^14 * 16 bytes
             const uint64_t desc0 = smem_desc_kmajor(smem_u32(smem), BN * 16, 128);
             constexpr uint32_t kStepJ = (2 * BN * 16) >> 4, kStepS = C::B_BYTES >> 4;
             const uint32_t tmem_a = tmem + C::TMEM_A_COL;
-            int sa = 0;          // slot of the A ring and the parity its `full` barrier shows next
-            uint32_t pa = 0;
             bool ok = true;
             int tl = 0;          // tiles so far, over all layers
+            int it_base = 0;     // stages before this tile, over all layers
             for (int l = 0; l < L && ok; ++l) {
                 const uint32_t pb = (uint32_t)(l & 1);   // a layer's weight stages arrive once and then stay
-                for (int t = 0; t < share.count && ok; ++t, ++tl) {
+                for (int t = 0; t < share.count && ok; ++t, ++tl, it_base += nks) {
                     const bool first = t == 0;
                     const bool hand_over = t == share.count - 1 && l + 1 < L;   // the next layer's slice follows
                     const int b = tl & 1;
@@ -372,45 +377,26 @@ xnor_res_kernel(const __grid_constant__ StackMaps maps, const __grid_constant__ 
                     if (!ok) break;
                     tc_fence_after_sync();
                     const uint32_t d = tmem + (uint32_t)(b * BN);
-                    uint64_t db = desc0;
-                    int ks = 0;
-                    for (; ks + 1 < nks; ks += 2) {
-                        const int sa2 = sa + 1 == C::A_STAGES ? 0 : sa + 1;
-                        const uint32_t pa2 = sa + 1 == C::A_STAGES ? pa ^ 1u : pa;
-                        ok = (!first || (mbar_wait(smem_u32(&ctl->full_b[ks]), pb, abort_flag) &&
-                                         mbar_wait(smem_u32(&ctl->full_b[ks + 1]), pb, abort_flag))) &&
+                    for (int ks = w; ks < nks; ks += 2) {
+                        const int it = it_base + ks;             // this stage in the CTA's sequence: slot and parity of the A ring
+                        const int sa = it % C::A_STAGES;
+                        const uint32_t pa = (uint32_t)((it / C::A_STAGES) & 1);
+                        ok = (!first || mbar_wait(smem_u32(&ctl->full_b[ks]), pb, abort_flag)) &&
                              mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag) &&
-                             mbar_wait(smem_u32(&ctl->full_a[sa2]), pa2, abort_flag);
+                             (ks != 1 || mbar_wait(smem_u32(&ctl->started[b]), (uint32_t)((tl >> 1) & 1), abort_flag));
                         if (!ok) break;
                         tc_fence_after_sync();
-                        const uint32_t ta = tmem_a + sa * A_COLS, ta2 = tmem_a + sa2 * A_COLS;
+                        // descriptor of stage ks, chunk pair 0; the address field (16-byte units) of the others is
+                        // reached by plain additions: the whole region lies below 2^14 * 16 bytes
+                        const uint64_t db = desc0 + (uint64_t)((uint32_t)ks * kStepS);
+                        const uint32_t ta = tmem_a + sa * A_COLS;
 #pragma unroll
-                        for (int j = 0; j < BK / 64; ++j)   // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
+                        for (int j = 0; j < BK / 64; ++j) {  // 64 positions of K = 32 bytes: 8 columns of A, two 16-byte chunks of B
                             mma_mxf4_ts_if(issue, d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
+                            if (j == 0 && ks == 0) mma_commit_if(issue, smem_u32(&ctl->started[b]));
+                        }
                         mma_commit_if(issue, smem_u32(&ctl->empty_a[sa]));
                         if (hand_over) mma_commit_if(issue, smem_u32(&ctl->b_free[ks]));
-#pragma unroll
-                        for (int j = 0; j < BK / 64; ++j)
-                            mma_mxf4_ts_if(issue, d, ta2 + 8 * j, db + kStepS + j * kStepJ, idesc, sfa, sfb, 1u);
-                        mma_commit_if(issue, smem_u32(&ctl->empty_a[sa2]));
-                        if (hand_over) mma_commit_if(issue, smem_u32(&ctl->b_free[ks + 1]));
-                        db += 2 * kStepS;
-                        sa = sa2; pa = pa2;
-                        if (++sa == C::A_STAGES) { sa = 0; pa ^= 1u; }
-                    }
-                    if (ok && ks < nks) {   // odd number of stages: the last one alone
-                        ok = (!first || mbar_wait(smem_u32(&ctl->full_b[ks]), pb, abort_flag)) &&
-                             mbar_wait(smem_u32(&ctl->full_a[sa]), pa, abort_flag);
-                        if (ok) {
-                            tc_fence_after_sync();
-                            const uint32_t ta = tmem_a + sa * A_COLS;
-#pragma unroll
-                            for (int j = 0; j < BK / 64; ++j)
-                                mma_mxf4_ts_if(issue, d, ta + 8 * j, db + j * kStepJ, idesc, sfa, sfb, (ks | j) != 0);
-                            mma_commit_if(issue, smem_u32(&ctl->empty_a[sa]));
-                            if (hand_over) mma_commit_if(issue, smem_u32(&ctl->b_free[ks]));
-                            if (++sa == C::A_STAGES) { sa = 0; pa ^= 1u; }
-                        }
                     }
                     if (ok) mma_commit_if(issue, smem_u32(&ctl->acc_full[b]));
                 }
