@@ -308,7 +308,8 @@ typedef struct bnn_model {
 
 /* Bytes of scratch for M frames.  bnn_forward_workspace_bytes is what makes bnn_forward
  * fastest: two ping-pong activation buffers, the arrival counters of binary hidden layers that
- * run as one launch (a few bytes per 128 frames and layer), and room for the split-activation
+ * run as one launch (a few bytes per 128 frames and layer) and of the log-softmax that follows the
+ * top layer's kernel (4 bytes per 512 frames), and room for the split-activation
  * images: of the widest sign-weight layer (see bnn_signw_gemm_ws; two of them when such layers
  * follow one another, because each writes the next one's image while it reads its own) or of a
  * real-valued layer fed with fp32 activations (see bnn_output_layer_ws).
