@@ -345,8 +345,8 @@ BNN_API int bnn_forward(const bnn_model* model, const float* X, int ldx, int M,
  *   - Inputs and outputs (model, X, logp) are still the caller's.
  *   - Limit: bnn_forward_min_workspace_bytes(model, M) must not exceed the array; otherwise the
  *     call launches nothing and returns BNN_ERR_WORKSPACE.  (For a 2048-wide network 8 MiB holds
- *     16376 frames of binary activations -- the activation buffers plus the counters of the stacked
- *     binary layers -- or 512 frames of fp32 hardtanh activations.)
+ *     16379 frames of binary activations -- the activation buffers plus the counters of the stacked
+ *     binary layers and of the log-softmax that follows the top layer -- or 511 frames of fp32 hardtanh activations.)
  *   - This call makes no cudaMalloc/cudaFree and uses no allocating library routine.
  *   - The first call on each device looks up the array's device address (with that device
  *     current), and the CUDA runtime may load this library's device code -- the array with it --
