@@ -176,15 +176,16 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ roofline bookkeeping
-def xnor_kernel_name(k, xnor_path, prepared):
-    """The kernel bnn_forward runs for a binary hidden layer of fan-in k (see bnn_api.cu)."""
+def xnor_kernel_name(k, xnor_path, prepared, stacked=True):
+    """The kernel bnn_forward runs for a binary hidden layer of fan-in k (see bnn_api.cu); `stacked`: the
+    layer is one of a run of equal layers that goes out as one launch."""
     if xnor_path == "popc":
         return "xnor_popc_kernel"
     if xnor_path == "tensor-unprepared":
         return "xnor_tc_kernel"
     if prepared == "stream":
         return "xnor_img_kernel"
-    if k <= 2048 or (prepared == "resident" and k <= 3072):
+    if k <= 2048 or (k <= 3072 and (prepared == "resident" or stacked)):
         return "xnor_res_kernel"
     return "xnor_tc_kernel"
 
@@ -200,7 +201,7 @@ def choose_tensor_regime(peaks, clocks, timed_s):
     return "burst", peaks["bf16_tflops"], why
 
 
-def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tensor", prepared="auto"):
+def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tensor", prepared="auto", stacked=True):
     """Per layer: algorithmic work, the pipe that bounds the kernel and its peak.
 
     peaks["bf16"] is the bf16 figure chosen for this run (burst or sustained); peaks["mxf4"] the
@@ -244,7 +245,7 @@ def layer_table(cfg, frames, peaks, sm_mhz, xnor_path="tensor", real_path="tenso
             tiles_m, tiles_n = -(-frames // 128), -(-cfg.hidden // 192)
             kpad = -(-k // 256) * 256
             smem_bytes = tiles_m * tiles_n * kpad * (192 * (0.5 + 0.5 + 0.125 + 0.125) + 128 * (0.125 + 0.125))
-            kern = xnor_kernel_name(k, xnor_path, prepared)
+            kern = xnor_kernel_name(k, xnor_path, prepared, stacked and cfg.n_hidden > 2)
             if kern == "xnor_img_kernel":
                 # weights prepared once: their widened image arrives by bulk copies (4 bits written,
                 # 4 bits read by the tensor core per weight bit and tile visit); nothing else
@@ -508,7 +509,8 @@ def run_ours(args):
         torch.cuda.synchronize()
         mxf4_rate = work / (e0.elapsed_time(e1) / 3 * 1e-3) / 1e12
     peaks["mxf4"] = mxf4_rate or 4.0 * bf16_peak
-    rows = layer_table(cfg, frames, peaks, ck.get("sm_mhz"), args.xnor_path, args.real_path, args.xnor_prepared)
+    rows = layer_table(cfg, frames, peaks, ck.get("sm_mhz"), args.xnor_path, args.real_path, args.xnor_prepared,
+                       stacked=not args.no_stack)
     assert len(rows) == len(layer_ms)
     for r, t in zip(rows, layer_ms):
         r["ms"] = t

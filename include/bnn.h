@@ -384,7 +384,10 @@ BNN_API int bnn_forward_events(const bnn_model* model, const float* X, int ldx, 
  *                        layers) runs for a fused Sign layer: BNN_PREPARED_STREAM reads the
  *                        weight image from L2 for every tile of frames; BNN_PREPARED_RESIDENT
  *                        keeps a tile of units' weights in shared memory for the whole launch
- *                        (needs K <= 3072; other shapes stream); AUTO picks by shape.
+ *                        (needs K <= 3072; other shapes stream); AUTO picks by shape (resident for
+ *                        K <= 2048; for a single layer of larger fan-in the kernel that widens the packed
+ *                        weights on the fly; runs of equal layers, see BNN_OPT_XNOR_STACK, are resident
+ *                        up to K = 3072).
  *   BNN_OPT_SMALL_BATCH: 1 (default) lets bnn_forward run batches of up to 16 frames -- the
  *                        matrix-vector regime the paper has in mind for embedded recognisers
  *                        (Section 1) -- on kernels that spread each layer's weights over all SMs,

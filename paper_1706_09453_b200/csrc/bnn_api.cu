@@ -99,14 +99,17 @@ int validate_model(const bnn_model* model) {
 }
 
 // Whether hidden layer l can be part of a run launched as one kernel: a fused Sign layer on packed
-// input with prepared weights, of a shape the resident-weights kernel takes on its fast tiles.
+// input with prepared weights, of a shape the resident-weights kernel takes (fan-in up to 3072).  As
+// ONE launch of several layers that kernel also wins on its narrow tiles (fan-in above 2048: AMI-scale
+// hidden layers 1.70 ms for five against 5 x 0.39 for the kernel that widens both operands on the fly);
+// a single such layer is left to bnn_xnor_gemm_prepared's own choice.
 bool stackable(const bnn_model* model, int l) {
     const bnn_layer& y = model->layers[l];
     if (y.kind != BNN_LAYER_XNOR || y.act != BNN_ACT_SIGN_PACK || !y.W_prepared) return false;
     if (g_xnor_path == BNN_PATH_CUDA_CORE || g_xnor_prepared == BNN_PREPARED_STREAM || y.K > kMaxKTensor) return false;
     if (reinterpret_cast<uintptr_t>(y.W_prepared) & 255u) return false;
     if (!xnor_res_applicable(y.N, y.K)) return false;
-    return y.K <= 2048 || g_xnor_prepared == BNN_PREPARED_RESIDENT;
+    return true;
 }
 
 }  // namespace
