@@ -156,6 +156,7 @@ def test_forward_stacked_hidden_layers_edge_shapes(env, hidden, n_hidden, frames
     (2100, 4000, 0, False),   # 5 frame groups x 32 class tiles, ragged last group, the wide-row variant
     (4700, 2000, 1, True),    # 10 groups x 16 class tiles, the narrow-row variant; (0,1) activations; log-prior
     (2561, 3400, 0, True),    # one frame in the last group
+    (2100, 4100, 0, False),   # more classes than the following kernel holds in registers: the kernels run one after the other
 ])
 def test_forward_log_softmax_following_the_top_layer(env, frames, classes, values, with_prior):
     """The log-softmax launched behind the top layer's kernel, taking each group of 512 frames as soon as
@@ -186,6 +187,11 @@ def test_forward_log_softmax_following_the_top_layer(env, frames, classes, value
     assert (a - b).abs().max().item() <= 1e-5
     for _ in range(3):   # the counters are cleared by every call
         assert torch.equal(dn.forward(Xd), a)
+    # rows of the output that are not 16-byte aligned: the following kernel does not apply, same result
+    wide = torch.full((frames, classes + 3), 7.0, dtype=torch.float32, device="cuda:0")
+    c = dn.forward(Xd, logp=wide[:, :classes])
+    assert (c - a).abs().max().item() <= 1e-5
+    assert bool((wide[:, classes:] == 7.0).all())
     assert B.bnn_device_status() == 0
 
 
