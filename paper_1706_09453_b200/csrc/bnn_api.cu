@@ -301,7 +301,9 @@ static int signw_impl(const float* X, int ldx, const uint32_t* Wp, int ldwp,
                       int M, int N, int K, float* Y, int ldy,
                       const bnn_epilogue* epi, void* workspace, size_t workspace_bytes,
                       int splice_dim, int splice_left, void* stream,
-                      bool image_ready = false, void* out_image = nullptr, int out_kind = 0) {
+                      bool image_ready = false, void* out_image = nullptr, int out_kind = 0,
+                      int* clear = nullptr, int clear_words = 0, bool* cleared = nullptr) {
+    if (cleared) *cleared = false;
     if (int rc = check_dims(M, N, K)) return rc;
     if (!X && !image_ready) return BNN_ERR_NULL;
     if (ldx < (splice_dim > 0 ? splice_dim : K)) return BNN_ERR_SHAPE;
@@ -328,8 +330,13 @@ static int signw_impl(const float* X, int ldx, const uint32_t* Wp, int ldwp,
     if (!a.Y && !a.out_bits && !out_image) return BNN_ERR_NULL;
     if (g_real_path != BNN_PATH_CUDA_CORE) {
         if (workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255u) &&
-            workspace_bytes >= signw_image_bytes(M, K, g_signw_terms))
-            return launch_signw_img(a, g_signw_terms, workspace, image_ready, out_image, out_kind, (cudaStream_t)stream);
+            workspace_bytes >= signw_image_bytes(M, K, g_signw_terms)) {
+            // the kernel that splits the activations can clear the caller's counters on its way
+            const bool clears = clear && clear_words > 0 && !image_ready;
+            if (cleared) *cleared = clears;
+            return launch_signw_img(a, g_signw_terms, workspace, image_ready, out_image, out_kind,
+                                    clears ? clear : nullptr, clears ? clear_words : 0, (cudaStream_t)stream);
+        }
         if (splice_dim > 0 || image_ready || out_image) return BNN_ERR_WORKSPACE;
         return launch_signw_tc(a, g_signw_terms, (cudaStream_t)stream);
     }
@@ -548,6 +555,7 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
     // would take away its programmatic overlap with the first layer's tail.
     // The same goes for the counters on which the log-softmax follows the top layer's kernel.
     int* top_done = nullptr;
+    bool clear_pending = false, clear_by_first = false;
     if (!small && lay.sync > 0) {
         bool any = false;
         for (int l = 0; g_xnor_stack && l + 1 < L && !any; ++l)
@@ -557,7 +565,14 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
         if (g_softmax_follow && !events && lay.sync > lay.stack_sync && top.kind == BNN_LAYER_REAL_OUT && top.W_prepared &&
             L > 1 && model->layers[L - 2].act == BNN_ACT_SIGN_PACK && out_tc_more_than_one_wave(M, top.N))
             top_done = sync + lay.stack_sync / sizeof(int);
-        if ((any || top_done) && cudaMemsetAsync(sync, 0, lay.sync, (cudaStream_t)stream) != cudaSuccess) return BNN_ERR_CUDA;
+        clear_pending = any || top_done;
+        // When the first layer splits its input into an image, that kernel clears them on its way (a memset
+        // node of its own costs about 4 us per step in a replayed graph); otherwise a memset does.
+        clear_by_first = clear_pending && model->layers[0].kind == BNN_LAYER_SIGNW && g_real_path != BNN_PATH_CUDA_CORE;
+        if (clear_pending && !clear_by_first) {
+            if (cudaMemsetAsync(sync, 0, lay.sync, (cudaStream_t)stream) != cudaSuccess) return BNN_ERR_CUDA;
+            clear_pending = false;
+        }
     }
     bool chain_in = false;   // the layer before wrote this layer's split-activation image (slot chain_slot)
     int chain_slot = 0;
@@ -672,9 +687,17 @@ int bnn_forward_events(const bnn_model* model, const float* X, int ldx, int M,
                 if (!chain_out || (layer_out && layer_out[l])) yf = static_cast<float*>(out);
                 out_ld = y.N;
             }
+            bool cleared = false;
             rc = signw_impl(static_cast<const float*>(in), in_ld, y.Wp, y.ldwp, M, y.N, y.K,
                             yf, y.N, &e, img_in, chain_in ? img_half : (chain_out ? img_half : img_bytes),
-                            l == 0 ? splice_dim : 0, model->splice_left, stream, chain_in, img_out, to_real ? 1 : 0);
+                            l == 0 ? splice_dim : 0, model->splice_left, stream, chain_in, img_out, to_real ? 1 : 0,
+                            (l == 0 && clear_by_first) ? sync : nullptr, (int)(lay.sync / sizeof(int)), &cleared);
+            if (l == 0 && clear_pending) {
+                // the layer took another kernel than the one that clears the counters: clear them now
+                if (rc == BNN_OK && !cleared && cudaMemsetAsync(sync, 0, lay.sync, (cudaStream_t)stream) != cudaSuccess)
+                    return BNN_ERR_CUDA;
+                clear_pending = false;
+            }
             in_ld = out_ld;
             if (chain_out) chain_slot = (chain_in ? chain_slot : 0) ^ 1;
             chain_in = chain_out;

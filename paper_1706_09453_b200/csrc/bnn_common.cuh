@@ -195,8 +195,10 @@ size_t signw_image_bytes(int M, int K, int terms);
 // written as the image of a following layer of this kind with fan-in N.
 // out_kind 0: that layer's own image (bf16 terms, blocks of 128 frames); 1: the image the real-valued
 // layer on fp32 activations reads (two fp16 terms, blocks of 256 frames, outf_image_bytes(M, N) bytes).
+// clear / clear_words (optional, only with image_ready == false): words the splitting kernel sets to zero on
+// its way -- bnn_forward's counters, which would otherwise need a memset of their own in front of it.
 int launch_signw_img(const RealGemmArgs& a, int terms, void* workspace, bool image_ready, void* out_image, int out_kind,
-                     cudaStream_t st);
+                     int* clear, int clear_words, cudaStream_t st);
 size_t out_prepared_bytes(int C, int H);
 int launch_out_prepare(const float* W, int ldw, int C, int H, void* prepared, cudaStream_t st);
 // `done` (optional, out_tc_done_bytes(M) zeroed bytes): one counter per out_tc_group_rows() frames, then

@@ -71,9 +71,12 @@ __device__ __forceinline__ float bf16_hi_as_float(uint32_t w) { return __uint_as
 template <int NT>
 __global__ void __launch_bounds__(256)
 x_split_kernel(const float* __restrict__ X, int ldx, int M, int K, int nks, uint8_t* __restrict__ img,
-               int sdim, int sleft) {
+               int sdim, int sleft, int* __restrict__ clear, int clear_words) {
     __shared__ float raw[BM][BK + 1];
     pdl_trigger();   // the GEMM may be scheduled as SMs free up; it waits before it reads the image
+    // As the first kernel of a forward pass this one also clears the pass's counters (a few hundred
+    // words): a memset node of its own in front of it costs about 4 us per step.
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < clear_words; i += gridDim.x * blockDim.x) clear[i] = 0;
     const int mt = blockIdx.x / nks, ks = blockIdx.x % nks;
     const int t = threadIdx.x;
     // coalesced read: 8 consecutive threads fetch the 32 floats of one row segment.  With splicing
@@ -555,7 +558,8 @@ __global__ void __launch_bounds__(THREADS, 1) signw_img_kernel(Args g) {
 }
 
 template <int NT>
-int launch_nt(const RealGemmArgs& r, void* workspace, bool image_ready, void* out_image, int out_kind, cudaStream_t st) {
+int launch_nt(const RealGemmArgs& r, void* workspace, bool image_ready, void* out_image, int out_kind, int* clear,
+              int clear_words, cudaStream_t st) {
     using C = Cfg<NT>;
     constexpr int SMEM = C::STAGES * C::STAGE_BYTES + (int)sizeof(Control) + 128;
     const int sms = device_sm_count();
@@ -565,7 +569,8 @@ int launch_nt(const RealGemmArgs& r, void* workspace, bool image_ready, void* ou
     // (when the kernel before this one in the stream already wrote the image -- the layer that produced
     // these activations -- there is nothing to split)
     if (!image_ready)
-        x_split_kernel<NT><<<mt * nks, 256, 0, st>>>(r.Af, r.lda, r.M, r.K, nks, img, r.splice_dim, r.splice_left);
+        x_split_kernel<NT><<<mt * nks, 256, 0, st>>>(r.Af, r.lda, r.M, r.K, nks, img, r.splice_dim, r.splice_left, clear,
+                                                     clear ? clear_words : 0);
     Args a{static_cast<uint8_t*>(out_image), ceil_div(r.N, BK), out_kind, img, r.Bb, r.ldb, r.M, r.N, r.K, r.scale, r.shift, r.act, r.sign_mode, r.Y, r.ldy, r.out_bits, r.ldob,
            tc_status()};
     if (!a.status.word) return BNN_ERR_CUDA;
@@ -582,9 +587,10 @@ size_t signw_image_bytes(int M, int K, int terms) {
 }
 
 int launch_signw_img(const RealGemmArgs& r, int terms, void* workspace, bool image_ready, void* out_image, int out_kind,
-                     cudaStream_t st) {
-    return terms == 3 ? launch_nt<3>(r, workspace, image_ready, out_image, out_kind, st)
-                      : launch_nt<2>(r, workspace, image_ready, out_image, out_kind, st);
+                     int* clear, int clear_words, cudaStream_t st) {
+    if (clear && image_ready) return BNN_ERR_UNSUPPORTED;   // no split kernel runs: nobody to clear the words
+    return terms == 3 ? launch_nt<3>(r, workspace, image_ready, out_image, out_kind, clear, clear_words, st)
+                      : launch_nt<2>(r, workspace, image_ready, out_image, out_kind, clear, clear_words, st);
 }
 
 }  // namespace bnn
